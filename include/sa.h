@@ -1,0 +1,206 @@
+/* sa.h — C ABI of the shift-accumulate decode-attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes decode-time attention of one query vector per head against a key
+ * cache stored as signed power-of-two fixed-point codes, after "Shift-Accumulate Attention:
+ * Multiplier-Free Query-Key Products for Transformer Decoding".  Citations below name the
+ * paper's sections and equations.
+ *
+ * General rules for every function
+ *   - `extern "C"`, returns an sa_status, never throws, never aborts.
+ *   - Pointers are DEVICE pointers unless the parameter name ends in `_host`.  All memory is
+ *     owned by the caller; the library allocates no device memory and keeps no state.
+ *   - Work is enqueued on the caller's stream (`sa_stream` is a `cudaStream_t`); no function
+ *     synchronises.  Arguments are validated on the host before anything is launched; a call
+ *     that returns an error has launched nothing.
+ *   - Half-precision data is passed as IEEE binary16 bit patterns in `uint16_t`.
+ *   - Inputs must be finite.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *
+ * Number formats (section II-A, II-D, II-E)
+ *   Key element  K^_jm = s_j * sigma * (1 + j/2^k) * 2^-e,  e in 0..6, code e = 7 is an exact
+ *   zero, k in {0, 1, 2, 4} mantissa bits (PoT-4, PoT-M1, PoT-M2, PoT-M4), s_j = the key
+ *   vector's largest magnitude (binary16).  Rounding is to the nearest codeword in log2 on the
+ *   grid continued below e = 6; an element that rounds to e >= 7 becomes the zero code.
+ *   Canonical code byte: bit 7 sign (1 = negative), bits 6..4 e, bits 3..0 the mantissa
+ *   left-aligned (j << (4 - k)); zero is 0x70.
+ *   Query  Q_im ~ Delta_i * qhat_im, qhat in [-127, 127], Delta_i = amax_i / 127.
+ *   Value  V_jm ~ vhat_jm * 2^-g_j, vhat INT8, g_j the largest integer with amax_j * 2^g_j <= 127.
+ *
+ * Cache layout (this library's own; section II-F only fixes what is stored)
+ *   The page pool is n_pages * n_kv_heads blocks of `page_bytes`; block (p, h) starts at
+ *   ((size_t)p * n_kv_heads + h) * page_bytes and holds page_tokens = 64 tokens of KV head h:
+ *     kcode_off: key codes in 16-byte chunks, chunk c of token t at (c * 64 + t) * 16.
+ *                Byte container (any k): chunk c holds elements 16c .. 16c+15, one canonical
+ *                byte each.  Nibble container (PoT-4 only): chunk c holds elements 32c .. 32c+31,
+ *                byte i = element 32c+2i in the low nibble and 32c+2i+1 in the high nibble,
+ *                nibble = sign << 3 | e.
+ *     meta_off : 64 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.
+ *     v_off    : vhat, int8, row-major [64][head_dim].
+ *   For code = SA_KV_FP16 the block holds unquantised binary16 data: K in 16-byte chunks of 8
+ *   elements (chunk c of token t at (c * 64 + t) * 16), no metadata, then V row-major
+ *   [64][head_dim].
+ */
+#ifndef SA_H_
+#define SA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* sa_stream; /* a cudaStream_t; NULL is the default stream */
+
+typedef enum {
+    SA_OK = 0,
+    SA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, inconsistent head counts ...   */
+    SA_ERR_UNSUPPORTED = 2, /* head_dim, code, layout or head-room outside what is implemented */
+    SA_ERR_ALIGNMENT = 3,   /* a pointer is not aligned as documented                          */
+    SA_ERR_CAPACITY = 4,    /* workspace or staging buffer too small, page table too short     */
+    SA_ERR_CUDA = 5         /* the CUDA runtime refused a launch or a copy                     */
+} sa_status;
+
+/* Key code family: the value is k, the number of mantissa bits (eq. (2), eq. (5)). */
+enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_KV_FP16 = 16 };
+/* How key codes are stored in a page. */
+enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1 };
+/* flags */
+#define SA_FLAG_HADAMARD 1u /* rotate Q and K by the normalised Walsh-Hadamard matrix before quantising */
+
+typedef struct {
+    int head_dim;    /* 64 or 128 */
+    int n_q_heads;   /* multiple of n_kv_heads */
+    int n_kv_heads;
+    int code;        /* SA_POT4 / SA_POTM1 / SA_POTM2 / SA_POTM4, or SA_KV_FP16 for the FP16 baseline cache */
+    int klayout;     /* SA_KLAYOUT_BYTE, or SA_KLAYOUT_NIBBLE (only with SA_POT4) */
+    int headroom_F;  /* fixed-point head-room F of eq. (3); 0 selects the default E + k = 6 + k.
+                        Must satisfy F >= 6 + k (eq. (4): every shift is a left shift) and
+                        head_dim * 127 * (2^(k+1) - 1) * 2^(F - k) < 2^31 (INT32 accumulator) */
+    int page_tokens; /* 64 */
+    unsigned flags;  /* SA_FLAG_HADAMARD */
+} sa_config;
+
+typedef struct {
+    size_t page_bytes; /* bytes of one (page, KV head) block */
+    size_t kcode_off;  /* offsets inside a block */
+    size_t meta_off;
+    size_t v_off;
+    size_t align;      /* required alignment of the pool base pointer */
+} sa_layout;
+
+typedef struct {
+    void* pages;               /* page pool, n_pages * n_kv_heads * page_bytes bytes                     */
+    const int32_t* page_table; /* [batch, max_pages_per_seq]: pool index of each sequence's logical page */
+    int32_t* seq_lens;         /* [batch]: tokens already cached per sequence                            */
+    int batch;
+    int max_pages_per_seq;
+    int n_pages;
+} sa_cache;
+
+int sa_version(void);
+const char* sa_status_string(sa_status s);
+
+/* Byte layout of one (page, KV head) block for this configuration.  Host only, no CUDA call. */
+sa_status sa_get_layout(const sa_config* cfg, sa_layout* out);
+
+/* Bytes of scratch that sa_decode_attention / sa_decode_attention_fp16 need for a cache with
+ * `batch` sequences of at most `max_pages_per_seq` pages (split-K partial results, section II-F:
+ * the kernel grid has a split dimension).  Host only, no CUDA call.  The scratch needs no
+ * initialisation and may be shared by calls that do not overlap on the GPU. */
+sa_status sa_workspace_bytes(const sa_config* cfg, int batch, int max_pages_per_seq, size_t* out);
+
+/* Key encode (eq. (2), eq. (5); nearest-in-log2 rounding, section II-D).
+ * K [n, n_kv_heads, head_dim] binary16 -> codes [n, n_kv_heads, head_dim] canonical bytes and
+ * scales [n, n_kv_heads] binary16.  With SA_FLAG_HADAMARD each head vector is rotated first. */
+sa_status sa_encode_keys(const sa_config* cfg, const uint16_t* K, int64_t n, uint8_t* codes,
+                         uint16_t* scales, sa_stream stream);
+
+/* Query quantisation (eq. (2)): Q [batch, n_q_heads, head_dim] binary16 -> q_hat int8 of the same
+ * shape and delta [batch, n_q_heads] float.  With SA_FLAG_HADAMARD each head vector is rotated first. */
+sa_status sa_quantise_query(const sa_config* cfg, const uint16_t* Q, int batch, int8_t* q_hat,
+                            float* delta, sa_stream stream);
+
+/* Value quantisation (section II-E: INT8 with a power-of-two per-token scale).
+ * V [n, n_kv_heads, head_dim] binary16 -> v_hat int8 of the same shape and g [n, n_kv_heads] int8. */
+sa_status sa_quantise_values(const sa_config* cfg, const uint16_t* V, int64_t n, int8_t* v_hat,
+                             int8_t* g, sa_stream stream);
+
+/* Append one token per sequence (the cache write of section II-F: the cache stores only
+ * quantised data).  K_new, V_new [batch, n_kv_heads, head_dim] binary16.  Sequence b's token
+ * is encoded / quantised as above and written at position seq_lens[b] of its page
+ * page_table[b][seq_lens[b] / 64]; the page must already be mapped.  If bump_lens is non-zero
+ * the kernel then increments seq_lens[b]; otherwise the caller does.  With code = SA_KV_FP16 the
+ * binary16 data is stored as is. */
+sa_status sa_append_kv(const sa_config* cfg, const sa_cache* cache, const uint16_t* K_new,
+                       const uint16_t* V_new, int bump_lens, sa_stream stream);
+
+/* Bulk build of a cache: K, V [sum_b T_b, n_kv_heads, head_dim] binary16, sequence b occupying
+ * rows cu_lens_host[b] .. cu_lens_host[b+1] (HOST array of batch + 1 entries).  Writes tokens
+ * 0 .. T_b - 1 of every sequence; does not touch seq_lens. */
+sa_status sa_fill_kv(const sa_config* cfg, const sa_cache* cache, const uint16_t* K,
+                     const uint16_t* V, const int64_t* cu_lens_host, sa_stream stream);
+
+/* Decode attention over the quantised cache — the hot path (section II-B eq. (3), II-C eq. (4),
+ * II-D eq. (5), II-E, II-F):
+ *   Q is quantised (and rotated, if flagged) inside the kernel; for every cached key the integer
+ *   score A = sum_m sigma * qhat * (2^k + j) << (F - k - e) is formed exactly in INT32 with
+ *   shifts, sign flips and adds; logits z = A * Delta * s * 2^-F * log2(e) / sqrt(d) feed an
+ *   online softmax whose running maximum is an integer in the log2 domain, so that every
+ *   rescale is an exact power of two; O accumulates p * vhat * 2^-g in FP32; the key axis is
+ *   split over thread blocks and the partial (M, l, O) triples are merged with exact
+ *   power-of-two factors.
+ * Q [batch, n_q_heads, head_dim] binary16; O [batch, n_q_heads, head_dim] float.
+ * A sequence with seq_lens[b] == 0 yields zeros.
+ * dbg_scores (nullable): int32 [batch, n_q_heads, max_pages_per_seq * 64]; receives A for every
+ * cached key (test hook; slows the call down).
+ * Results are deterministic run to run (fixed split assignment, no floating-point atomics). */
+sa_status sa_decode_attention(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                              float* O, void* workspace, size_t workspace_bytes,
+                              int32_t* dbg_scores, sa_stream stream);
+
+/* The same decode step over an unquantised binary16 cache (cfg->code = SA_KV_FP16): textbook
+ * softmax(Q K^T / sqrt(d)) V of eq. (1) with FP32 accumulation.  Baseline for a like-for-like
+ * throughput ratio (the paper compared with a framework's FP16 attention). */
+sa_status sa_decode_attention_fp16(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                                   float* O, void* workspace, size_t workspace_bytes,
+                                   sa_stream stream);
+
+/* The two decode entry points with their kernels selectable, for callers that want to time or
+ * overlap them separately: stages is a bit mask, 1 = the main kernel (scores, softmax, A.V; writes
+ * the split-K partials into the workspace), 2 = the merge of the partials into O.  stages = 3 is
+ * what sa_decode_attention / sa_decode_attention_fp16 do.  (Measurement hook; the paper's
+ * kernel description in section II-F has no counterpart of the split.) */
+sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                                     float* O, void* workspace, size_t workspace_bytes,
+                                     int32_t* dbg_scores, int stages, sa_stream stream);
+sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const sa_cache* cache,
+                                          const uint16_t* Q, float* O, void* workspace,
+                                          size_t workspace_bytes, int stages, sa_stream stream);
+
+/* Test hook: unpack sequence b of a quantised cache into canonical arrays for its first
+ * n_tokens tokens: codes [n_tokens, n_kv_heads, head_dim] canonical bytes, scales
+ * [n_tokens, n_kv_heads] binary16, v_hat [n_tokens, n_kv_heads, head_dim] int8, g
+ * [n_tokens, n_kv_heads] int8.  Any output pointer may be NULL.  n_tokens is given by the
+ * caller (HOST value) and must not exceed max_pages_per_seq * 64. */
+sa_status sa_debug_unpack(const sa_config* cfg, const sa_cache* cache, int b, int n_tokens,
+                          uint8_t* codes, uint16_t* scales, int8_t* v_hat, int8_t* g,
+                          sa_stream stream);
+
+/* One decode step driven from HOST buffers (convenience for callers whose activations live on
+ * the host): copies Q_host [batch, n_q_heads, head_dim], K_new_host and V_new_host
+ * [batch, n_kv_heads, head_dim] (binary16, ideally pinned) into `staging`, appends the new token
+ * to every sequence (incrementing seq_lens), runs the decode attention matching cfg->code
+ * (quantised or SA_KV_FP16) and copies O [batch, n_q_heads, head_dim] float to O_host.
+ * Everything is asynchronous on `stream`; synchronise it before reading O_host.
+ * `staging` is device scratch of at least sa_staging_bytes(); not shared between overlapping calls. */
+sa_status sa_staging_bytes(const sa_config* cfg, int batch, size_t* out);
+sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q_host,
+                              const uint16_t* K_new_host, const uint16_t* V_new_host, float* O_host,
+                              void* staging, size_t staging_bytes, void* workspace,
+                              size_t workspace_bytes, sa_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SA_H_ */

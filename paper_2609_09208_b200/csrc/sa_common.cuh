@@ -1,0 +1,186 @@
+// Shared declarations of the CUDA library: host-side plan/validation helpers and the small
+// exact-arithmetic device functions used by more than one kernel.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sa.h"
+
+#define SA_HD __host__ __device__ __forceinline__
+#define SA_D __device__ __forceinline__
+
+namespace sa {
+
+constexpr int kPageTokens = 64;
+constexpr int kNumSMs = 148;              // B200
+constexpr int kEmax = 6;                  // largest exponent of the 3-bit field
+constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no key seen yet"
+
+// ---------------------------------------------------------------------------------------------
+// Host-side description of a validated configuration.
+// ---------------------------------------------------------------------------------------------
+struct Plan {
+    int d, Hq, Hkv, G, k;     // k = mantissa bits (0 for SA_KV_FP16)
+    bool fp16, nibble, hadamard;
+    int F;                    // head-room actually used
+    int f_extra;              // F - (6 + k): applied as one final left shift of the INT32 sum
+    sa_layout lay;
+};
+
+sa_status make_plan(const sa_config* cfg, Plan* out);
+// number of splits of the key axis for a cache of this shape, and queries handled per block
+void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt);
+
+// ---------------------------------------------------------------------------------------------
+// Exact helpers (usable on host for unit tests of the arithmetic, and on device).
+// ---------------------------------------------------------------------------------------------
+
+// Normalise a non-zero binary16 magnitude (15 bits) to M * 2^X with M in [1024, 2047].
+SA_HD void half_normalise(uint32_t mag_bits, int* M, int* X) {
+    const int ex = (int)(mag_bits >> 10);
+    const int man = (int)(mag_bits & 0x3ff);
+    if (ex != 0) {
+        *M = 1024 + man;
+        *X = ex - 25;
+    } else {
+#ifdef __CUDA_ARCH__
+        const int sh = __clz(man) - 21;
+#else
+        int sh = 0;
+        while (((man << sh) & 0x400) == 0) ++sh;
+#endif
+        *M = man << sh;
+        *X = -24 - sh;
+    }
+}
+
+// Code of one key element (section II-A, II-D): `a_bits` the element's binary16 bits, `s_bits`
+// the magnitude bits of the vector's scale (the largest magnitude in the vector), K the number of
+// mantissa bits.  Returns the canonical byte.  Integer arithmetic only, hence exact:
+//   u = a/s = rho * 2^-e0 with rho in [1, 2);  j = floor((rho - 1) 2^K);  with n = 2^K + j the
+//   neighbours on the grid are n and n + 1 (in units of 2^(-K-e0)), and the upper one is nearer
+//   in log2 exactly when rho^2 4^K >= n (n + 1).
+template <int K>
+SA_HD uint8_t encode_element(uint32_t a_bits, uint32_t s_bits) {
+    const uint32_t mag = a_bits & 0x7fffu;
+    if (mag == 0) return 0x70;
+    int Ma, Xa, Ms, Xs;
+    half_normalise(mag, &Ma, &Xa);
+    half_normalise(s_bits & 0x7fffu, &Ms, &Xs);
+    int e0 = Xs - Xa;
+    uint32_t num = (uint32_t)Ma;
+    if (Ma < Ms) { e0 += 1; num <<= 1; }
+    if (e0 > 8) return 0x70;                       // far below the grid; also keeps e0 small
+    uint32_t j = ((num - (uint32_t)Ms) << K) / (uint32_t)Ms;
+    const unsigned long long n = (1u << K) + j;
+    const unsigned long long lhs = (unsigned long long)num * num << (2 * K);
+    const unsigned long long rhs = n * (n + 1) * (unsigned long long)Ms * (unsigned long long)Ms;
+    if (lhs >= rhs) {
+        ++j;
+        if (j == (1u << K)) { j = 0; --e0; }
+    }
+    if (e0 >= 7) return 0x70;
+    return (uint8_t)(((a_bits >> 15) << 7) | ((uint32_t)e0 << 4) | (j << (4 - K)));
+}
+
+// Power-of-two exponent g of the value scale: the largest g with amax * 2^g <= 127
+// (section II-E).  amax = M * 2^X, so amax * 2^g <= 127  <=>  M * 2^(X + g + 4) <= 2032.
+SA_HD int value_exponent(uint32_t amax_bits) {
+    if ((amax_bits & 0x7fffu) == 0) return 0;
+    int M, X;
+    half_normalise(amax_bits & 0x7fffu, &M, &X);
+    return (M <= 2032) ? (-4 - X) : (-5 - X);
+}
+
+#ifdef __CUDACC__
+// ---------------------------------------------------------------------------------------------
+// Device-only helpers.
+// ---------------------------------------------------------------------------------------------
+
+// Left shift with the PTX guarantee that amounts >= 32 give 0.  The zero code (e = 7) yields
+// the shift amount 6 - 7 = 0xffffffff, so a zero element contributes 0 without a branch.
+SA_D uint32_t shl_clamp(uint32_t x, uint32_t n) {
+    uint32_t r;
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(n));
+    return r;
+}
+
+SA_D uint32_t warp_max_u32(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+SA_D float warp_max_f32(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+SA_D float warp_sum_f32(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+SA_D float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Packed FP32 pair multiply-add of sm_100: d = a * b + c on two lanes held in one 64-bit register.
+SA_D unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+SA_D unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+SA_D void unpack_f32x2(unsigned long long v, float* lo, float* hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(*lo), "=f"(*hi) : "l"(v));
+}
+
+// Walsh-Hadamard rotation of one head vector spread over a warp: lane l holds elements
+// l*EPL .. l*EPL+EPL-1 in x[].  Sylvester order, butterflies with strides 1, 2, ..., d/2, each
+// (a, b) <- (a + b, a - b) in FP32 with one rounding per add (no contraction is possible: there
+// is no multiply), then one multiply by 1/sqrt(d) and a round to binary16.  Returns the rotated
+// elements as binary16 bit patterns.
+template <int EPL>
+SA_D void hadamard_warp(float (&x)[EPL], uint32_t (&bits)[EPL], int lane) {
+#pragma unroll
+    for (int h = 1; h < EPL; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < EPL; ++i)
+            if ((i & h) == 0) {
+                const float a = x[i], b = x[i + h];
+                x[i] = __fadd_rn(a, b);
+                x[i + h] = __fsub_rn(a, b);
+            }
+    }
+#pragma unroll
+    for (int hl = 1; hl < 32; hl <<= 1) {
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) {
+            const float other = __shfl_xor_sync(0xffffffffu, x[i], hl);
+            x[i] = (lane & hl) ? __fsub_rn(other, x[i]) : __fadd_rn(x[i], other);
+        }
+    }
+    const float scale = (EPL == 2) ? 0.125f : 0.088388346f;   // 1/sqrt(64), 1/sqrt(128)
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) bits[i] = __half_as_ushort(__float2half_rn(__fmul_rn(x[i], scale)));
+}
+
+// 2^e as a float, built from the exponent field; e must lie in [-126, 127].
+SA_D float pow2i(int e) { return __int_as_float((e + 127) << 23); }
+// 2^e for e <= 0, flushing to 0 below the normal range (used for softmax rescales, which are
+// exact power-of-two factors because the running maximum is an integer).
+SA_D float pow2i_neg(int e) { return e < -126 ? 0.0f : __int_as_float((e + 127) << 23); }
+
+SA_D float half_bits_to_float(uint32_t b) { return __half2float(__ushort_as_half((unsigned short)b)); }
+#endif  // __CUDACC__
+
+}  // namespace sa

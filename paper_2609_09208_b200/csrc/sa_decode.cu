@@ -1,0 +1,226 @@
+// Decode attention over the power-of-two key cache: the hot path.
+//
+// Grid (split, KV head x query chunk, sequence), 128 threads.  A block quantises its GT query
+// heads into shared memory, then each of its four warps walks its own 32-key tiles of the
+// block's slice of the key axis with a private online-softmax state, so the main loop has no
+// block-wide barrier.  Per tile: lane = key for the integer scores (section II-B eq. (3) with
+// the mantissa code of eq. (5)), warp-shuffle maxima and an integer running maximum in the log2
+// domain (section II-E), then lane = (token group, 8 output dims) for the floating-point A.V
+// over the INT8 values.  The four warps' states and then the blocks' partial results are merged
+// with exact power-of-two factors.
+#include "sa_common.cuh"
+#include "sa_datapath.cuh"
+#include "sa_decode_common.cuh"
+#include "sa_quant.cuh"
+
+namespace sa {
+
+template <int D, int KB, bool NIB, int GT>
+__global__ void __launch_bounds__(128) decode_kernel(DecodeArgs a) {
+    constexpr int EPL = D / 32;
+    constexpr int CH = NIB ? D / 32 : D / 16;      // 16-byte code chunks per key
+    constexpr int LPT = D / 8;                     // lanes covering one token's value row
+    constexpr int TS = 32 / LPT;                   // token groups in the A.V phase
+    constexpr int TPL = 32 / TS;                   // tokens per lane per tile
+    __shared__ __align__(16) int32_t q_s[D][GT];
+    __shared__ float qscale_s[GT];
+    __shared__ __align__(16) float2 p_s[4][32][GT];
+    __shared__ __align__(16) float red_s[4][GT][D + 2];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chunks = a.G / GT;
+    const int kvh = blockIdx.y / chunks;
+    const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;     // first query head of this block
+    const int b = blockIdx.z;
+    const int split = blockIdx.x;
+
+    // ---- prologue: quantise the GT query heads (eq. (2)) into shared memory ----
+    for (int g = warp; g < GT; g += 4) {
+        uint32_t bits[EPL];
+        load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
+        int q[EPL];
+        const float delta = quantise_query_vec<EPL>(bits, lane, a.hadamard != 0, q);
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) q_s[lane * EPL + i][g] = q[i];
+        if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
+    }
+    __syncthreads();
+
+    const int len = a.seq_lens[b];
+    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
+    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
+    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+
+    int M[GT];
+    float l[GT];
+    unsigned long long acc[GT][4];
+#pragma unroll
+    for (int g = 0; g < GT; ++g) {
+        M[g] = kMNone;
+        l[g] = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[g][j] = 0ull;
+    }
+    const int ts = lane / LPT, dc = lane % LPT;
+
+    for (int tile = tile0 + warp; tile < tile1; tile += 4) {
+        const int lp = tile >> 1;
+        const int tk0 = (tile & 1) * 32;                     // first token of the tile inside its page
+        const int n_valid = min(32, len - tile * 32);
+        const int pidx = a.page_table[(size_t)b * a.max_pages + lp];
+        if (pidx < 0 || pidx >= a.n_pages) continue;          // unmapped page: skipped, never dereferenced
+        const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+
+        // ---- phase 1: integer scores, lane = key ----
+        uint4 kc[CH];
+#pragma unroll
+        for (int c = 0; c < CH; ++c)
+            kc[c] = __ldg(reinterpret_cast<const uint4*>(block + a.kcode_off + ((size_t)c * kPageTokens + tk0 + lane) * 16));
+        const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(block + a.meta_off + (size_t)(tk0 + lane) * 4));
+
+        Planes<KB, GT> pl;
+        pl.clear();
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const uint32_t w4[4] = {kc[c].x, kc[c].y, kc[c].z, kc[c].w};
+#pragma unroll
+            for (int wi = 0; wi < 4; ++wi) {
+                const uint32_t w = w4[wi];
+                if (!NIB) {
+                    pl.corrections_bytes(w);
+#pragma unroll
+                    for (int bi = 0; bi < 4; ++bi) {
+                        const int m = c * 16 + wi * 4 + bi;
+                        int32_t q[GT];
+                        load_q<GT>(&q_s[m][0], q);
+                        pl.element((w >> (8 * bi)) & 0xffu, q);
+                    }
+                } else {
+                    pl.corrections_nibbles(w);
+#pragma unroll
+                    for (int ni = 0; ni < 8; ++ni) {
+                        const int m = c * 32 + wi * 8 + ni;
+                        int32_t q[GT];
+                        load_q<GT>(&q_s[m][0], q);
+                        pl.element(((w >> (4 * ni)) & 0xfu) << 4, q);
+                    }
+                }
+            }
+        }
+
+        // ---- phase 2: logits, integer running maximum, weights ----
+        const bool valid = lane < n_valid;
+        const float s_j = half_bits_to_float(meta & 0xffffu);
+        const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
+        const float vscale = valid ? pow2i(-g_j) : 0.0f;      // 2^-g_j; g_j in [-10, 30] for written tokens
+        bool changed = false;
+        float resc[GT];
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            const int32_t A = pl.score(g, a.f_extra);
+            if (a.dbg_scores && valid)
+                a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A;
+            const float z = valid ? (float)A * qscale_s[g] * s_j : -INFINITY;
+            const float zmax = warp_max_f32(z);
+            const int Mt = (int)ceilf(fminf(fmaxf(zmax, -1.0e8f), 1.0e8f));
+            const int Mn = max(M[g], Mt);
+            resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);   // exact power of two
+            changed |= (Mn != M[g]);
+            M[g] = Mn;
+            const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
+            l[g] = l[g] * resc[g] + p;
+            const float pv = p * vscale;
+            p_s[warp][lane][g] = make_float2(pv, pv);
+        }
+        if (changed) {                                        // warp-uniform
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const unsigned long long r2 = pack_f32x2(resc[g], resc[g]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
+            }
+        }
+        __syncwarp();
+
+        // ---- phase 3: O += p * vhat * 2^-g, lane = (token group, 8 dims) ----
+        const uint8_t* vbase = block + a.v_off + (size_t)tk0 * D + dc * 8;
+#pragma unroll 4
+        for (int i = 0; i < TPL; ++i) {
+            const int t = ts + TS * i;
+            const uint2 vv = __ldg(reinterpret_cast<const uint2*>(vbase + (size_t)t * D));
+            unsigned long long v2[4];
+            v2[0] = pack_f32x2((float)(int8_t)(vv.x), (float)(int8_t)(vv.x >> 8));
+            v2[1] = pack_f32x2((float)(int8_t)(vv.x >> 16), (float)(int8_t)(vv.x >> 24));
+            v2[2] = pack_f32x2((float)(int8_t)(vv.y), (float)(int8_t)(vv.y >> 8));
+            v2[3] = pack_f32x2((float)(int8_t)(vv.y >> 16), (float)(int8_t)(vv.y >> 24));
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&p_s[warp][t][g]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[g][j] = ffma2(v2[j], pp, acc[g][j]);
+            }
+        }
+        __syncwarp();
+    }
+
+    // ---- merge the four warps of the block, write the block's partial ----
+    block_merge_and_store<D, GT>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
+}
+
+}  // namespace sa
+
+using namespace sa;
+
+template <int D, int KB, bool NIB>
+static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
+    switch (GT) {
+        case 8: decode_kernel<D, KB, NIB, 8><<<grid, 128, 0, s>>>(a); break;
+        case 4: decode_kernel<D, KB, NIB, 4><<<grid, 128, 0, s>>>(a); break;
+        case 2: decode_kernel<D, KB, NIB, 2><<<grid, 128, 0, s>>>(a); break;
+        default: decode_kernel<D, KB, NIB, 1><<<grid, 128, 0, s>>>(a); break;
+    }
+}
+
+template <int D>
+static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
+    if (p.nibble) { launch_gt<D, 0, true>(a, GT, grid, s); return; }
+    switch (p.k) {
+        case 0: launch_gt<D, 0, false>(a, GT, grid, s); break;
+        case 1: launch_gt<D, 1, false>(a, GT, grid, s); break;
+        case 2: launch_gt<D, 2, false>(a, GT, grid, s); break;
+        default: launch_gt<D, 4, false>(a, GT, grid, s); break;
+    }
+}
+
+extern "C" sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_cache* cache,
+                                                const uint16_t* Q, float* O, void* workspace,
+                                                size_t workspace_bytes, int32_t* dbg_scores, int stages,
+                                                sa_stream stream) {
+    Plan p;
+    sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    if (p.fp16) return SA_ERR_UNSUPPORTED;
+    if ((stages & ~3) || stages == 0) return SA_ERR_INVALID_ARG;
+    DecodeArgs a;
+    int GT;
+    st = make_decode_args(p, cache, Q, O, workspace, workspace_bytes, &a, &GT);
+    if (st != SA_OK) return st;
+    if (dbg_scores && (reinterpret_cast<uintptr_t>(dbg_scores) & 3)) return SA_ERR_ALIGNMENT;
+    a.dbg_scores = dbg_scores;
+    // logits in the log2 domain: A * Delta * s * 2^-F * log2(e) / sqrt(d)
+    a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / (double)(1LL << p.F));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (stages & 1) {
+        const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
+        if (p.d == 64) launch_code<64>(p, a, GT, grid, s);
+        else launch_code<128>(p, a, GT, grid, s);
+        if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
+    }
+    return (stages & 2) ? launch_merge(p, a, s) : SA_OK;
+}
+
+extern "C" sa_status sa_decode_attention(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                                         float* O, void* workspace, size_t workspace_bytes,
+                                         int32_t* dbg_scores, sa_stream stream) {
+    return sa_decode_attention_stages(cfg, cache, Q, O, workspace, workspace_bytes, dbg_scores, 3, stream);
+}

@@ -1,0 +1,152 @@
+// Pieces shared by the quantised and the FP16 decode kernels: kernel arguments, the merge of
+// the four warps of a block, and the split-K merge (section II-F: the grid has a split
+// dimension; the merge rule follows from the integer running maximum of section II-E:
+// M* = max_s M_s, every partial is rescaled by the exact factor 2^(M_s - M*)).
+#pragma once
+#include "sa_common.cuh"
+
+namespace sa {
+
+struct DecodeArgs {
+    const uint8_t* pages;
+    const int32_t* page_table;
+    const int32_t* seq_lens;
+    const uint16_t* Q;
+    float* O;
+    float* partials;          // [n_splits][batch][Hq][D + 2]: {M (int bits), l, O[D]}
+    int32_t* dbg_scores;
+    size_t dbg_stride;
+    int batch, Hq, Hkv, G, max_pages, n_pages, n_splits, f_extra, hadamard;
+    size_t page_bytes, kcode_off, meta_off, v_off;
+    float zscale;
+};
+
+template <int GT>
+SA_D void load_q(const int32_t* src, int32_t (&q)[GT]) {
+    if constexpr (GT >= 4) {
+#pragma unroll
+        for (int i = 0; i < GT / 4; ++i) {
+            const int4 v = reinterpret_cast<const int4*>(src)[i];
+            q[4 * i] = v.x; q[4 * i + 1] = v.y; q[4 * i + 2] = v.z; q[4 * i + 3] = v.w;
+        }
+    } else if constexpr (GT == 2) {
+        const int2 v = *reinterpret_cast<const int2*>(src);
+        q[0] = v.x; q[1] = v.y;
+    } else {
+        q[0] = src[0];
+    }
+}
+
+// Per-warp states (M, l, O) -> one partial per block.  acc[g][j] holds output dims
+// dc*8 + 2j, dc*8 + 2j + 1 summed over this lane's token group; token groups sit LPT lanes apart.
+template <int D, int GT>
+SA_D void block_merge_and_store(const DecodeArgs& a, float (&red_s)[4][GT][D + 2], const int (&M)[GT],
+                                float (&l)[GT], unsigned long long (&acc)[GT][4], int lane, int warp,
+                                int ts, int dc, int LPT, int b, int h0, int split) {
+#pragma unroll
+    for (int g = 0; g < GT; ++g) {
+        const float lsum = warp_sum_f32(l[g]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float lo, hi;
+            unpack_f32x2(acc[g][j], &lo, &hi);
+            for (int off = LPT; off < 32; off <<= 1) {
+                lo += __shfl_xor_sync(0xffffffffu, lo, off);
+                hi += __shfl_xor_sync(0xffffffffu, hi, off);
+            }
+            if (ts == 0) {
+                red_s[warp][g][2 + dc * 8 + 2 * j] = lo;
+                red_s[warp][g][2 + dc * 8 + 2 * j + 1] = hi;
+            }
+        }
+        if (lane == 0) {
+            red_s[warp][g][0] = __int_as_float(M[g]);
+            red_s[warp][g][1] = lsum;
+        }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 128) {
+        const int g = idx / (D + 1), c = idx % (D + 1);       // c = 0: l, c >= 1: O[c - 1]
+        int Ms = kMNone;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) Ms = max(Ms, __float_as_int(red_s[w][g][0]));
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const int Mw = __float_as_int(red_s[w][g][0]);
+            if (Mw != kMNone) v += red_s[w][g][1 + c] * pow2i_neg(Mw - Ms);
+        }
+        float* dst = a.partials + (((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2);
+        dst[1 + c] = v;
+        if (c == 0) dst[0] = __int_as_float(Ms);
+    }
+}
+
+// One block per (sequence, query head), D threads: merge the splits and normalise.
+template <int D>
+__global__ void __launch_bounds__(D) merge_kernel(const float* __restrict__ partials, float* __restrict__ O,
+                                                  int n_splits, int n_rows) {
+    const int row = blockIdx.x;                               // b * Hq + h
+    const int dd = threadIdx.x;
+    int Ms = kMNone;
+    for (int s = 0; s < n_splits; ++s)
+        Ms = max(Ms, __float_as_int(partials[((size_t)s * n_rows + row) * (D + 2)]));
+    float l = 0.0f, o = 0.0f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float* p = partials + ((size_t)s * n_rows + row) * (D + 2);
+        const int M = __float_as_int(p[0]);
+        if (M == kMNone) continue;
+        const float f = pow2i_neg(M - Ms);
+        l += p[1] * f;
+        o += p[2 + dd] * f;
+    }
+    O[(size_t)row * D + dd] = (l > 0.0f) ? o / l : 0.0f;
+}
+
+inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16_t* Q, float* O,
+                                  void* workspace, size_t workspace_bytes, DecodeArgs* a, int* gt) {
+    if (!c || !c->pages || !c->page_table || !c->seq_lens || !Q || !O) return SA_ERR_INVALID_ARG;
+    if (c->batch <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return SA_ERR_INVALID_ARG;
+    if (c->batch > 65535) return SA_ERR_CAPACITY;
+    auto mis = [](const void* ptr, size_t al) { return (reinterpret_cast<uintptr_t>(ptr) & (al - 1)) != 0; };
+    if (mis(c->pages, p.lay.align) || mis(c->page_table, 4) || mis(c->seq_lens, 4) || mis(Q, 16) || mis(O, 16))
+        return SA_ERR_ALIGNMENT;
+    int S, GT;
+    split_plan(p, c->batch, c->max_pages_per_seq, &S, &GT);
+    const size_t need = (size_t)S * c->batch * p.Hq * (p.d + 2) * sizeof(float);
+    if (!workspace || workspace_bytes < need) return SA_ERR_CAPACITY;
+    if (mis(workspace, 16)) return SA_ERR_ALIGNMENT;
+    a->pages = static_cast<const uint8_t*>(c->pages);
+    a->page_table = c->page_table;
+    a->seq_lens = c->seq_lens;
+    a->Q = Q;
+    a->O = O;
+    a->partials = static_cast<float*>(workspace);
+    a->dbg_scores = nullptr;
+    a->dbg_stride = (size_t)c->max_pages_per_seq * kPageTokens;
+    a->batch = c->batch;
+    a->Hq = p.Hq;
+    a->Hkv = p.Hkv;
+    a->G = p.G;
+    a->max_pages = c->max_pages_per_seq;
+    a->n_pages = c->n_pages;
+    a->n_splits = S;
+    a->f_extra = p.f_extra;
+    a->hadamard = p.hadamard ? 1 : 0;
+    a->page_bytes = p.lay.page_bytes;
+    a->kcode_off = p.lay.kcode_off;
+    a->meta_off = p.lay.meta_off;
+    a->v_off = p.lay.v_off;
+    a->zscale = 0.0f;
+    *gt = GT;
+    return SA_OK;
+}
+
+inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s) {
+    const int rows = a.batch * a.Hq;
+    if (p.d == 64) merge_kernel<64><<<rows, 64, 0, s>>>(a.partials, a.O, a.n_splits, rows);
+    else merge_kernel<128><<<rows, 128, 0, s>>>(a.partials, a.O, a.n_splits, rows);
+    return cudaGetLastError() == cudaSuccess ? SA_OK : SA_ERR_CUDA;
+}
+
+}  // namespace sa

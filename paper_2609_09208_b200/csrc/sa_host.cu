@@ -1,0 +1,176 @@
+// Host side of the C ABI: configuration validation, page layout, split plan, and the
+// host-buffer convenience entry.  No kernels live here.
+#include "sa_common.cuh"
+
+namespace sa {
+
+sa_status make_plan(const sa_config* cfg, Plan* out) {
+    if (!cfg || !out) return SA_ERR_INVALID_ARG;
+    Plan p{};
+    if (cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->n_q_heads % cfg->n_kv_heads != 0)
+        return SA_ERR_INVALID_ARG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return SA_ERR_UNSUPPORTED;
+    if (cfg->page_tokens != kPageTokens) return SA_ERR_UNSUPPORTED;
+    if (cfg->flags & ~SA_FLAG_HADAMARD) return SA_ERR_INVALID_ARG;
+    p.d = cfg->head_dim;
+    p.Hq = cfg->n_q_heads;
+    p.Hkv = cfg->n_kv_heads;
+    p.G = p.Hq / p.Hkv;
+    p.hadamard = (cfg->flags & SA_FLAG_HADAMARD) != 0;
+    p.fp16 = (cfg->code == SA_KV_FP16);
+    if (p.fp16) {
+        if (cfg->klayout != SA_KLAYOUT_BYTE) return SA_ERR_UNSUPPORTED;
+        if (p.hadamard) return SA_ERR_UNSUPPORTED;   // the rotation is a pre-quantisation transform
+        p.k = 0;
+        p.nibble = false;
+        p.F = 0;
+        p.f_extra = 0;
+        p.lay.kcode_off = 0;
+        p.lay.meta_off = (size_t)kPageTokens * p.d * 2;   // empty metadata block
+        p.lay.v_off = p.lay.meta_off;
+        p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d * 2;
+        p.lay.align = 256;
+        *out = p;
+        return SA_OK;
+    }
+    if (cfg->code != SA_POT4 && cfg->code != SA_POTM1 && cfg->code != SA_POTM2 && cfg->code != SA_POTM4)
+        return SA_ERR_UNSUPPORTED;
+    p.k = cfg->code;
+    if (cfg->klayout == SA_KLAYOUT_NIBBLE) {
+        if (p.k != 0) return SA_ERR_UNSUPPORTED;
+        p.nibble = true;
+    } else if (cfg->klayout != SA_KLAYOUT_BYTE) {
+        return SA_ERR_UNSUPPORTED;
+    }
+    p.F = cfg->headroom_F == 0 ? kEmax + p.k : cfg->headroom_F;
+    if (p.F < kEmax + p.k) return SA_ERR_UNSUPPORTED;           // eq. (4): left shifts only
+    if (p.F - p.k > 24) return SA_ERR_UNSUPPORTED;
+    // INT32 accumulator bound: d * 127 * (2^(k+1) - 1) * 2^(F - k) < 2^31
+    const long long bound = (long long)p.d * 127 * ((1LL << (p.k + 1)) - 1) * (1LL << (p.F - p.k));
+    if (bound >= (1LL << 31)) return SA_ERR_UNSUPPORTED;
+    p.f_extra = p.F - p.k - kEmax;
+    const size_t kbytes = p.nibble ? (size_t)p.d / 2 : (size_t)p.d;
+    p.lay.kcode_off = 0;
+    p.lay.meta_off = (size_t)kPageTokens * kbytes;
+    p.lay.v_off = p.lay.meta_off + (size_t)kPageTokens * 4;
+    p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d;
+    p.lay.align = 256;
+    *out = p;
+    return SA_OK;
+}
+
+void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt) {
+    int GT = 1;
+    for (int c = 8; c >= 1; c >>= 1)
+        if (p.G % c == 0) { GT = c; break; }
+    // One thread block per (split, KV head x query chunk, sequence).  Aim for a few blocks per
+    // SM; every block should still own at least one 32-key tile per warp.
+    const long long units = (long long)batch * p.Hkv * (p.G / GT);
+    const long long target = (long long)kNumSMs * 4;
+    long long S = (target + units - 1) / units;
+    const long long max_tiles = (long long)max_pages * (kPageTokens / 32);
+    long long cap = max_tiles / 4;
+    if (cap < 1) cap = 1;
+    if (S > cap) S = cap;
+    if (S > 512) S = 512;
+    if (S < 1) S = 1;
+    *n_splits = (int)S;
+    *gt = GT;
+}
+
+}  // namespace sa
+
+using namespace sa;
+
+extern "C" {
+
+int sa_version(void) { return 1; }
+
+const char* sa_status_string(sa_status s) {
+    switch (s) {
+        case SA_OK: return "ok";
+        case SA_ERR_INVALID_ARG: return "invalid argument";
+        case SA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case SA_ERR_ALIGNMENT: return "misaligned pointer";
+        case SA_ERR_CAPACITY: return "buffer too small";
+        case SA_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+sa_status sa_get_layout(const sa_config* cfg, sa_layout* out) {
+    if (!out) return SA_ERR_INVALID_ARG;
+    Plan p;
+    const sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    *out = p.lay;
+    return SA_OK;
+}
+
+sa_status sa_workspace_bytes(const sa_config* cfg, int batch, int max_pages_per_seq, size_t* out) {
+    if (!out || batch <= 0 || max_pages_per_seq <= 0) return SA_ERR_INVALID_ARG;
+    Plan p;
+    const sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    int S, GT;
+    split_plan(p, batch, max_pages_per_seq, &S, &GT);
+    *out = (size_t)S * batch * p.Hq * (p.d + 2) * sizeof(float);
+    return SA_OK;
+}
+
+sa_status sa_staging_bytes(const sa_config* cfg, int batch, size_t* out) {
+    if (!out || batch <= 0) return SA_ERR_INVALID_ARG;
+    Plan p;
+    const sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    const size_t q = (size_t)batch * p.Hq * p.d * 2;
+    const size_t kv = (size_t)batch * p.Hkv * p.d * 2;
+    const size_t o = (size_t)batch * p.Hq * p.d * 4;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    *out = up(q) + 2 * up(kv) + up(o);
+    return SA_OK;
+}
+
+sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q_host,
+                              const uint16_t* K_new_host, const uint16_t* V_new_host, float* O_host,
+                              void* staging, size_t staging_bytes, void* workspace,
+                              size_t workspace_bytes, sa_stream stream) {
+    if (!cache || !Q_host || !K_new_host || !V_new_host || !O_host || !staging) return SA_ERR_INVALID_ARG;
+    Plan p;
+    sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    if (cache->batch <= 0) return SA_ERR_INVALID_ARG;
+    size_t need;
+    st = sa_staging_bytes(cfg, cache->batch, &need);
+    if (st != SA_OK) return st;
+    if (staging_bytes < need) return SA_ERR_CAPACITY;
+    if (reinterpret_cast<uintptr_t>(staging) & 255) return SA_ERR_ALIGNMENT;
+    size_t ws_need;
+    st = sa_workspace_bytes(cfg, cache->batch, cache->max_pages_per_seq, &ws_need);
+    if (st != SA_OK) return st;
+    if (!workspace || workspace_bytes < ws_need) return SA_ERR_CAPACITY;
+    const size_t q = (size_t)cache->batch * p.Hq * p.d * 2;
+    const size_t kv = (size_t)cache->batch * p.Hkv * p.d * 2;
+    const size_t o = (size_t)cache->batch * p.Hq * p.d * 4;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    char* base = static_cast<char*>(staging);
+    uint16_t* dQ = reinterpret_cast<uint16_t*>(base);
+    uint16_t* dK = reinterpret_cast<uint16_t*>(base + up(q));
+    uint16_t* dV = reinterpret_cast<uint16_t*>(base + up(q) + up(kv));
+    float* dO = reinterpret_cast<float*>(base + up(q) + 2 * up(kv));
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(dQ, Q_host, q, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+    if (cudaMemcpyAsync(dK, K_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+    if (cudaMemcpyAsync(dV, V_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+    st = sa_append_kv(cfg, cache, dK, dV, 1, stream);
+    if (st != SA_OK) return st;
+    if (p.fp16)
+        st = sa_decode_attention_fp16(cfg, cache, dQ, dO, workspace, workspace_bytes, stream);
+    else
+        st = sa_decode_attention(cfg, cache, dQ, dO, workspace, workspace_bytes, nullptr, stream);
+    if (st != SA_OK) return st;
+    if (cudaMemcpyAsync(O_host, dO, o, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SA_ERR_CUDA;
+    return SA_OK;
+}
+
+}  // extern "C"

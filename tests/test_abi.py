@@ -1,0 +1,123 @@
+"""The C-ABI library without a GPU: it loads, exports every symbol the header declares, and its
+host-side validation and layout arithmetic behave as documented (nothing here launches a kernel)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2609_09208_b200 import binding as sa
+from paper_2609_09208_b200 import build as sa_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    sa_build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "sa.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(sa_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(sa.EXPORTS), declared ^ set(sa.EXPORTS)
+    lib = sa.lib()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert lib.sa_version() >= 1
+    assert sa.status_string(0) == "ok" and "unsupported" in sa.status_string(2)
+
+
+@pytest.mark.parametrize("d,code,nibble,want", [
+    (64, sa.SA_POT4, True, 100), (64, sa.SA_POT4, False, 132), (64, sa.SA_POTM1, False, 132),
+    (64, sa.SA_POTM4, False, 132), (128, sa.SA_POT4, True, 196), (128, sa.SA_POTM4, False, 260),
+    (64, sa.SA_KV_FP16, False, 256), (128, sa.SA_KV_FP16, False, 512)])
+def test_layout_bytes_per_key(d, code, nibble, want):
+    lay = sa.get_layout(sa.make_config(d, 32, 4, code, nibble=nibble))
+    assert lay.page_bytes == want * 64
+    assert lay.page_bytes % 128 == 0 and lay.meta_off % 16 == 0 and lay.v_off % 16 == 0
+    assert lay.kcode_off == 0 and lay.meta_off <= lay.v_off < lay.page_bytes
+
+
+def test_layout_is_within_a_byte_of_the_papers_record_sizes():
+    # the paper's records: 101 B (PoT-4), 133 B (8-bit code), 256 B (FP16) per key at d = 64
+    golden = {}
+    for line in open(os.path.join(ROOT, "tests", "golden", "paper_constants.txt")):
+        line = line.split("#")[0]
+        if "=" in line:
+            k, v = line.split("=")
+            golden[k.strip()] = float(v)
+    per_key = lambda code, nib: sa.get_layout(sa.make_config(64, 32, 4, code, nibble=nib)).page_bytes / 64
+    assert abs(per_key(sa.SA_POT4, True) - golden["bytes_per_key_pot4"]) <= 1
+    assert abs(per_key(sa.SA_POTM4, False) - golden["bytes_per_key_int8"]) <= 1
+    assert per_key(sa.SA_KV_FP16, False) == golden["bytes_per_key_fp16"]
+    assert abs(per_key(sa.SA_KV_FP16, False) / per_key(sa.SA_POT4, True) - golden["kv_cache_ratio"]) < 0.1
+
+
+def _status(fn, *args):
+    try:
+        fn(*args)
+    except sa.SaError as e:
+        return e.status
+    return 0
+
+
+def test_config_validation():
+    ok = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    assert _status(sa.get_layout, ok) == 0
+    assert _status(sa.get_layout, sa.make_config(96, 32, 4, sa.SA_POTM4)) == 2          # head_dim
+    assert _status(sa.get_layout, sa.make_config(64, 30, 4, sa.SA_POTM4)) == 1          # Hq % Hkv
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, 3)) == 2                     # no 3-bit mantissa
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POTM1, nibble=True)) == 2
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_KV_FP16, hadamard=True)) == 2
+    bad = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    bad.page_tokens = 32
+    assert _status(sa.get_layout, bad) == 2
+    bad = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    bad.flags = 8
+    assert _status(sa.get_layout, bad) == 1
+    # head-room: F >= 6 + k (left shifts only), and the INT32 bound d*127*(2^(k+1)-1)*2^(F-k) < 2^31
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POT4, headroom_F=5)) == 2
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POT4, headroom_F=7)) == 0
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POT4, headroom_F=18)) == 0   # 64*127*2^18 < 2^31
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POT4, headroom_F=19)) == 2
+    assert _status(sa.get_layout, sa.make_config(128, 32, 8, sa.SA_POTM4, headroom_F=16)) == 0  # 128*127*31*2^12 < 2^31
+    assert _status(sa.get_layout, sa.make_config(128, 32, 8, sa.SA_POTM4, headroom_F=17)) == 2
+
+
+def test_workspace_and_staging_sizes():
+    cfg = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    w = sa.workspace_bytes(cfg, 1, 512)
+    assert w > 0 and w % (32 * 66 * 4) == 0
+    n_splits = w // (32 * 66 * 4)
+    assert 1 <= n_splits <= 512
+    assert sa.workspace_bytes(cfg, 16, 256) % (16 * 32 * 66 * 4) == 0
+    assert sa.workspace_bytes(cfg, 1, 1) == 32 * 66 * 4          # a single page: no split
+    assert _status(sa.workspace_bytes, cfg, 0, 4) == 1
+    assert sa.staging_bytes(cfg, 2) >= 2 * (32 * 64 * 2 + 2 * 4 * 64 * 2 + 32 * 64 * 4)
+
+
+def test_entry_points_reject_bad_arguments_before_any_cuda_call():
+    lib = sa.lib()
+    cfg = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    null = C.c_void_p(0)
+    one = C.c_void_p(256)       # a non-null, aligned, never dereferenced address
+    assert lib.sa_encode_keys(C.byref(cfg), null, C.c_int64(4), one, one, null) == 1
+    assert lib.sa_encode_keys(C.byref(cfg), C.c_void_p(257), C.c_int64(4), one, one, null) == 3
+    assert lib.sa_encode_keys(C.byref(cfg), one, C.c_int64(0), one, one, null) == 0      # nothing to do
+    assert lib.sa_quantise_query(C.byref(cfg), null, C.c_int(1), one, one, null) == 1
+    assert lib.sa_quantise_values(C.byref(cfg), one, C.c_int64(-1), one, one, null) == 1
+    cache = sa.SaCache(0, 256, 256, 1, 4, 4)
+    assert lib.sa_decode_attention(C.byref(cfg), C.byref(cache), one, one, one, C.c_size_t(1 << 30), null, null) == 1
+    cache = sa.SaCache(256, 256, 256, 1, 4, 4)
+    assert lib.sa_decode_attention(C.byref(cfg), C.byref(cache), one, one, one, C.c_size_t(8), null, null) == 4
+    assert lib.sa_decode_attention(C.byref(cfg), C.byref(cache), one, one, C.c_void_p(260), C.c_size_t(1 << 30), null, null) == 3
+    cache = sa.SaCache(264, 256, 256, 1, 4, 4)                                            # pool base not 256-aligned
+    assert lib.sa_append_kv(C.byref(cfg), C.byref(cache), one, one, C.c_int(1), null) == 3
+    fp = sa.make_config(64, 32, 4, sa.SA_KV_FP16)
+    cache = sa.SaCache(256, 256, 256, 1, 4, 4)
+    assert lib.sa_decode_attention(C.byref(fp), C.byref(cache), one, one, one, C.c_size_t(1 << 30), null, null) == 2
+    assert lib.sa_decode_attention_fp16(C.byref(cfg), C.byref(cache), one, one, one, C.c_size_t(1 << 30), null) == 2
+    assert lib.sa_debug_unpack(C.byref(cfg), C.byref(cache), C.c_int(3), C.c_int(1), null, null, null, null, null) == 1
+    assert lib.sa_debug_unpack(C.byref(cfg), C.byref(cache), C.c_int(0), C.c_int(4 * 64 + 1), null, null, null, null, null) == 4

@@ -1,0 +1,371 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Integer results (codes, scales, quantised queries and values, INT32 scores) must be
+bit-exact; the attention output must agree within 1e-3 (FP32, unit-variance values)."""
+import numpy as np
+import pytest
+
+from oracle import sa_oracle as ora
+from paper_2609_09208_b200 import binding as sa
+from paper_2609_09208_b200 import build as sa_build
+from paper_2609_09208_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL_O = 1e-3
+E = 6
+
+
+@pytest.fixture(scope="module")
+def dev():
+    import torch
+    sa_build.build()
+    sa.lib()
+    return torch.device("cuda:0")
+
+
+def t16(x, dev):
+    """float16 numpy -> CUDA tensor of its bits (int16 storage; the library only sees bytes)."""
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev)
+
+
+def cfg_of(case, *, code=None, F=0):
+    code = case.code_k if code is None else code
+    return sa.make_config(case.head_dim, case.n_q_heads, case.n_kv_heads, code, nibble=case.nibble,
+                          headroom_F=F, hadamard=case.hadamard)
+
+
+def build_cache(case, dev, *, cfg=None, permute_seed=None, extra_tokens=0):
+    cfg = cfg or cfg_of(case)
+    n_pages = int(np.maximum((case.lens + extra_tokens + 63) // 64, 1).sum())
+    perm = synth.page_permutation(n_pages, permute_seed) if permute_seed is not None else None
+    cache = sa.PagedCache(cfg, case.lens, dev, extra_tokens=extra_tokens, permutation=perm)
+    cache.fill(t16(case.K, dev), t16(case.V, dev), case.cu_lens)
+    return cfg, cache
+
+
+def run_decode(case, dev, *, F=0, want_scores=True, permute_seed=None):
+    import torch
+    cfg = cfg_of(case, F=F)
+    cfg, cache = build_cache(case, dev, cfg=cfg, permute_seed=permute_seed)
+    O = torch.full((case.batch, case.n_q_heads, case.head_dim), float("nan"), dtype=torch.float32, device=dev)
+    dbg = None
+    if want_scores:
+        dbg = torch.full((case.batch, case.n_q_heads, cache.max_pages * 64), -7, dtype=torch.int32, device=dev)
+    sa.decode_attention(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, dbg)
+    torch.cuda.synchronize()
+    return O.cpu().numpy(), (dbg.cpu().numpy() if want_scores else None), cache
+
+
+def check_against_oracle(case, O, dbg, *, F=0, n_threads=8):
+    F = F or E + case.code_k
+    ref = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, case.code_k, F, hadamard=case.hadamard,
+                               want_scores=dbg is not None, n_threads=n_threads)
+    assert ref["overflow"] == 0
+    if dbg is not None:
+        for b in range(case.batch):
+            T = int(case.lens[b])
+            assert np.array_equal(dbg[b, :, :T].astype(np.int64), ref["A"][b][:, :T]), "integer scores differ (sequence %d)" % b
+            assert np.all(dbg[b, :, T:] == -7), "scores written beyond the sequence length"
+    err = np.max(np.abs(O.astype(np.float64) - ref["O"])) if O.size else 0.0
+    assert np.isfinite(O).all()
+    assert err <= TOL_O, "max |dO| = %g" % err
+    return err
+
+
+# ------------------------------------------------------------------------------- quantisers
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("k", [0, 1, 2, 4])
+@pytest.mark.parametrize("hadamard", [False, True])
+def test_encode_keys_bit_exact(dev, d, k, hadamard):
+    import torch
+    rng = np.random.default_rng(1000 + d + k)
+    Hkv, n = 3, 1500                                    # 4500 vectors: many blocks and a ragged tail
+    K = synth.outlier_keys_fp16(rng, n, Hkv, d)
+    K[5, 1, :] = 0                                      # an all-zero vector
+    K[6, 0, 3] = 0
+    K.view(np.uint16)[7, 2, :8] = [1, 2, 0x8001, 0x03FF, 0x0400, 0x7BFF, 0xFBFF, 0x8000]   # subnormals, extremes, -0
+    cfg = sa.make_config(d, Hkv, Hkv, k, hadamard=hadamard)
+    codes = torch.zeros((n, Hkv, d), dtype=torch.uint8, device=dev)
+    scales = torch.zeros((n, Hkv), dtype=torch.int16, device=dev)
+    sa.encode_keys(cfg, t16(K, dev), codes, scales)
+    torch.cuda.synchronize()
+    Kr = ora.hadamard_fp16(K) if hadamard else K
+    want_c, want_s = ora.encode_keys(Kr, k)
+    assert np.array_equal(scales.cpu().numpy().view(np.uint16), want_s.view(np.uint16))
+    assert np.array_equal(codes.cpu().numpy(), want_c)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("hadamard", [False, True])
+def test_quantise_query_bit_exact(dev, d, hadamard):
+    import torch
+    rng = np.random.default_rng(1100 + d)
+    B, Hq = 37, 8
+    Q = (rng.standard_normal((B, Hq, d)) * np.exp(rng.standard_normal((B, Hq, 1)))).astype(np.float16)
+    Q[3, 2] = 0
+    cfg = sa.make_config(d, Hq, Hq, sa.SA_POTM4, hadamard=hadamard)
+    qh = torch.zeros((B, Hq, d), dtype=torch.int8, device=dev)
+    dl = torch.zeros((B, Hq), dtype=torch.float32, device=dev)
+    sa.quantise_query(cfg, t16(Q, dev), qh, dl)
+    torch.cuda.synchronize()
+    want_q, want_d = ora.quantise_query(ora.hadamard_fp16(Q) if hadamard else Q)
+    assert np.array_equal(qh.cpu().numpy(), want_q)
+    assert np.array_equal(dl.cpu().numpy().view(np.uint32), want_d.view(np.uint32))
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_quantise_values_bit_exact(dev, d):
+    import torch
+    rng = np.random.default_rng(1200 + d)
+    n, Hkv = 1111, 2
+    V = (rng.standard_normal((n, Hkv, d)) * np.exp(rng.uniform(-9, 9, (n, Hkv, 1)))).astype(np.float16)
+    V[4, 1] = 0
+    V.view(np.uint16)[9, 0, :4] = [1, 0x7BFF, 0xFBFF, 0x8001]
+    cfg = sa.make_config(d, Hkv, Hkv, sa.SA_POTM1)
+    vh = torch.zeros((n, Hkv, d), dtype=torch.int8, device=dev)
+    g = torch.zeros((n, Hkv), dtype=torch.int8, device=dev)
+    sa.quantise_values(cfg, t16(V, dev), vh, g)
+    torch.cuda.synchronize()
+    want_v, want_g = ora.quantise_value(V)
+    assert np.array_equal(g.cpu().numpy(), want_g)
+    assert np.array_equal(vh.cpu().numpy(), want_v)
+
+
+# ------------------------------------------------------------------------------- cache write
+def _unpack(cfg, cache, b, T, case, dev):
+    import torch
+    Hkv, d = case.n_kv_heads, case.head_dim
+    codes = torch.zeros((T, Hkv, d), dtype=torch.uint8, device=dev)
+    scales = torch.zeros((T, Hkv), dtype=torch.int16, device=dev)
+    vh = torch.zeros((T, Hkv, d), dtype=torch.int8, device=dev)
+    g = torch.zeros((T, Hkv), dtype=torch.int8, device=dev)
+    sa.debug_unpack(cfg, cache.handle, b, T, codes, scales, vh, g)
+    torch.cuda.synchronize()
+    return codes.cpu().numpy(), scales.cpu().numpy().view(np.uint16), vh.cpu().numpy(), g.cpu().numpy()
+
+
+@pytest.mark.parametrize("d,k,nibble,hadamard", [(64, 0, True, False), (64, 0, False, True), (64, 1, False, False),
+                                                 (64, 4, False, True), (128, 0, True, False), (128, 2, False, False),
+                                                 (128, 4, False, True)])
+def test_fill_and_unpack_bit_exact(dev, d, k, nibble, hadamard):
+    case = synth.make_case("fill", [130, 0, 64, 1, 257], 4, 2, d, k, outliers=True, nibble=nibble,
+                           hadamard=hadamard, seed=1300 + d + k)
+    cfg, cache = build_cache(case, dev, permute_seed=5)
+    for b in range(case.batch):
+        T = int(case.lens[b])
+        if T == 0:
+            continue
+        K = case.K[case.cu_lens[b]:case.cu_lens[b + 1]]
+        V = case.V[case.cu_lens[b]:case.cu_lens[b + 1]]
+        want_c, want_s = ora.encode_keys(ora.hadamard_fp16(K) if hadamard else K, k)
+        want_v, want_g = ora.quantise_value(V)
+        codes, scales, vh, g = _unpack(cfg, cache, b, T, case, dev)
+        assert np.array_equal(codes, want_c) and np.array_equal(scales, want_s.view(np.uint16))
+        assert np.array_equal(vh, want_v) and np.array_equal(g, want_g)
+
+
+@pytest.mark.parametrize("d,k,nibble", [(64, 4, False), (64, 0, True), (128, 1, False)])
+def test_append_matches_bulk_fill(dev, d, k, nibble):
+    import torch
+    lens = np.array([62, 0, 127])
+    n_app = 4                                          # crosses a page boundary for the first and last sequence
+    full = synth.make_case("app", lens + n_app, 4, 2, d, k, nibble=nibble, seed=1400 + d + k)
+    cfg = cfg_of(full)
+    cache = sa.PagedCache(cfg, lens, dev, extra_tokens=n_app, permutation=synth.page_permutation(
+        int(np.maximum((lens + n_app + 63) // 64, 1).sum()), 9))
+    # bulk-fill the first lens[b] tokens, then append the rest one token at a time
+    idx0 = np.concatenate([np.arange(full.cu_lens[b], full.cu_lens[b] + lens[b]) for b in range(3)]).astype(np.int64)
+    cu0 = np.concatenate([[0], np.cumsum(lens)])
+    cache.fill(t16(full.K[idx0], dev), t16(full.V[idx0], dev), cu0)
+    for i in range(n_app):
+        rows = np.array([full.cu_lens[b] + lens[b] + i for b in range(3)])
+        sa.append_kv(cfg, cache.handle, t16(full.K[rows], dev), t16(full.V[rows], dev), True)
+    torch.cuda.synchronize()
+    assert cache.seq_lens.cpu().numpy().tolist() == (lens + n_app).tolist()
+    for b in range(3):
+        T = int(lens[b] + n_app)
+        K = full.K[full.cu_lens[b]:full.cu_lens[b + 1]]
+        V = full.V[full.cu_lens[b]:full.cu_lens[b + 1]]
+        want_c, want_s = ora.encode_keys(K, k)
+        want_v, want_g = ora.quantise_value(V)
+        codes, scales, vh, g = _unpack(cfg, cache, b, T, full, dev)
+        assert np.array_equal(codes, want_c) and np.array_equal(scales, want_s.view(np.uint16))
+        assert np.array_equal(vh, want_v) and np.array_equal(g, want_g)
+    # a full sequence is left untouched
+    tight = sa.PagedCache(cfg, [64], dev)
+    tight.seq_lens.fill_(64)
+    sa.append_kv(cfg, tight.handle, t16(full.K[:1], dev), t16(full.V[:1], dev), True)
+    torch.cuda.synchronize()
+    assert int(tight.seq_lens[0]) == 64
+
+
+# ------------------------------------------------------------------------------- decode attention
+def test_config1_single_head_pot4(dev):
+    case = synth.config1()
+    O, dbg, _ = run_decode(case, dev, F=6)
+    check_against_oracle(case, O, dbg, F=6)
+
+
+def test_config2_llama_shape_potm1_outliers(dev):
+    case = synth.config2()
+    O, dbg, _ = run_decode(case, dev)
+    check_against_oracle(case, O, dbg)
+
+
+@pytest.mark.parametrize("k,nibble,hadamard,outliers", [
+    (4, False, False, False), (4, False, True, False), (4, False, True, True),
+    (0, False, False, False), (0, True, False, False), (0, True, True, True)])
+def test_config3_T32k_full_size(dev, k, nibble, hadamard, outliers):
+    case = synth.config3(k, hadamard=hadamard, nibble=nibble, outliers=outliers)
+    O, dbg, _ = run_decode(case, dev)
+    check_against_oracle(case, O, dbg)
+
+
+def test_config4_ragged_paged_batch_potm2(dev):
+    case = synth.config4()
+    O, dbg, _ = run_decode(case, dev, permute_seed=44)
+    check_against_oracle(case, O, dbg)
+
+
+@pytest.mark.parametrize("T,B,k", [(1024, 1, 0), (1024, 8, 1), (4096, 8, 4), (16384, 1, 1), (4096, 32, 0)])
+def test_config5_d128_cells_in_full(dev, T, B, k):
+    case = synth.config5(T, B, k)
+    O, dbg, _ = run_decode(case, dev)
+    check_against_oracle(case, O, dbg)
+
+
+def test_config5_largest_cells_sampled_sequences(dev):
+    """T = 128k x B = 8, PoT-M4, d = 128 (the cache is built sequence by sequence from seeded
+    inputs; the oracle recomputes two sampled sequences in full, scores included)."""
+    import torch
+    T, B, k, d, Hq, Hkv = 131072, 8, 4, 128, 32, 8
+    cfg = sa.make_config(d, Hq, Hkv, k)
+    cache = sa.PagedCache(cfg, [T] * B, dev)
+    Q = synth.gaussian_fp16(np.random.default_rng(7), (B, Hq, d))
+    kept = {}
+    for b in range(B):
+        one = synth.make_case("c5big", [T], Hq, Hkv, d, k, outliers=True, seed=5100 + b)
+        sub = sa.SaCache(cache.pages.data_ptr(), cache.page_table[b:b + 1].contiguous().data_ptr(),
+                         cache.seq_lens[b:b + 1].data_ptr(), 1, cache.max_pages, cache.n_pages)
+        sa.fill_kv(cfg, sub, t16(one.K, dev), t16(one.V, dev), one.cu_lens)
+        torch.cuda.synchronize()
+        if b in (2, 7):
+            kept[b] = one
+    cache.seq_lens.fill_(T)
+    O = torch.zeros((B, Hq, d), dtype=torch.float32, device=dev)
+    dbg = torch.zeros((B, Hq, cache.max_pages * 64), dtype=torch.int32, device=dev)
+    sa.decode_attention(cfg, cache.handle, t16(Q, dev), O, cache.workspace, dbg)
+    torch.cuda.synchronize()
+    O = O.cpu().numpy()
+    for b, one in kept.items():
+        ref = ora.decode_attention(Q[b:b + 1], one.K, one.V, one.cu_lens, k, E + k, want_scores=True, n_threads=8)
+        assert np.array_equal(dbg[b].cpu().numpy().astype(np.int64), ref["A"][0])
+        assert np.max(np.abs(O[b] - ref["O"][0])) <= TOL_O
+    assert np.isfinite(O).all()
+
+
+@pytest.mark.parametrize("lens", [[0], [1], [31], [32], [33], [63], [64], [65], [127, 0, 129, 1], [4097]])
+@pytest.mark.parametrize("k,nibble", [(0, True), (4, False)])
+def test_edge_lengths(dev, lens, k, nibble):
+    case = synth.make_case("edge", lens, 8, 2, 64, k, nibble=nibble, seed=1500 + sum(lens) + k)
+    O, dbg, _ = run_decode(case, dev, permute_seed=3)
+    check_against_oracle(case, O, dbg)
+    for b, T in enumerate(lens):
+        if T == 0:
+            assert not O[b].any()
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(1, 1), (2, 1), (4, 4), (6, 2), (12, 1), (16, 2), (32, 4)])
+def test_query_group_sizes(dev, Hq, Hkv):
+    case = synth.make_case("gqa", [300, 77], Hq, Hkv, 64, 2, outliers=True, seed=1600 + Hq)
+    O, dbg, _ = run_decode(case, dev)
+    check_against_oracle(case, O, dbg)
+
+
+@pytest.mark.parametrize("k,F", [(0, 7), (0, 18), (1, 9), (4, 12), (4, 16)])
+def test_headroom_F(dev, k, F):
+    # F = 7 with PoT-4 is the paper's worked bound (d * 127 * 2^7); larger F only shifts the exact integer
+    d = 128 if F == 16 else 64
+    case = synth.make_case("F", [200], 8, 2, d, k, seed=1700 + F)
+    if (d * 127 * ((1 << (k + 1)) - 1)) << (F - k) >= 2 ** 31:
+        pytest.skip("outside the INT32 bound")
+    O, dbg, _ = run_decode(case, dev, F=F)
+    check_against_oracle(case, O, dbg, F=F)
+
+
+def test_attained_int32_bound_and_determinism(dev):
+    import torch
+    # keys equal to +scale everywhere (e = 0) and a constant query attain d * 127 * 2^F exactly
+    d, T = 64, 100
+    case = synth.make_case("bound", [T], 2, 1, d, 0, seed=1)
+    case.K[:] = np.float16(1.5)
+    case.Q[:] = np.float16(-2.0)
+    O, dbg, _ = run_decode(case, dev, F=18)
+    assert np.all(dbg[0, :, :T] == -(64 * 127 * 2 ** 18))
+    check_against_oracle(case, O, dbg, F=18)
+    case = synth.config3(4, T=8192)
+    o1, s1, _ = run_decode(case, dev)
+    o2, s2, _ = run_decode(case, dev)
+    assert np.array_equal(o1.view(np.uint32), o2.view(np.uint32)) and np.array_equal(s1, s2)
+
+
+def test_unmapped_pages_are_skipped_not_read(dev):
+    import torch
+    case = synth.make_case("unmapped", [200], 8, 2, 64, 4, seed=1800)
+    cfg, cache = build_cache(case, dev)
+    cache.page_table[0, 1] = -1                     # tokens 64..127 vanish
+    cache.page_table[0, 2] = cache.n_pages + 5      # out of range: also skipped
+    O = torch.zeros((1, 8, 64), dtype=torch.float32, device=dev)
+    sa.decode_attention(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, None)
+    torch.cuda.synchronize()
+    keep = np.r_[0:64, 192:200]
+    sub = synth.Case("sub", case.Q, case.K[keep], case.V[keep], np.array([0, len(keep)]), 8, 2, 64, 4)
+    ref = ora.decode_attention(sub.Q, sub.K, sub.V, sub.cu_lens, 4, 10)
+    assert np.max(np.abs(O.cpu().numpy() - ref["O"])) <= TOL_O
+
+
+# ------------------------------------------------------------------------------- FP16 baseline kernel
+@pytest.mark.parametrize("d,Hq,Hkv,lens", [(64, 32, 4, [4096]), (64, 8, 2, [0, 1, 33, 700]), (128, 32, 8, [2048, 100]),
+                                           (64, 1, 1, [1024]), (64, 32, 4, [32768])])
+def test_fp16_kernel_matches_textbook_attention(dev, d, Hq, Hkv, lens):
+    import torch
+    case = synth.make_case("fp16", lens, Hq, Hkv, d, 0, seed=1900 + d + len(lens))
+    cfg = sa.make_config(d, Hq, Hkv, sa.SA_KV_FP16)
+    _, cache = build_cache(case, dev, cfg=cfg, permute_seed=2)
+    O = torch.full((case.batch, Hq, d), float("nan"), dtype=torch.float32, device=dev)
+    sa.decode_attention_fp16(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace)
+    torch.cuda.synchronize()
+    O = O.cpu().numpy()
+    for b in range(case.batch):
+        K = case.K[case.cu_lens[b]:case.cu_lens[b + 1]]
+        V = case.V[case.cu_lens[b]:case.cu_lens[b + 1]]
+        ref = ora.sdpa_fp16(case.Q[b], K, V)
+        assert np.max(np.abs(O[b] - ref)) <= TOL_O
+
+
+# ------------------------------------------------------------------------------- host-buffer entry
+@pytest.mark.parametrize("code", [sa.SA_POTM4, sa.SA_KV_FP16])
+def test_decode_step_from_host_buffers(dev, code):
+    import torch
+    lens = np.array([100, 64, 0])
+    full = synth.make_case("host", lens + 1, 8, 2, 64, 4, seed=2000)
+    cfg = sa.make_config(64, 8, 2, code)
+    cache = sa.PagedCache(cfg, lens, dev, extra_tokens=1)
+    idx0 = np.concatenate([np.arange(full.cu_lens[b], full.cu_lens[b] + lens[b]) for b in range(3)]).astype(np.int64)
+    cache.fill(t16(full.K[idx0], dev), t16(full.V[idx0], dev), np.concatenate([[0], np.cumsum(lens)]))
+    last = np.array([full.cu_lens[b + 1] - 1 for b in range(3)])
+    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).pin_memory()
+    Qh, Kh, Vh = pin(full.Q), pin(full.K[last]), pin(full.V[last])
+    Oh = torch.zeros((3, 8, 64), dtype=torch.float32).pin_memory()
+    staging = torch.empty(sa.staging_bytes(cfg, 3), dtype=torch.uint8, device=dev)
+    sa.decode_step_host(cfg, cache.handle, Qh, Kh, Vh, Oh, staging, cache.workspace)
+    torch.cuda.synchronize()
+    assert cache.seq_lens.cpu().numpy().tolist() == (lens + 1).tolist()
+    for b in range(3):
+        K = full.K[full.cu_lens[b]:full.cu_lens[b + 1]]
+        V = full.V[full.cu_lens[b]:full.cu_lens[b + 1]]
+        if code == sa.SA_KV_FP16:
+            ref = ora.sdpa_fp16(full.Q[b], K, V)
+        else:
+            ref = ora.decode_attention(full.Q[b:b + 1], K, V, np.array([0, len(K)]), 4, 10)["O"][0]
+        assert np.max(np.abs(Oh.numpy()[b] - ref)) <= TOL_O

@@ -1,0 +1,90 @@
+"""The library's exact-arithmetic functions, compiled for the host, against the CPU oracle.
+
+The key-element encoder, the value exponent and the plane-accumulator score datapath are plain
+integer code that nvcc also compiles for the host; this checks them exhaustively / on random
+inputs without a GPU.  (The same functions run on the device in the -m gpu parity tests.)"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+import pytest
+
+from oracle import sa_oracle as ora
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(HERE, "host_harness.cu")
+LIB = os.path.join(HERE, "_build", "libhh.so")
+CSRC = os.path.join(HERE, "..", "paper_2609_09208_b200", "csrc")
+
+
+@pytest.fixture(scope="module")
+def hh():
+    os.makedirs(os.path.dirname(LIB), exist_ok=True)
+    deps = [SRC] + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")]
+    if not os.path.exists(LIB) or any(os.path.getmtime(d) > os.path.getmtime(LIB) for d in deps):
+        subprocess.check_call(["/usr/local/cuda/bin/nvcc", "-std=c++17", "-O2", "-shared", "-Xcompiler", "-fPIC",
+                               "-Wno-deprecated-gpu-targets", "-o", LIB, SRC])
+    lib = C.CDLL(LIB)
+    lib.hh_score.restype = C.c_int32
+    return lib
+
+
+SCALES = [0x3C00, 0x7BFF, 0x3A66, 0x0400, 0x01F3, 0x4D2B, 0x0001, 0x2E66]
+
+
+@pytest.mark.parametrize("k", [0, 1, 2, 4])
+@pytest.mark.parametrize("s_bits", SCALES)
+def test_encode_element_exhaustive_vs_oracle(hh, k, s_bits):
+    mags = np.arange(0, s_bits + 1, dtype=np.uint16)
+    vals = (mags | ((np.arange(len(mags)) % 2).astype(np.uint16) << 15)).astype(np.uint16)
+    got = np.empty(len(vals), dtype=np.uint8)
+    hh.hh_encode_many(C.c_int(k), vals.ctypes.data_as(C.c_void_p), C.c_int64(len(vals)), C.c_uint(s_bits),
+                      got.ctypes.data_as(C.c_void_p))
+    d = 64
+    n_vec = (len(vals) + d - 2) // (d - 1)
+    K = np.zeros((n_vec, d), dtype=np.uint16)
+    K[:, 0] = s_bits
+    flat = np.zeros(n_vec * (d - 1), dtype=np.uint16)
+    flat[: len(vals)] = vals
+    K[:, 1:] = flat.reshape(n_vec, d - 1)
+    want = ora.encode_keys(K, k)[0][:, 1:].reshape(-1)[: len(vals)]
+    assert np.array_equal(got, want)
+
+
+def test_value_exponent_all_magnitudes(hh):
+    mags = np.arange(0, 0x7C00, dtype=np.uint16)          # every finite binary16 magnitude
+    V = np.zeros((len(mags), 64), dtype=np.uint16)
+    V[:, 5] = mags
+    _, g = ora.quantise_value(V)
+    got = np.array([hh.hh_value_exponent(C.c_uint(int(m))) for m in mags], dtype=np.int8)
+    assert np.array_equal(got, g)
+
+
+@pytest.mark.parametrize("k", [0, 1, 2, 4])
+@pytest.mark.parametrize("d", [64, 128])
+def test_plane_datapath_equals_oracle_scores(hh, k, d):
+    rng = np.random.default_rng(100 + k + d)
+    for trial in range(200):
+        e = rng.integers(0, 8, d)
+        j = rng.integers(0, 1 << k, d)
+        sgn = rng.integers(0, 2, d)
+        codes = ((sgn << 7) | (e << 4) | (j << (4 - k))).astype(np.uint8)
+        if trial % 3 == 0:
+            codes[e == 7] = 0x70                    # canonical zeros
+        if trial == 1:
+            codes[:] = 0x80 | (j << (4 - k))        # every term negative with the largest shift
+        q = rng.integers(-127, 128, d).astype(np.int8)
+        if trial == 2:
+            q[:] = 127
+        for f_extra in (0, 1):
+            F = 6 + k + f_extra
+            want, ov = ora.scores(q[None, :], codes[None, None, :], k, F)
+            assert ov == 0
+            got = hh.hh_score(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p),
+                              C.c_int(d), C.c_int(f_extra), C.c_int(0))
+            assert got == int(want[0, 0]), (trial, f_extra)
+            if k == 0:
+                got_n = hh.hh_score(C.c_int(0), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p),
+                                    C.c_int(d), C.c_int(f_extra), C.c_int(1))
+                assert got_n == int(want[0, 0])
