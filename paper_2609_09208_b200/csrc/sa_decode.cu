@@ -16,7 +16,7 @@
 namespace sa {
 
 template <int D, int KB, bool NIB, int GT>
-__global__ void __launch_bounds__(128) decode_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kernel(DecodeArgs a) {
     constexpr int EPL = D / 32;
     constexpr int CH = NIB ? D / 32 : D / 16;      // 16-byte code chunks per key
     constexpr int LPT = D / 8;                     // lanes covering one token's value row
@@ -72,17 +72,19 @@ __global__ void __launch_bounds__(128) decode_kernel(DecodeArgs a) {
         const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
 
         // ---- phase 1: integer scores, lane = key ----
-        uint4 kc[CH];
-#pragma unroll
-        for (int c = 0; c < CH; ++c)
-            kc[c] = __ldg(reinterpret_cast<const uint4*>(block + a.kcode_off + ((size_t)c * kPageTokens + tk0 + lane) * 16));
+        // One 16-byte chunk of codes per iteration; the next chunk is already in flight.  The loop
+        // is deliberately not unrolled over chunks: the body (16 or 32 elements x GT queries) is
+        // what has to stay resident in the instruction cache.
+        const uint4* kptr = reinterpret_cast<const uint4*>(block + a.kcode_off) + tk0 + lane;
         const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(block + a.meta_off + (size_t)(tk0 + lane) * 4));
-
         Planes<KB, GT> pl;
         pl.clear();
-#pragma unroll
+        uint4 cur = __ldg(kptr);
+#pragma unroll 1
         for (int c = 0; c < CH; ++c) {
-            const uint32_t w4[4] = {kc[c].x, kc[c].y, kc[c].z, kc[c].w};
+            const uint4 nxt = __ldg(kptr + (size_t)min(c + 1, CH - 1) * kPageTokens);
+            const uint32_t w4[4] = {cur.x, cur.y, cur.z, cur.w};
+            const int32_t* qrow = &q_s[c * (NIB ? 32 : 16)][0];
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
                 const uint32_t w = w4[wi];
@@ -90,22 +92,21 @@ __global__ void __launch_bounds__(128) decode_kernel(DecodeArgs a) {
                     pl.corrections_bytes(w);
 #pragma unroll
                     for (int bi = 0; bi < 4; ++bi) {
-                        const int m = c * 16 + wi * 4 + bi;
                         int32_t q[GT];
-                        load_q<GT>(&q_s[m][0], q);
+                        load_q<GT>(qrow + (wi * 4 + bi) * GT, q);
                         pl.element((w >> (8 * bi)) & 0xffu, q);
                     }
                 } else {
                     pl.corrections_nibbles(w);
 #pragma unroll
                     for (int ni = 0; ni < 8; ++ni) {
-                        const int m = c * 32 + wi * 8 + ni;
                         int32_t q[GT];
-                        load_q<GT>(&q_s[m][0], q);
+                        load_q<GT>(qrow + (wi * 8 + ni) * GT, q);
                         pl.element(((w >> (4 * ni)) & 0xfu) << 4, q);
                     }
                 }
             }
+            cur = nxt;
         }
 
         // ---- phase 2: logits, integer running maximum, weights ----

@@ -82,25 +82,49 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (&red_s)[4][GT][D + 2
     }
 }
 
-// One block per (sequence, query head), D threads: merge the splits and normalise.
+// One block per (sequence, query head): kMergeGroups groups of D threads each take every
+// kMergeGroups-th split (independent, unrolled loads), then the groups are combined in shared
+// memory and the result is normalised.
+constexpr int kMergeGroups = 4;
+
 template <int D>
-__global__ void __launch_bounds__(D) merge_kernel(const float* __restrict__ partials, float* __restrict__ O,
-                                                  int n_splits, int n_rows) {
+__global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __restrict__ partials,
+                                                                 float* __restrict__ O, int n_splits, int n_rows) {
+    __shared__ int m_s[D * kMergeGroups / 32];
+    __shared__ float o_s[kMergeGroups][D + 1];
     const int row = blockIdx.x;                               // b * Hq + h
-    const int dd = threadIdx.x;
+    const int dd = threadIdx.x % D, grp = threadIdx.x / D;
+    const size_t stride = (size_t)n_rows * (D + 2);
+    const float* base = partials + (size_t)row * (D + 2);
+    // global maximum of the integer running maxima
     int Ms = kMNone;
-    for (int s = 0; s < n_splits; ++s)
-        Ms = max(Ms, __float_as_int(partials[((size_t)s * n_rows + row) * (D + 2)]));
+    for (int s = threadIdx.x; s < n_splits; s += D * kMergeGroups) Ms = max(Ms, __float_as_int(base[s * stride]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Ms = max(Ms, __shfl_xor_sync(0xffffffffu, Ms, o));
+    if ((threadIdx.x & 31) == 0) m_s[threadIdx.x >> 5] = Ms;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < D * kMergeGroups / 32; ++w) Ms = max(Ms, m_s[w]);
     float l = 0.0f, o = 0.0f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float* p = partials + ((size_t)s * n_rows + row) * (D + 2);
+#pragma unroll 4
+    for (int s = grp; s < n_splits; s += kMergeGroups) {
+        const float* p = base + s * stride;
         const int M = __float_as_int(p[0]);
-        if (M == kMNone) continue;
-        const float f = pow2i_neg(M - Ms);
+        const float f = (M == kMNone) ? 0.0f : pow2i_neg(M - Ms);
         l += p[1] * f;
         o += p[2 + dd] * f;
     }
-    O[(size_t)row * D + dd] = (l > 0.0f) ? o / l : 0.0f;
+    o_s[grp][dd] = o;
+    if (dd == 0) o_s[grp][D] = l;
+    __syncthreads();
+    if (grp == 0) {
+#pragma unroll
+        for (int g = 1; g < kMergeGroups; ++g) {
+            o += o_s[g][dd];
+            l += o_s[g][D];
+        }
+        O[(size_t)row * D + dd] = (l > 0.0f) ? o / l : 0.0f;
+    }
 }
 
 inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16_t* Q, float* O,
@@ -144,8 +168,8 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
 
 inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s) {
     const int rows = a.batch * a.Hq;
-    if (p.d == 64) merge_kernel<64><<<rows, 64, 0, s>>>(a.partials, a.O, a.n_splits, rows);
-    else merge_kernel<128><<<rows, 128, 0, s>>>(a.partials, a.O, a.n_splits, rows);
+    if (p.d == 64) merge_kernel<64><<<rows, 64 * kMergeGroups, 0, s>>>(a.partials, a.O, a.n_splits, rows);
+    else merge_kernel<128><<<rows, 128 * kMergeGroups, 0, s>>>(a.partials, a.O, a.n_splits, rows);
     return cudaGetLastError() == cudaSuccess ? SA_OK : SA_ERR_CUDA;
 }
 
