@@ -178,6 +178,40 @@ sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const sa_cache* 
                                           const uint16_t* Q, float* O, void* workspace,
                                           size_t workspace_bytes, int stages, sa_stream stream);
 
+/* sa_decode_attention for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the same kernels, not a step of the method.)
+ *
+ * Who needs it: code that must call the decode step from a place where cudaMalloc (or a framework
+ * allocator built on it) is off limits — a plug-in invoked inside another runtime's execution
+ * callback, a serving loop whose device memory pool is frozen once start-up is over, a process
+ * whose allocator may not be re-entered — and that therefore cannot produce the workspace the
+ * normal entry point asks for.  Here the split-K partial results go into a fixed array compiled
+ * into the library instead (SA_STATIC_SCRATCH_BYTES, 256-byte aligned).  The caller still passes
+ * the cache, Q, O and, optionally, dbg_scores, exactly as for sa_decode_attention; results are
+ * identical to it.  The call allocates nothing and frees nothing.
+ *
+ * Costs and rules:
+ *   - Every GPU on which the library is used holds SA_STATIC_SCRATCH_BYTES from the moment the
+ *     library's code is loaded on it until the process exits, whether or not this entry point is
+ *     ever called.
+ *   - The scratch bounds the problem: with S the split count the library picks for the cache
+ *     shape, S * batch * n_q_heads * (head_dim + 2) * 4 bytes must fit.  A larger problem is
+ *     refused with SA_ERR_CAPACITY and nothing is launched; use sa_decode_attention with a
+ *     workspace of sa_workspace_bytes() for it.  (Batch 1, 32 query heads, head_dim 64 at any
+ *     length fits; so does the ragged batch-16 configuration.)
+ *   - The first call on each device looks up the array's device address (one CUDA runtime query,
+ *     made with that device current, then cached).  Make that first call outside any stream
+ *     capture; later calls on the same device do no such query.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     Nothing in it has to be cleared — each call overwrites every entry it later reads — but two
+ *     calls that overlap on the GPU (different streams, or graphs replayed concurrently) race on
+ *     it and corrupt each other's output.  Serialise them, or give the overlapping ones their own
+ *     workspace through sa_decode_attention.
+ *   - cfg->code must be one of the power-of-two codes (not SA_KV_FP16). */
+#define SA_STATIC_SCRATCH_BYTES (4u << 20)
+sa_status sa_decode_attention_static(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                                     float* O, int32_t* dbg_scores, sa_stream stream);
+
 /* Test hook: unpack sequence b of a quantised cache into canonical arrays for its first
  * n_tokens tokens: codes [n_tokens, n_kv_heads, head_dim] canonical bytes, scales
  * [n_tokens, n_kv_heads] binary16, v_hat [n_tokens, n_kv_heads, head_dim] int8, g

@@ -22,6 +22,7 @@ EXPORTS = [
     "sa_version", "sa_status_string", "sa_get_layout", "sa_workspace_bytes", "sa_encode_keys",
     "sa_quantise_query", "sa_quantise_values", "sa_append_kv", "sa_fill_kv", "sa_decode_attention",
     "sa_decode_attention_fp16", "sa_decode_attention_stages", "sa_decode_attention_fp16_stages", "sa_debug_unpack", "sa_staging_bytes", "sa_decode_step_host",
+    "sa_decode_attention_static",
 ]
 
 
@@ -165,6 +166,17 @@ def decode_attention_fp16(cfg, cache: SaCache, Q, O, workspace, stages: int = 3)
                                                    C.c_size_t(workspace.numel() * workspace.element_size()),
                                                    C.c_int(stages), _stream())
     _check(st, "sa_decode_attention_fp16")
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def decode_attention_static(cfg, cache: SaCache, Q, O, dbg_scores=None):
+    """sa_decode_attention without a caller workspace: the split-K partials use the library's fixed
+    scratch array (for callers that cannot allocate device memory).  Raises SaError(status 4) when the
+    problem needs more than STATIC_SCRATCH_BYTES.  Calls sharing a device must not overlap on the GPU."""
+    _check(lib().sa_decode_attention_static(C.byref(cfg), C.byref(cache), _ptr(Q), _ptr(O), _ptr(dbg_scores),
+                                            _stream()), "sa_decode_attention_static")
 
 
 def debug_unpack(cfg, cache: SaCache, b: int, n_tokens: int, codes=None, scales=None, v_hat=None, g=None):

@@ -225,3 +225,64 @@ extern "C" sa_status sa_decode_attention(const sa_config* cfg, const sa_cache* c
                                          int32_t* dbg_scores, sa_stream stream) {
     return sa_decode_attention_stages(cfg, cache, Q, O, workspace, workspace_bytes, dbg_scores, 3, stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// Decode attention for callers that cannot allocate device memory.
+//
+// Some hosts of this library have no way to hand it a workspace: code that runs where
+// cudaMalloc is forbidden or unavailable (a plug-in called inside another runtime's execution
+// callback, a latency-critical serving loop whose memory pool is frozen after start-up, a host
+// process whose allocator must not be re-entered).  For them the split-K partials live in the
+// fixed array below, which is part of the library image: every GPU on which the library's module
+// is loaded holds these SA_STATIC_SCRATCH_BYTES until the process exits.
+//
+// The array's name is only a host-side stand-in for the symbol; the device address is obtained
+// once per device with cudaGetSymbolAddress and cached.
+// ---------------------------------------------------------------------------------------------
+#include <mutex>
+
+static __device__ __align__(256) unsigned char sa_static_scratch[SA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxScratchDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxScratchDevices] = {};
+
+// Device address of sa_static_scratch on the CURRENT device (looked up on first use).
+sa_status static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxScratchDevices) return SA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, sa_static_scratch) != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return SA_ERR_CUDA;
+        }
+        g_scratch_addr[dev] = ptr;
+    }
+    *out = g_scratch_addr[dev];
+    return SA_OK;
+}
+}  // namespace
+
+extern "C" sa_status sa_decode_attention_static(const sa_config* cfg, const sa_cache* cache,
+                                                const uint16_t* Q, float* O, int32_t* dbg_scores,
+                                                sa_stream stream) {
+    Plan p;
+    sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    if (p.fp16) return SA_ERR_UNSUPPORTED;
+    if (!cache || cache->batch <= 0 || cache->max_pages_per_seq <= 0) return SA_ERR_INVALID_ARG;
+    int S, GT;
+    split_plan(p, cache->batch, cache->max_pages_per_seq, &S, &GT);
+    const size_t need = (size_t)S * cache->batch * p.Hq * (p.d + 2) * sizeof(float);
+    if (need > (size_t)SA_STATIC_SCRATCH_BYTES) return SA_ERR_CAPACITY;   // problem too large for the fixed scratch
+    void* scratch = nullptr;
+    st = static_scratch_address(&scratch);
+    if (st != SA_OK) return st;
+    // Nothing in the scratch has to start at zero: the main kernel writes every partial that the
+    // merge kernel reads, so contents left by an earlier call are simply overwritten.
+    return sa_decode_attention_stages(cfg, cache, Q, O, scratch, (size_t)SA_STATIC_SCRATCH_BYTES, dbg_scores, 3,
+                                      stream);
+}
