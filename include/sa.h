@@ -30,10 +30,12 @@
  *   The page pool is n_pages * n_kv_heads blocks of `page_bytes`; block (p, h) starts at
  *   ((size_t)p * n_kv_heads + h) * page_bytes and holds page_tokens = 64 tokens of KV head h:
  *     kcode_off: key codes in 16-byte chunks, chunk c of token t at (c * 64 + t) * 16.
- *                Byte container (any k): chunk c holds elements 16c .. 16c+15, one canonical
- *                byte each.  Nibble container (PoT-4 only): chunk c holds elements 32c .. 32c+31,
- *                byte i = element 32c+2i in the low nibble and 32c+2i+1 in the high nibble,
- *                nibble = sign << 3 | e.
+ *                Byte container (any k): chunk c holds elements 16c .. 16c+15, one byte each:
+ *                the canonical byte with its exponent field replaced by g = 7 - e (g = 0 for the
+ *                zero code), i.e. canonical ^ 0x70, so that g - 1 is the shift amount and zeroed
+ *                memory reads as zero codes.  Nibble container (PoT-4 only): chunk c holds
+ *                elements 32c .. 32c+31, byte i = element 32c+2i in the low nibble and 32c+2i+1
+ *                in the high nibble, nibble = sign << 3 | g.
  *     meta_off : 64 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.
  *     v_off    : vhat, int8, row-major [64][head_dim].
  *   For code = SA_KV_FP16 the block holds unquantised binary16 data: K in 16-byte chunks of 8
@@ -211,6 +213,16 @@ sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const sa_cache* 
 #define SA_STATIC_SCRATCH_BYTES (4u << 20)
 sa_status sa_decode_attention_static(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                                      float* O, int32_t* dbg_scores, sa_stream stream);
+
+/* Instruction-throughput micro-benchmark (measurement aid; the paper has no counterpart — it stands
+ * in for the paper's disassembly-based operation counts, section III and Table V).  Launches `blocks`
+ * blocks of 256 threads in which every thread runs iters * 64 instructions of one kind on 8
+ * independent chains.  kind: 0 variable shift, 1 three-input logic op, 2 three-input add,
+ * 3 multiply-add by one (an add issued on the FMA pipe), 4 byte permute, 5 shift/multiply-add mix,
+ * 6 logic/multiply-add mix, 7 FP32 FMA, 8 packed FP32x2 FMA, 9 integer multiply-add, 10 dp4a,
+ * 11 population count + add, 12 int8-to-float + add, 13 shift/logic/multiply-add mix.
+ * `sink` is one device word (practically never written).  The caller times the launch. */
+sa_status sa_pipe_microbench(int kind, int iters, int blocks, uint32_t* sink, sa_stream stream);
 
 /* Test hook: unpack sequence b of a quantised cache into canonical arrays for its first
  * n_tokens tokens: codes [n_tokens, n_kv_heads, head_dim] canonical bytes, scales

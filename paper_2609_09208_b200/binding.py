@@ -22,7 +22,7 @@ EXPORTS = [
     "sa_version", "sa_status_string", "sa_get_layout", "sa_workspace_bytes", "sa_encode_keys",
     "sa_quantise_query", "sa_quantise_values", "sa_append_kv", "sa_fill_kv", "sa_decode_attention",
     "sa_decode_attention_fp16", "sa_decode_attention_stages", "sa_decode_attention_fp16_stages", "sa_debug_unpack", "sa_staging_bytes", "sa_decode_step_host",
-    "sa_decode_attention_static",
+    "sa_decode_attention_static", "sa_pipe_microbench",
 ]
 
 
@@ -166,6 +166,15 @@ def decode_attention_fp16(cfg, cache: SaCache, Q, O, workspace, stages: int = 3)
                                                    C.c_size_t(workspace.numel() * workspace.element_size()),
                                                    C.c_int(stages), _stream())
     _check(st, "sa_decode_attention_fp16")
+
+
+PIPE_KINDS = ["shl", "lop3", "iadd3", "imad_by_one", "prmt", "shl+imad1", "lop3+imad1", "ffma", "ffma2",
+              "imad", "dp4a", "popc+add", "i2f+fadd", "shl+lop3+imad1"]
+
+
+def pipe_microbench(kind: int, iters: int, blocks: int, sink):
+    _check(lib().sa_pipe_microbench(C.c_int(kind), C.c_int(iters), C.c_int(blocks), _ptr(sink), _stream()),
+           "sa_pipe_microbench")
 
 
 STATIC_SCRATCH_BYTES = 4 << 20

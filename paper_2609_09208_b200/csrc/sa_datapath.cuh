@@ -1,11 +1,35 @@
-// The integer score datapath of the decode kernel, kept free of anything that only compiles for
-// the device so that its arithmetic can also be exercised on the host by the unit tests.
+// The integer score datapath of the decode kernel (section II-B eq. (3), II-C eq. (4), II-D
+// eq. (5)): shifts, sign flips, masks and adds only.  Everything here also compiles for the host so
+// that the unit tests can run the very same arithmetic against the CPU oracle without a GPU.
+//
+// Term of element m at head-room F0 = 6 + KB:  sigma * (qhat << r) * (2^KB + j),  r = 6 - e >= 0.
+//
+// * Two queries share one 32-bit register: P = (q_hi << 16) + q_lo as a 32-bit integer (a negative
+//   q_lo borrows from the upper half; all arithmetic below is plain integer arithmetic on P, so
+//   the two halves stay exact as long as the lower half's running sum fits in 16 bits).  One
+//   shift, one logic op and one add then serve two (query, element) pairs.
+// * The mantissa is handled in KB + 1 "planes": plane KB takes sigma*(P << r) of every element,
+//   plane b < KB only of the elements whose mantissa bit b is set; score = sum_b plane_b << b.
+// * The sign flip is a bitwise complement fused with the plane mask into one logic op
+//   ((x ^ S) & m); the "+1" that a two's complement would add is restored per key from population
+//   counts of the sign bits (it only concerns the lower half: the upper half of ~x is exact).
+// * A window of 4 elements (4 * 127 * 2^6 + 4 < 2^15) is accumulated in the packed register,
+//   whose lower half is biased by 0x8000 so that it never borrows; then both halves are added
+//   into 32-bit totals, weighted by the plane's 2^b.
+// * Adds are written as multiply-add by a 1 the compiler cannot see, so that they issue on the
+//   FMA pipe while shifts and logic ops issue on the ALU pipe: on sm_100a the two pipes run side
+//   by side (64 + 64 thread-instructions per clock per SM), and the integer ALU pipe is what
+//   bounds this kernel.
+//
+// Physical code format inside a page (differs from the canonical byte only in the exponent field):
+// byte = sign << 7 | g << 4 | mantissa, g = 7 - e for a non-zero element and 0 for the zero code,
+// i.e. physical = canonical ^ 0x70 (and nibble = canonical nibble ^ 0x7).  The shift amount is
+// g - 1, which is 0xffffffff for the zero code, and a shift by 32 or more returns 0.
 #pragma once
 #include "sa_common.cuh"
 
 namespace sa {
 
-// Left shift that returns 0 for amounts >= 32 (PTX shl.b32 semantics).
 SA_HD uint32_t shl_clamp_hd(uint32_t x, uint32_t n) {
 #ifdef __CUDA_ARCH__
     return shl_clamp(x, n);
@@ -20,61 +44,171 @@ SA_HD int popc_hd(uint32_t x) {
     return __builtin_popcount(x);
 #endif
 }
+// Byte permute with the generic PTX semantics: selector nibble n picks byte (n & 7) of {a, b};
+// with bit 3 set the byte's most significant bit is replicated over the result byte instead.
+SA_HD uint32_t prmt_hd(uint32_t a, uint32_t b, uint32_t sel) {
+#ifdef __CUDA_ARCH__
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+#else
+    const unsigned long long ab = ((unsigned long long)b << 32) | a;
+    uint32_t d = 0;
+    for (int n = 0; n < 4; ++n) {
+        const uint32_t s = (sel >> (4 * n)) & 0xfu;
+        uint32_t byte = (uint32_t)(ab >> (8 * (s & 7u))) & 0xffu;
+        if (s & 8u) byte = (byte & 0x80u) ? 0xffu : 0x00u;
+        d |= byte << (8 * n);
+    }
+    return d;
+#endif
+}
+// a + b, issued as a * one + b (one == 1 at run time) so that it executes on the FMA pipe.
+SA_HD uint32_t add_fma(uint32_t a, uint32_t b, uint32_t one) {
+#ifdef __CUDA_ARCH__
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(one), "r"(b));
+    return d;
+#else
+    return a * one + b;
+#endif
+}
 
-// -------------------------------------------------------------------------------------------
-// Integer scores of one key against GT queries: shift / sign-flip / add only.
+// NP consecutive 32-bit words (NP = 1, 2 or 4; 4 * NP-byte aligned) with one vector load.
+template <int NP>
+SA_HD void load_np(const uint32_t* src, uint32_t (&q)[NP]) {
+    if constexpr (NP == 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(src);
+        q[0] = v.x; q[1] = v.y; q[2] = v.z; q[3] = v.w;
+    } else if constexpr (NP == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(src);
+        q[0] = v.x; q[1] = v.y;
+    } else {
+        q[0] = src[0];
+    }
+}
+
+// a * w + c on the FMA pipe (w is a power of two held in a register: a shift-and-add).
+SA_HD uint32_t mad_fma(uint32_t a, uint32_t w, uint32_t c) {
+#ifdef __CUDA_ARCH__
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(w), "r"(c));
+    return d;
+#else
+    return a * w + c;
+#endif
+}
+
+SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (uint32_t)q_lo; }
+
+// Accumulators for 2 * NP queries against one key.
 //
-// With F0 = 6 + KB the term of element m is  sigma * (qhat << r) * (2^KB + j),  r = 6 - e >= 0.
-// It is accumulated in KB + 1 "planes": plane KB takes sigma*(qhat << r) of every element, plane
-// b < KB only of the elements whose mantissa bit b is set; the score is
-// sum_b plane_b << b.  The sign flip is a bitwise complement (x ^ S, S = 0 or -1) and the
-// missing "+1" of the two's complement is added per key from population counts of the sign
-// bits, which all GT queries share.  The zero code gives r = 0xffffffff, for which the shift
-// returns 0.
-// -------------------------------------------------------------------------------------------
-template <int KB, int GT>
-struct Planes {
-    int32_t acc[KB + 1][GT];
-    int32_t corr[KB + 1];
-    SA_HD void clear() {
+// Flush of a window register W = h * 2^16 + l (l = biased lower half, 0 <= l < 2^16): instead of
+// separating both halves, two totals are kept modulo 2^32,
+//     tot += W << b        and        hit += h << b        (h = W >> 16, arithmetic),
+// and at the end  lower-query sum = tot - (hit << 16)  (exact: the true value is far below 2^32)
+// and  upper-query sum = hit.  That is one ALU instruction and two FMA-pipe multiply-adds (by the
+// plane weight 2^b held in a register) per window register.
+template <int KB, int NP>
+struct PackedPlanes {
+    uint32_t win[KB + 1][NP];   // window sums, lower half biased by 0x8000
+    uint32_t tot[NP], hit[NP];  // running totals, see above
+    uint32_t corr;              // sum_b 2^b * (number of complemented terms in plane b)
+    uint32_t n_windows;
+    uint32_t pw[KB + 1];        // plane weights 2^b as run-time values (pw[0] doubles as the opaque 1)
+
+    SA_HD void begin(uint32_t one) {
+        corr = 0;
+        n_windows = 0;
 #pragma unroll
-        for (int b = 0; b <= KB; ++b) {
-            corr[b] = 0;
+        for (int b = 0; b <= KB; ++b) pw[b] = one << b;
 #pragma unroll
-            for (int g = 0; g < GT; ++g) acc[b][g] = 0;
+        for (int p = 0; p < NP; ++p) tot[p] = hit[p] = 0;
+    }
+    // r: shift amount (>= 32 for the zero code); S: 0 or 0xffffffff; mask[b]: 0 or 0xffffffff.
+    // FIRST: the first element of a window starts from the bias instead of the previous sum.
+    template <bool FIRST>
+    SA_HD void element(uint32_t r, uint32_t S, const uint32_t* mask, const uint32_t* qp) {
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const uint32_t x = shl_clamp_hd(qp[p], r);
+            win[KB][p] = add_fma(x ^ S, FIRST ? 0x8000u : win[KB][p], pw[0]);
+#pragma unroll
+            for (int b = 0; b < KB; ++b) win[b][p] = add_fma((x ^ S) & mask[b], FIRST ? 0x8000u : win[b][p], pw[0]);
         }
     }
-    // one element: canonical code byte `cb` (only bits 7..(4-KB) are looked at), queries q[g]
-    SA_HD void element(uint32_t cb, const int32_t (&q)[GT]) {
-        const uint32_t r = 6u - ((cb >> 4) & 7u);
-        const int32_t S = -(int32_t)((cb >> 7) & 1u);
-        int32_t mask[KB > 0 ? KB : 1];
+    SA_HD void window_end() {
+        ++n_windows;
 #pragma unroll
-        for (int b = 0; b < KB; ++b) mask[b] = -(int32_t)((cb >> (4 - KB + b)) & 1u);
+        for (int b = 0; b <= KB; ++b)
 #pragma unroll
-        for (int g = 0; g < GT; ++g) {
-            const int32_t xs = (int32_t)shl_clamp_hd((uint32_t)q[g], r) ^ S;
-            acc[KB][g] += xs;
-#pragma unroll
-            for (int b = 0; b < KB; ++b) acc[b][g] += xs & mask[b];
-        }
+            for (int p = 0; p < NP; ++p) {
+                const uint32_t h = (uint32_t)((int32_t)win[b][p] >> 16);      // exact upper half
+                tot[p] = mad_fma(win[b][p], pw[b], tot[p]);
+                hit[p] = mad_fma(h, pw[b], hit[p]);
+            }
     }
-    // four canonical bytes in one word: the +1 corrections of the complemented terms
-    SA_HD void corrections_bytes(uint32_t w) {
-        const uint32_t neg = w & 0x80808080u;
-        corr[KB] += popc_hd(neg);
-#pragma unroll
-        for (int b = 0; b < KB; ++b) corr[b] += popc_hd(neg & (w << (3 + KB - b)));
-    }
-    // eight nibbles (sign << 3 | e) in one word (PoT-4 only)
-    SA_HD void corrections_nibbles(uint32_t w) { corr[KB] += popc_hd(w & 0x88888888u); }
-    SA_HD int32_t score(int g, int f_extra) const {
-        // unsigned arithmetic: the shifts are exact modulo 2^32 and the true sum fits in INT32
-        uint32_t a = (uint32_t)(acc[KB][g] + corr[KB]) << KB;
-#pragma unroll
-        for (int b = 0; b < KB; ++b) a += (uint32_t)(acc[b][g] + corr[b]) << b;
-        return (int32_t)(a << f_extra);
+    // score of query g (g even: lower half of register g / 2), before the final head-room shift
+    SA_HD int32_t score(int g) const {
+        const uint32_t bias = n_windows * 0x8000u * ((2u << KB) - 1u);
+        return (g & 1) ? (int32_t)hit[g >> 1] : (int32_t)(tot[g >> 1] - (hit[g >> 1] << 16) - bias + corr);
     }
 };
+
+// One 32-bit word of the byte container = 4 elements.  qp points at the packed queries of the
+// word's first element; consecutive elements are `stride` words apart.
+template <int KB, int NP>
+SA_HD void accumulate_word_bytes(PackedPlanes<KB, NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
+    // shift amounts g - 1 per byte: 0..6, and 0xff for the zero code (g = 0)
+    const uint32_t gw = (w >> 4) & 0x07070707u;
+    const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;
+    const uint32_t neg = w & 0x80808080u;
+    uint32_t wb[KB > 0 ? KB : 1];
+    pl.corr += (uint32_t)popc_hd(neg) << KB;
+#pragma unroll
+    for (int b = 0; b < KB; ++b) {
+        wb[b] = w << (3 + KB - b);              // mantissa bit b of every byte moved to the byte's top bit
+        pl.corr += (uint32_t)popc_hd(neg & wb[b]) << b;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t rep = 0x8888u | (0x1111u * i);          // replicate the top bit of byte i
+        const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);       // byte i, zero-extended
+        const uint32_t S = prmt_hd(w, 0u, rep);
+        uint32_t mask[KB > 0 ? KB : 1];
+#pragma unroll
+        for (int b = 0; b < KB; ++b) mask[b] = prmt_hd(wb[b], 0u, rep);
+        uint32_t q[NP];
+        load_np<NP>(qp + i * stride, q);
+        if (i == 0) pl.template element<true>(r, S, mask, q);
+        else pl.template element<false>(r, S, mask, q);
+    }
+    pl.window_end();
+}
+
+// One 32-bit word of the nibble container (PoT-4 only) = 8 elements, two windows.
+template <int NP>
+SA_HD void accumulate_word_nibbles(PackedPlanes<0, NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
+    const uint32_t ge = w & 0x07070707u, go = (w >> 4) & 0x07070707u;   // g of even / odd elements
+    const uint32_t re = (ge + 0x7f7f7f7fu) ^ 0x80808080u, ro = (go + 0x7f7f7f7fu) ^ 0x80808080u;
+    const uint32_t we = w << 4;                                         // even elements' sign at the byte's top bit
+    pl.corr += (uint32_t)popc_hd(w & 0x88888888u);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int ni = half * 4 + i;                                // element within the word
+            const int byte = ni >> 1;
+            const uint32_t rep = 0x8888u | (0x1111u * byte);
+            const uint32_t r = prmt_hd((ni & 1) ? ro : re, 0u, 0x4440u | byte);
+            const uint32_t S = prmt_hd((ni & 1) ? w : we, 0u, rep);
+            uint32_t q[NP];
+            load_np<NP>(qp + ni * stride, q);
+            if (i == 0) pl.template element<true>(r, S, nullptr, q);
+            else pl.template element<false>(r, S, nullptr, q);
+        }
+        pl.window_end();
+    }
+}
 
 }  // namespace sa

@@ -16,13 +16,16 @@
 namespace sa {
 
 template <int D, int KB, bool NIB, int GT>
-__global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
     constexpr int EPL = D / 32;
     constexpr int CH = NIB ? D / 32 : D / 16;      // 16-byte code chunks per key
-    constexpr int LPT = D / 8;                     // lanes covering one token's value row
+    constexpr int NJ = 2;                          // output-dim pairs per lane in the A.V phase (4 dims)
+    constexpr int LPT = D / (2 * NJ);              // lanes covering one token's value row
     constexpr int TS = 32 / LPT;                   // token groups in the A.V phase
     constexpr int TPL = 32 / TS;                   // tokens per lane per tile
-    __shared__ __align__(16) int32_t q_s[D][GT];
+    constexpr int NP = (GT + 1) / 2;               // packed query registers: two queries each
+    __shared__ int32_t q_s[D][GT];
+    __shared__ __align__(16) uint32_t qp_s[D][NP];
     __shared__ float qscale_s[GT];
     __shared__ __align__(16) float2 p_s[4][32][GT];
     __shared__ __align__(16) float red_s[4][GT][D + 2];
@@ -45,6 +48,11 @@ __global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kern
         if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
     }
     __syncthreads();
+    for (int idx = threadIdx.x; idx < D * NP; idx += 128) {
+        const int m = idx / NP, p = idx % NP;
+        qp_s[m][p] = pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0);
+    }
+    __syncthreads();
 
     const int len = a.seq_lens[b];
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
@@ -53,13 +61,13 @@ __global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kern
 
     int M[GT];
     float l[GT];
-    unsigned long long acc[GT][4];
+    unsigned long long acc[GT][NJ];
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         M[g] = kMNone;
         l[g] = 0.0f;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[g][j] = 0ull;
+        for (int j = 0; j < NJ; ++j) acc[g][j] = 0ull;
     }
     const int ts = lane / LPT, dc = lane % LPT;
 
@@ -77,34 +85,17 @@ __global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kern
         // what has to stay resident in the instruction cache.
         const uint4* kptr = reinterpret_cast<const uint4*>(block + a.kcode_off) + tk0 + lane;
         const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(block + a.meta_off + (size_t)(tk0 + lane) * 4));
-        Planes<KB, GT> pl;
-        pl.clear();
+        PackedPlanes<KB, NP> pl;
+        pl.begin(a.one);
         uint4 cur = __ldg(kptr);
 #pragma unroll 1
         for (int c = 0; c < CH; ++c) {
             const uint4 nxt = __ldg(kptr + (size_t)min(c + 1, CH - 1) * kPageTokens);
             const uint32_t w4[4] = {cur.x, cur.y, cur.z, cur.w};
-            const int32_t* qrow = &q_s[c * (NIB ? 32 : 16)][0];
 #pragma unroll
             for (int wi = 0; wi < 4; ++wi) {
-                const uint32_t w = w4[wi];
-                if (!NIB) {
-                    pl.corrections_bytes(w);
-#pragma unroll
-                    for (int bi = 0; bi < 4; ++bi) {
-                        int32_t q[GT];
-                        load_q<GT>(qrow + (wi * 4 + bi) * GT, q);
-                        pl.element((w >> (8 * bi)) & 0xffu, q);
-                    }
-                } else {
-                    pl.corrections_nibbles(w);
-#pragma unroll
-                    for (int ni = 0; ni < 8; ++ni) {
-                        int32_t q[GT];
-                        load_q<GT>(qrow + (wi * 8 + ni) * GT, q);
-                        pl.element(((w >> (4 * ni)) & 0xfu) << 4, q);
-                    }
-                }
+                if constexpr (!NIB) accumulate_word_bytes<KB, NP>(pl, w4[wi], &qp_s[c * 16 + wi * 4][0], NP);
+                else accumulate_word_nibbles<NP>(pl, w4[wi], &qp_s[c * 32 + wi * 8][0], NP);
             }
             cur = nxt;
         }
@@ -118,7 +109,7 @@ __global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kern
         float resc[GT];
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
-            const int32_t A = pl.score(g, a.f_extra);
+            const int32_t A = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
             if (a.dbg_scores && valid)
                 a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A;
             const float z = valid ? (float)A * qscale_s[g] * s_j : -INFINITY;
@@ -138,34 +129,32 @@ __global__ void __launch_bounds__(128, (KB == 4 && GT == 8) ? 3 : 4) decode_kern
             for (int g = 0; g < GT; ++g) {
                 const unsigned long long r2 = pack_f32x2(resc[g], resc[g]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
+                for (int j = 0; j < NJ; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
             }
         }
         __syncwarp();
 
-        // ---- phase 3: O += p * vhat * 2^-g, lane = (token group, 8 dims) ----
-        const uint8_t* vbase = block + a.v_off + (size_t)tk0 * D + dc * 8;
+        // ---- phase 3: O += p * vhat * 2^-g, lane = (token group, 4 dims) ----
+        const uint8_t* vbase = block + a.v_off + (size_t)tk0 * D + dc * (2 * NJ);
 #pragma unroll 4
         for (int i = 0; i < TPL; ++i) {
             const int t = ts + TS * i;
-            const uint2 vv = __ldg(reinterpret_cast<const uint2*>(vbase + (size_t)t * D));
-            unsigned long long v2[4];
-            v2[0] = pack_f32x2((float)(int8_t)(vv.x), (float)(int8_t)(vv.x >> 8));
-            v2[1] = pack_f32x2((float)(int8_t)(vv.x >> 16), (float)(int8_t)(vv.x >> 24));
-            v2[2] = pack_f32x2((float)(int8_t)(vv.y), (float)(int8_t)(vv.y >> 8));
-            v2[3] = pack_f32x2((float)(int8_t)(vv.y >> 16), (float)(int8_t)(vv.y >> 24));
+            const uint32_t vv = __ldg(reinterpret_cast<const uint32_t*>(vbase + (size_t)t * D));
+            unsigned long long v2[NJ];
+            v2[0] = pack_f32x2((float)(int8_t)(vv), (float)(int8_t)(vv >> 8));
+            v2[1] = pack_f32x2((float)(int8_t)(vv >> 16), (float)(int8_t)(vv >> 24));
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&p_s[warp][t][g]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[g][j] = ffma2(v2[j], pp, acc[g][j]);
+                for (int j = 0; j < NJ; ++j) acc[g][j] = ffma2(v2[j], pp, acc[g][j]);
             }
         }
         __syncwarp();
     }
 
     // ---- merge the four warps of the block, write the block's partial ----
-    block_merge_and_store<D, GT>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
+    block_merge_and_store<D, GT, NJ>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
 }
 
 }  // namespace sa

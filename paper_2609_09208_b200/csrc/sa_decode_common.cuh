@@ -19,6 +19,7 @@ struct DecodeArgs {
     int batch, Hq, Hkv, G, max_pages, n_pages, n_splits, f_extra, hadamard;
     size_t page_bytes, kcode_off, meta_off, v_off;
     float zscale;
+    uint32_t one;             // the value 1, opaque to the compiler (adds issued as multiply-add)
 };
 
 template <int GT>
@@ -38,16 +39,16 @@ SA_D void load_q(const int32_t* src, int32_t (&q)[GT]) {
 }
 
 // Per-warp states (M, l, O) -> one partial per block.  acc[g][j] holds output dims
-// dc*8 + 2j, dc*8 + 2j + 1 summed over this lane's token group; token groups sit LPT lanes apart.
-template <int D, int GT>
+// dc*2*NJ + 2j, dc*2*NJ + 2j + 1 summed over this lane's token group; token groups sit LPT lanes apart.
+template <int D, int GT, int NJ>
 SA_D void block_merge_and_store(const DecodeArgs& a, float (&red_s)[4][GT][D + 2], const int (&M)[GT],
-                                float (&l)[GT], unsigned long long (&acc)[GT][4], int lane, int warp,
+                                float (&l)[GT], unsigned long long (&acc)[GT][NJ], int lane, int warp,
                                 int ts, int dc, int LPT, int b, int h0, int split) {
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         const float lsum = warp_sum_f32(l[g]);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < NJ; ++j) {
             float lo, hi;
             unpack_f32x2(acc[g][j], &lo, &hi);
             for (int off = LPT; off < 32; off <<= 1) {
@@ -55,8 +56,8 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (&red_s)[4][GT][D + 2
                 hi += __shfl_xor_sync(0xffffffffu, hi, off);
             }
             if (ts == 0) {
-                red_s[warp][g][2 + dc * 8 + 2 * j] = lo;
-                red_s[warp][g][2 + dc * 8 + 2 * j + 1] = hi;
+                red_s[warp][g][2 + dc * (2 * NJ) + 2 * j] = lo;
+                red_s[warp][g][2 + dc * (2 * NJ) + 2 * j + 1] = hi;
             }
         }
         if (lane == 0) {
@@ -162,6 +163,7 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->meta_off = p.lay.meta_off;
     a->v_off = p.lay.v_off;
     a->zscale = 0.0f;
+    a->one = 1u;
     *gt = GT;
     return SA_OK;
 }

@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(128) decode_fp16_kernel(DecodeArgs a) {
         __syncwarp();
     }
 
-    block_merge_and_store<D, GT>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
+    block_merge_and_store<D, GT, 4>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
 }
 
 }  // namespace sa

@@ -88,6 +88,9 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
     uint8_t kc[EPL], vc[EPL];
     const uint32_t smax = encode_key_vec<EPL, K>(kb, lane, a.hadamard != 0, kc);
     const int gg = quantise_value_vec<EPL>(vb, vc);
+    // physical exponent field g = 7 - e (0 for the zero code): canonical byte ^ 0x70
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) kc[i] ^= 0x70;
     uint8_t* kdst = block + a.kcode_off;
     if (!NIB) {
         const int m = lane * EPL;                   // first element of this lane
@@ -192,13 +195,13 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
         if (!NIB) {
             const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) c[i] = src[i];
+            for (int i = 0; i < EPL; ++i) c[i] = src[i] ^ 0x70;
         } else {
             const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 5) * kPageTokens + t) * 16 + ((m & 31) >> 1);
 #pragma unroll
             for (int i = 0; i < EPL / 2; ++i) {
-                c[2 * i] = (uint8_t)(src[i] << 4);
-                c[2 * i + 1] = (uint8_t)(src[i] & 0xf0);
+                c[2 * i] = (uint8_t)((src[i] << 4) ^ 0x70);
+                c[2 * i + 1] = (uint8_t)((src[i] & 0xf0) ^ 0x70);
             }
         }
         store_bytes<EPL>(codes + (size_t)v * D + m, c);

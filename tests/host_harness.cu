@@ -5,27 +5,29 @@
 
 using namespace sa;
 
+// Scores of one key (canonical code bytes) against 8 queries, through the same packed plane
+// datapath and word decoders the decode kernel uses (physical codes = canonical ^ 0x70).
 template <int K>
-static int32_t score_one(const uint8_t* codes, const int8_t* q, int d, int f_extra, bool nibble_path) {
-    Planes<K, 1> pl;
-    pl.clear();
-    for (int m0 = 0; m0 < d; m0 += 4) {
-        uint32_t w = 0;
-        for (int i = 0; i < 4; ++i) w |= (uint32_t)codes[m0 + i] << (8 * i);
-        if (!nibble_path) pl.corrections_bytes(w);
-        for (int i = 0; i < 4; ++i) {
-            const int32_t qq[1] = {q[m0 + i]};
-            pl.element((w >> (8 * i)) & 0xffu, qq);
+static void score8(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
+    alignas(16) static uint32_t qp[128][4];
+    for (int m = 0; m < d; ++m)
+        for (int p = 0; p < 4; ++p) qp[m][p] = pack_pair(q8[(2 * p) * d + m], q8[(2 * p + 1) * d + m]);
+    PackedPlanes<K, 4> pl;
+    pl.begin(1u);
+    if (!nibble_path) {
+        for (int m0 = 0; m0 < d; m0 += 4) {
+            uint32_t w = 0;
+            for (int i = 0; i < 4; ++i) w |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * i);
+            accumulate_word_bytes<K, 4>(pl, w, &qp[m0][0], 4);
         }
-    }
-    if (nibble_path) {  // eight sign/exponent nibbles per word
+    } else if constexpr (K == 0) {
         for (int m0 = 0; m0 < d; m0 += 8) {
             uint32_t w = 0;
-            for (int i = 0; i < 8; ++i) w |= (uint32_t)(codes[m0 + i] >> 4) << (4 * i);
-            pl.corrections_nibbles(w);
+            for (int i = 0; i < 8; ++i) w |= (uint32_t)((canon[m0 + i] ^ 0x70) >> 4) << (4 * i);
+            accumulate_word_nibbles<4>(pl, w, &qp[m0][0], 4);
         }
     }
-    return pl.score(0, f_extra);
+    for (int g = 0; g < 8; ++g) out[g] = pl.score(g);
 }
 
 extern "C" {
@@ -41,12 +43,12 @@ void hh_encode_many(int k, const uint16_t* a_bits, int64_t n, unsigned s_bits, u
     for (int64_t i = 0; i < n; ++i) out[i] = (uint8_t)hh_encode_element(k, a_bits[i], s_bits);
 }
 int hh_value_exponent(unsigned amax_bits) { return value_exponent(amax_bits); }
-int32_t hh_score(int k, const uint8_t* codes, const int8_t* q, int d, int f_extra, int nibble_path) {
+void hh_score8(int k, const uint8_t* canon, const int8_t* q8, int d, int nibble_path, int32_t* out) {
     switch (k) {
-        case 0: return score_one<0>(codes, q, d, f_extra, nibble_path != 0);
-        case 1: return score_one<1>(codes, q, d, f_extra, false);
-        case 2: return score_one<2>(codes, q, d, f_extra, false);
-        default: return score_one<4>(codes, q, d, f_extra, false);
+        case 0: score8<0>(canon, q8, d, nibble_path != 0, out); break;
+        case 1: score8<1>(canon, q8, d, false, out); break;
+        case 2: score8<2>(canon, q8, d, false, out); break;
+        default: score8<4>(canon, q8, d, false, out); break;
     }
 }
 }

@@ -26,7 +26,6 @@ def hh():
         subprocess.check_call(["/usr/local/cuda/bin/nvcc", "-std=c++17", "-O2", "-shared", "-Xcompiler", "-fPIC",
                                "-Wno-deprecated-gpu-targets", "-o", LIB, SRC])
     lib = C.CDLL(LIB)
-    lib.hh_score.restype = C.c_int32
     return lib
 
 
@@ -63,28 +62,41 @@ def test_value_exponent_all_magnitudes(hh):
 
 @pytest.mark.parametrize("k", [0, 1, 2, 4])
 @pytest.mark.parametrize("d", [64, 128])
-def test_plane_datapath_equals_oracle_scores(hh, k, d):
+def test_packed_plane_datapath_equals_oracle_scores(hh, k, d):
+    """Eight queries (two per 32-bit register) against one key through the kernel's word decoders
+    and packed plane accumulators, including the cases that stress the 16-bit halves: every term
+    negative at the largest shift, extreme queries, zero codes with and without a sign bit."""
     rng = np.random.default_rng(100 + k + d)
-    for trial in range(200):
+    out = np.zeros(8, dtype=np.int32)
+    for trial in range(300):
         e = rng.integers(0, 8, d)
         j = rng.integers(0, 1 << k, d)
         sgn = rng.integers(0, 2, d)
+        if trial % 7 == 1:
+            e[:] = 0                                # largest shift everywhere
+        if trial % 7 == 2:
+            sgn[:] = 1
+        if trial % 7 == 3:
+            j[:] = (1 << k) - 1
         codes = ((sgn << 7) | (e << 4) | (j << (4 - k))).astype(np.uint8)
         if trial % 3 == 0:
-            codes[e == 7] = 0x70                    # canonical zeros
-        if trial == 1:
-            codes[:] = 0x80 | (j << (4 - k))        # every term negative with the largest shift
-        q = rng.integers(-127, 128, d).astype(np.int8)
-        if trial == 2:
+            codes[e == 7] = 0x70                    # canonical zeros (otherwise: zero codes keep their sign bit)
+        else:
+            codes[e == 7] &= 0xF0                   # a zero code has no mantissa bits
+        q = rng.integers(-127, 128, (8, d)).astype(np.int8)
+        if trial % 5 == 1:
             q[:] = 127
-        for f_extra in (0, 1):
-            F = 6 + k + f_extra
-            want, ov = ora.scores(q[None, :], codes[None, None, :], k, F)
-            assert ov == 0
-            got = hh.hh_score(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p),
-                              C.c_int(d), C.c_int(f_extra), C.c_int(0))
-            assert got == int(want[0, 0]), (trial, f_extra)
-            if k == 0:
-                got_n = hh.hh_score(C.c_int(0), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p),
-                                    C.c_int(d), C.c_int(f_extra), C.c_int(1))
-                assert got_n == int(want[0, 0])
+        if trial % 5 == 2:
+            q[::2] = -127
+            q[1::2] = 127
+        if trial % 5 == 3:
+            q[:] = -127
+        want, ov = ora.scores(q, codes[None, None, :], k, 6 + k)
+        assert ov == 0
+        hh.hh_score8(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
+                     C.c_int(0), out.ctypes.data_as(C.c_void_p))
+        assert np.array_equal(out.astype(np.int64), want[:, 0]), (trial, out, want[:, 0])
+        if k == 0:
+            hh.hh_score8(C.c_int(0), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
+                         C.c_int(1), out.ctypes.data_as(C.c_void_p))
+            assert np.array_equal(out.astype(np.int64), want[:, 0]), ("nibble", trial)
