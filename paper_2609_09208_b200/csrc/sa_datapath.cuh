@@ -125,17 +125,34 @@ struct PackedPlanes {
 #pragma unroll
         for (int p = 0; p < NP; ++p) tot[p] = hit[p] = 0;
     }
-    // r: shift amount (>= 32 for the zero code); S: 0 or 0xffffffff; mask[b]: 0 or 0xffffffff.
-    // FIRST: the first element of a window starts from the bias instead of the previous sum.
-    template <bool FIRST>
-    SA_HD void element(uint32_t r, uint32_t S, const uint32_t* mask, const uint32_t* qp) {
+    // First element of a window: starts every plane from the bias; the mantissa planes take the
+    // term through a mask.  r: shift amount (>= 32 for the zero code); S: 0 or 0xffffffff;
+    // mask[b]: 0 or 0xffffffff.
+    SA_HD void element_first(uint32_t r, uint32_t S, const uint32_t* mask, const uint32_t* qp) {
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
-            const uint32_t x = shl_clamp_hd(qp[p], r);
-            win[KB][p] = add_fma(x ^ S, FIRST ? 0x8000u : win[KB][p], pw[0]);
+            const uint32_t t = shl_clamp_hd(qp[p], r) ^ S;
+            win[KB][p] = add_fma(t, 0x8000u, pw[0]);
 #pragma unroll
-            for (int b = 0; b < KB; ++b) win[b][p] = add_fma((x ^ S) & mask[b], FIRST ? 0x8000u : win[b][p], pw[0]);
+            for (int b = 0; b < KB; ++b) win[b][p] = add_fma(t & mask[b], 0x8000u, pw[0]);
         }
+    }
+    // Later elements: a mantissa plane receives the term only if its bit is set.  The condition is
+    // the same for all queries, so it costs one predicate per (element, bit) instead of one logic
+    // op per (query pair, element, bit); the adds under it are predicated.
+    SA_HD void element_next(uint32_t r, uint32_t S, const bool* on, const uint32_t* qp) {
+        uint32_t t[NP];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            t[p] = shl_clamp_hd(qp[p], r) ^ S;
+            win[KB][p] = add_fma(t[p], win[KB][p], pw[0]);
+        }
+#pragma unroll
+        for (int b = 0; b < KB; ++b)
+            if (on[b]) {
+#pragma unroll
+                for (int p = 0; p < NP; ++p) win[b][p] = add_fma(t[p], win[b][p], pw[0]);
+            }
     }
     SA_HD void window_end() {
         ++n_windows;
@@ -175,13 +192,19 @@ SA_HD void accumulate_word_bytes(PackedPlanes<KB, NP>& pl, uint32_t w, const uin
         const uint32_t rep = 0x8888u | (0x1111u * i);          // replicate the top bit of byte i
         const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);       // byte i, zero-extended
         const uint32_t S = prmt_hd(w, 0u, rep);
-        uint32_t mask[KB > 0 ? KB : 1];
-#pragma unroll
-        for (int b = 0; b < KB; ++b) mask[b] = prmt_hd(wb[b], 0u, rep);
         uint32_t q[NP];
         load_np<NP>(qp + i * stride, q);
-        if (i == 0) pl.template element<true>(r, S, mask, q);
-        else pl.template element<false>(r, S, mask, q);
+        if (i == 0) {
+            uint32_t mask[KB > 0 ? KB : 1];
+#pragma unroll
+            for (int b = 0; b < KB; ++b) mask[b] = prmt_hd(wb[b], 0u, rep);
+            pl.element_first(r, S, mask, q);
+        } else {
+            bool on[KB > 0 ? KB : 1];
+#pragma unroll
+            for (int b = 0; b < KB; ++b) on[b] = (wb[b] & (0x80u << (8 * i))) != 0u;
+            pl.element_next(r, S, on, q);
+        }
     }
     pl.window_end();
 }
@@ -204,8 +227,8 @@ SA_HD void accumulate_word_nibbles(PackedPlanes<0, NP>& pl, uint32_t w, const ui
             const uint32_t S = prmt_hd((ni & 1) ? w : we, 0u, rep);
             uint32_t q[NP];
             load_np<NP>(qp + ni * stride, q);
-            if (i == 0) pl.template element<true>(r, S, nullptr, q);
-            else pl.template element<false>(r, S, nullptr, q);
+            if (i == 0) pl.element_first(r, S, nullptr, q);
+            else pl.element_next(r, S, nullptr, q);
         }
         pl.window_end();
     }

@@ -12,23 +12,46 @@
 #include "sa_datapath.cuh"
 #include "sa_decode_common.cuh"
 #include "sa_quant.cuh"
+#include "sa_stage.cuh"
 
 namespace sa {
 
+// Shared-memory plan of one block (dynamic shared memory, 128-byte aligned):
+//   [4 warps x kStages stage buffers][mbarriers][packed queries][query scales][weights p (also the
+//   scratch for the unpacked queries during the prologue)]; the block-merge scratch re-uses the stage
+//   buffers once every warp has left its tile loop.
+template <int D, int KB, bool NIB, int GT>
+struct DecodeSmem {
+    static constexpr int NP = (GT + 1) / 2;
+    static constexpr int CH = NIB ? D / 32 : D / 16;
+    using Stage = TileStage<CH, true, D>;
+    static constexpr int kStageOff = 0;
+    static constexpr int kMbarOff = 4 * kStages * Stage::kBytes;
+    static constexpr int kQpOff = kMbarOff + 128;
+    static constexpr int kQscaleOff = kQpOff + D * NP * 4;
+    static constexpr int kPOff = kQscaleOff + 128;
+    static constexpr int kPBytes = (4 * 32 * GT * 8 > D * GT * 4) ? 4 * 32 * GT * 8 : D * GT * 4;
+    static constexpr int kBytes = kPOff + kPBytes;
+    static_assert(4 * GT * (D + 2) * 4 <= 4 * kStages * Stage::kBytes, "merge scratch must fit in the stage buffers");
+};
+
 template <int D, int KB, bool NIB, int GT>
 __global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
+    using SM = DecodeSmem<D, KB, NIB, GT>;
+    using Stage = typename SM::Stage;
     constexpr int EPL = D / 32;
-    constexpr int CH = NIB ? D / 32 : D / 16;      // 16-byte code chunks per key
+    constexpr int NP = SM::NP;
+    constexpr int WORDS = NIB ? D / 8 : D / 4;     // 32-bit code words per key
     constexpr int NJ = 2;                          // output-dim pairs per lane in the A.V phase (4 dims)
     constexpr int LPT = D / (2 * NJ);              // lanes covering one token's value row
     constexpr int TS = 32 / LPT;                   // token groups in the A.V phase
     constexpr int TPL = 32 / TS;                   // tokens per lane per tile
-    constexpr int NP = (GT + 1) / 2;               // packed query registers: two queries each
-    __shared__ int32_t q_s[D][GT];
-    __shared__ __align__(16) uint32_t qp_s[D][NP];
-    __shared__ float qscale_s[GT];
-    __shared__ __align__(16) float2 p_s[4][32][GT];
-    __shared__ __align__(16) float red_s[4][GT][D + 2];
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint32_t (*qp_s)[NP] = reinterpret_cast<uint32_t (*)[NP]>(smem + SM::kQpOff);
+    float* qscale_s = reinterpret_cast<float*>(smem + SM::kQscaleOff);
+    float2 (*p_s)[32][GT] = reinterpret_cast<float2 (*)[32][GT]>(smem + SM::kPOff);
+    int32_t (*q_s)[GT] = reinterpret_cast<int32_t (*)[GT]>(smem + SM::kPOff);      // prologue only
+    float (*red_s)[GT][D + 2] = reinterpret_cast<float (*)[GT][D + 2]>(smem + SM::kStageOff);
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int chunks = a.G / GT;
@@ -36,8 +59,43 @@ __global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;     // first query head of this block
     const int b = blockIdx.z;
     const int split = blockIdx.x;
+    const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
+    const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
+    const uint8_t* stage_ptr0 = smem + SM::kStageOff + warp * kStages * Stage::kBytes;
 
-    // ---- prologue: quantise the GT query heads (eq. (2)) into shared memory ----
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) mbar_init(mbar0 + s * 8, 1u);
+        fence_mbar_init();
+        fence_proxy_async();
+    }
+    __syncwarp();
+
+    // ---- this warp's tiles; start the first copies before the query is quantised ----
+    const int len = a.seq_lens[b];
+    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
+    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
+    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int first = tile0 + warp;
+    const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
+    // Lane 0: start the copies of my i-th tile into stage i % kStages.  A tile whose page is not
+    // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
+    auto issue = [&](int i) {
+        const int tile = first + 4 * i;
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int s = i % kStages;
+        if (pidx < 0 || pidx >= a.n_pages) {
+            mbar_arrive(mbar0 + s * 8);
+        } else {
+            const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
+                         mbar0 + s * 8);
+        }
+    };
+    if (lane == 0)
+        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
+
+    // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register ----
     for (int g = warp; g < GT; g += 4) {
         uint32_t bits[EPL];
         load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
@@ -48,16 +106,20 @@ __global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
         if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < D * NP; idx += 128) {
+    uint32_t qp_reg[(D * NP + 127) / 128];
+#pragma unroll
+    for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+        const int idx = threadIdx.x + k * 128;
         const int m = idx / NP, p = idx % NP;
-        qp_s[m][p] = pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0);
+        qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
+    }
+    __syncthreads();                                           // q_s is about to be re-used as p_s
+#pragma unroll
+    for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+        const int idx = threadIdx.x + k * 128;
+        if (idx < D * NP) qp_s[idx / NP][idx % NP] = qp_reg[k];
     }
     __syncthreads();
-
-    const int len = a.seq_lens[b];
-    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
-    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
 
     int M[GT];
     float l[GT];
@@ -70,90 +132,114 @@ __global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
         for (int j = 0; j < NJ; ++j) acc[g][j] = 0ull;
     }
     const int ts = lane / LPT, dc = lane % LPT;
+    bool failed = false;
 
-    for (int tile = tile0 + warp; tile < tile1; tile += 4) {
-        const int lp = tile >> 1;
-        const int tk0 = (tile & 1) * 32;                     // first token of the tile inside its page
-        const int n_valid = min(32, len - tile * 32);
-        const int pidx = a.page_table[(size_t)b * a.max_pages + lp];
-        if (pidx < 0 || pidx >= a.n_pages) continue;          // unmapped page: skipped, never dereferenced
-        const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+    for (int i = 0; i < n_my; ++i) {
+        const int tile = first + 4 * i;
+        const int s = i % kStages;
+        const uint32_t parity = (uint32_t)(i / kStages) & 1u;
+        // the decision is made warp-uniform: a lane must never leave the loop alone
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(mbar0 + s * 8, parity))) {
+            failed = true;
+            // give the other stage's copy (already issued) a bounded chance to land before this
+            // warp's buffers are re-used by the block merge
+            if (i + 1 < n_my) (void)mbar_wait_bounded(mbar0 + ((i + 1) % kStages) * 8, (uint32_t)((i + 1) / kStages) & 1u);
+            break;
+        }
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const bool mapped = pidx >= 0 && pidx < a.n_pages;     // warp-uniform
+        const uint8_t* st = stage_ptr0 + s * Stage::kBytes;
+        if (mapped) {
+            const int n_valid = min(32, len - tile * 32);
 
-        // ---- phase 1: integer scores, lane = key ----
-        // One 16-byte chunk of codes per iteration; the next chunk is already in flight.  The loop
-        // is deliberately not unrolled over chunks: the body (16 or 32 elements x GT queries) is
-        // what has to stay resident in the instruction cache.
-        const uint4* kptr = reinterpret_cast<const uint4*>(block + a.kcode_off) + tk0 + lane;
-        const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(block + a.meta_off + (size_t)(tk0 + lane) * 4));
-        PackedPlanes<KB, NP> pl;
-        pl.begin(a.one);
-        uint4 cur = __ldg(kptr);
+            // ---- phase 1: integer scores, lane = key; one 32-bit code word (4 or 8 elements) per
+            // iteration, kept rolled so that the loop body stays in the instruction cache ----
+            PackedPlanes<KB, NP> pl;
+            pl.begin(a.one);
+            const uint32_t* cw = reinterpret_cast<const uint32_t*>(st) + lane * 4;
 #pragma unroll 1
-        for (int c = 0; c < CH; ++c) {
-            const uint4 nxt = __ldg(kptr + (size_t)min(c + 1, CH - 1) * kPageTokens);
-            const uint32_t w4[4] = {cur.x, cur.y, cur.z, cur.w};
-#pragma unroll
-            for (int wi = 0; wi < 4; ++wi) {
-                if constexpr (!NIB) accumulate_word_bytes<KB, NP>(pl, w4[wi], &qp_s[c * 16 + wi * 4][0], NP);
-                else accumulate_word_nibbles<NP>(pl, w4[wi], &qp_s[c * 32 + wi * 8][0], NP);
+            for (int wq = 0; wq < WORDS; ++wq) {
+                const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
+                if constexpr (!NIB) accumulate_word_bytes<KB, NP>(pl, w, &qp_s[wq * 4][0], NP);
+                else accumulate_word_nibbles<NP>(pl, w, &qp_s[wq * 8][0], NP);
             }
-            cur = nxt;
-        }
+            const uint32_t meta = reinterpret_cast<const uint32_t*>(st + Stage::kMetaOff)[lane];
 
-        // ---- phase 2: logits, integer running maximum, weights ----
-        const bool valid = lane < n_valid;
-        const float s_j = half_bits_to_float(meta & 0xffffu);
-        const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
-        const float vscale = valid ? pow2i(-g_j) : 0.0f;      // 2^-g_j; g_j in [-10, 30] for written tokens
-        bool changed = false;
-        float resc[GT];
-#pragma unroll
-        for (int g = 0; g < GT; ++g) {
-            const int32_t A = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
-            if (a.dbg_scores && valid)
-                a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A;
-            const float z = valid ? (float)A * qscale_s[g] * s_j : -INFINITY;
-            const float zmax = warp_max_f32(z);
-            const int Mt = (int)ceilf(fminf(fmaxf(zmax, -1.0e8f), 1.0e8f));
-            const int Mn = max(M[g], Mt);
-            resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);   // exact power of two
-            changed |= (Mn != M[g]);
-            M[g] = Mn;
-            const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
-            l[g] = l[g] * resc[g] + p;
-            const float pv = p * vscale;
-            p_s[warp][lane][g] = make_float2(pv, pv);
-        }
-        if (changed) {                                        // warp-uniform
+            // ---- phase 2: logits, integer running maximum, weights ----
+            const bool valid = lane < n_valid;
+            const float s_j = half_bits_to_float(meta & 0xffffu);
+            const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
+            const float vscale = valid ? pow2i(-g_j) : 0.0f;  // 2^-g_j; g_j in [-10, 30] for written tokens
+            bool changed = false;
+            float resc[GT];
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
-                const unsigned long long r2 = pack_f32x2(resc[g], resc[g]);
-#pragma unroll
-                for (int j = 0; j < NJ; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
+                const int32_t A = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
+                if (a.dbg_scores && valid)
+                    a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A;
+                const float z = valid ? (float)A * qscale_s[g] * s_j : -INFINITY;
+                const float zmax = warp_max_f32(z);
+                const int Mt = (int)ceilf(fminf(fmaxf(zmax, -1.0e8f), 1.0e8f));
+                const int Mn = max(M[g], Mt);
+                resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);          // exact power of two
+                changed |= (Mn != M[g]);
+                M[g] = Mn;
+                const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
+                l[g] = l[g] * resc[g] + p;
+                const float pv = p * vscale;
+                p_s[warp][lane][g] = make_float2(pv, pv);
             }
-        }
-        __syncwarp();
+            if (changed) {                                    // warp-uniform
+#pragma unroll
+                for (int g = 0; g < GT; ++g) {
+                    const unsigned long long r2 = pack_f32x2(resc[g], resc[g]);
+#pragma unroll
+                    for (int j = 0; j < NJ; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
+                }
+            }
+            __syncwarp();
 
-        // ---- phase 3: O += p * vhat * 2^-g, lane = (token group, 4 dims) ----
-        const uint8_t* vbase = block + a.v_off + (size_t)tk0 * D + dc * (2 * NJ);
+            // ---- phase 3: O += p * vhat * 2^-g, lane = (token group, 4 dims) ----
+            const uint8_t* vbase = st + Stage::kVOff + dc * (2 * NJ);
 #pragma unroll 4
-        for (int i = 0; i < TPL; ++i) {
-            const int t = ts + TS * i;
-            const uint32_t vv = __ldg(reinterpret_cast<const uint32_t*>(vbase + (size_t)t * D));
-            unsigned long long v2[NJ];
-            v2[0] = pack_f32x2((float)(int8_t)(vv), (float)(int8_t)(vv >> 8));
-            v2[1] = pack_f32x2((float)(int8_t)(vv >> 16), (float)(int8_t)(vv >> 24));
+            for (int k = 0; k < TPL; ++k) {
+                const int t = ts + TS * k;
+                const uint32_t vv = *reinterpret_cast<const uint32_t*>(vbase + t * D);
+                unsigned long long v2[NJ];
+                v2[0] = pack_f32x2((float)(int8_t)(vv), (float)(int8_t)(vv >> 8));
+                v2[1] = pack_f32x2((float)(int8_t)(vv >> 16), (float)(int8_t)(vv >> 24));
+                if constexpr (GT % 2 == 0) {
 #pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&p_s[warp][t][g]);
+                    for (int g = 0; g < GT; g += 2) {         // two queries' duplicated weights per 128-bit load
+                        const ulonglong2 pp = *reinterpret_cast<const ulonglong2*>(&p_s[warp][t][g]);
 #pragma unroll
-                for (int j = 0; j < NJ; ++j) acc[g][j] = ffma2(v2[j], pp, acc[g][j]);
+                        for (int j = 0; j < NJ; ++j) {
+                            acc[g][j] = ffma2(v2[j], pp.x, acc[g][j]);
+                            acc[g + 1][j] = ffma2(v2[j], pp.y, acc[g + 1][j]);
+                        }
+                    }
+                } else {
+                    const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&p_s[warp][t][0]);
+#pragma unroll
+                    for (int j = 0; j < NJ; ++j) acc[0][j] = ffma2(v2[j], pp, acc[0][j]);
+                }
             }
         }
-        __syncwarp();
+        __syncwarp();                                         // every lane is done with this stage and with p_s
+        if (lane == 0 && i + kStages < n_my) {
+            fence_proxy_async();
+            issue(i + kStages);
+        }
+    }
+    if (failed) {
+        // A bounded wait expired: make the failure visible in the output instead of returning a
+        // plausible number (no copy of this warp can still be in flight into a buffer it re-uses).
+#pragma unroll
+        for (int g = 0; g < GT; ++g) l[g] = __int_as_float(0x7fc00000);
     }
 
     // ---- merge the four warps of the block, write the block's partial ----
+    __syncthreads();                                           // the merge scratch re-uses the stage buffers
     block_merge_and_store<D, GT, NJ>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
 }
 
@@ -161,13 +247,25 @@ __global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
 
 using namespace sa;
 
+template <int D, int KB, bool NIB, int GT>
+static void launch_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
+    constexpr int bytes = DecodeSmem<D, KB, NIB, GT>::kBytes;
+    if (bytes > 48 * 1024) {
+        // opt in to more than 48 KB of dynamic shared memory (an attribute of the function; no allocation)
+        static const cudaError_t once = cudaFuncSetAttribute(decode_kernel<D, KB, NIB, GT>,
+                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        (void)once;
+    }
+    decode_kernel<D, KB, NIB, GT><<<grid, 128, bytes, s>>>(a);
+}
+
 template <int D, int KB, bool NIB>
 static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     switch (GT) {
-        case 8: decode_kernel<D, KB, NIB, 8><<<grid, 128, 0, s>>>(a); break;
-        case 4: decode_kernel<D, KB, NIB, 4><<<grid, 128, 0, s>>>(a); break;
-        case 2: decode_kernel<D, KB, NIB, 2><<<grid, 128, 0, s>>>(a); break;
-        default: decode_kernel<D, KB, NIB, 1><<<grid, 128, 0, s>>>(a); break;
+        case 8: launch_one<D, KB, NIB, 8>(a, grid, s); break;
+        case 4: launch_one<D, KB, NIB, 4>(a, grid, s); break;
+        case 2: launch_one<D, KB, NIB, 2>(a, grid, s); break;
+        default: launch_one<D, KB, NIB, 1>(a, grid, s); break;
     }
 }
 

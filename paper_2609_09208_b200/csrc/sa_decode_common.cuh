@@ -41,7 +41,7 @@ SA_D void load_q(const int32_t* src, int32_t (&q)[GT]) {
 // Per-warp states (M, l, O) -> one partial per block.  acc[g][j] holds output dims
 // dc*2*NJ + 2j, dc*2*NJ + 2j + 1 summed over this lane's token group; token groups sit LPT lanes apart.
 template <int D, int GT, int NJ>
-SA_D void block_merge_and_store(const DecodeArgs& a, float (&red_s)[4][GT][D + 2], const int (&M)[GT],
+SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], const int (&M)[GT],
                                 float (&l)[GT], unsigned long long (&acc)[GT][NJ], int lane, int warp,
                                 int ts, int dc, int LPT, int b, int h0, int split) {
 #pragma unroll

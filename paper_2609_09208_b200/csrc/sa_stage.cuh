@@ -1,0 +1,77 @@
+// Shared-memory staging of 32-token tiles with bulk-async (TMA, 1-D) copies and mbarriers.
+//
+// Each warp owns a small ring of stage buffers.  Lane 0 issues, for one tile, one bulk copy per
+// 16-byte code chunk (the page layout keeps chunk c of 32 consecutive tokens in 512 contiguous
+// bytes), one for the metadata and one for the value rows; all of them complete on the stage's
+// mbarrier, which the whole warp then polls.  Every wait is bounded: after kWaitLimit unsuccessful
+// polls the caller poisons its result with NaN and leaves its loop instead of spinning on.
+// Copies are plain (no cluster qualifier): every block stages its own tiles.
+#pragma once
+#include "sa_common.cuh"
+
+namespace sa {
+
+constexpr int kStages = 2;                    // stage buffers per warp
+constexpr uint32_t kWaitLimit = 1u << 18;     // polls of one mbarrier phase before giving up
+
+SA_D uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+SA_D void mbar_init(uint32_t mbar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+SA_D void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+SA_D void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// one arrival that also announces `bytes` of pending copy traffic
+SA_D void mbar_arrive_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+SA_D void mbar_arrive(uint32_t mbar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(mbar) : "memory");
+}
+SA_D bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(mbar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait for a phase; false if it did not complete within kWaitLimit polls.
+SA_D bool mbar_wait_bounded(uint32_t mbar, uint32_t parity) {
+    for (uint32_t it = 0; it < kWaitLimit; ++it)
+        if (mbar_try_wait(mbar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy; size and both addresses are multiples of 16 bytes
+SA_D void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(mbar)
+                 : "memory");
+}
+
+// Layout of one stage buffer: [code chunks: CHUNKS x 512 B][metadata: 128 B or none][values: 32 rows].
+template <int CHUNKS, bool HAS_META, int VROW_BYTES>
+struct TileStage {
+    static constexpr int kCodeBytes = CHUNKS * 512;
+    static constexpr int kMetaOff = kCodeBytes;
+    static constexpr int kMetaBytes = HAS_META ? 128 : 0;
+    static constexpr int kVOff = kCodeBytes + kMetaBytes;
+    static constexpr int kVBytes = 32 * VROW_BYTES;
+    static constexpr int kBytes = kVOff + kVBytes;            // a multiple of 128
+
+    // Issued by one lane.  `block` is the (page, KV head) block, tk0 the tile's first token (0 or 32).
+    SA_D static void issue(uint32_t dst, const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off,
+                           int tk0, uint32_t mbar) {
+        mbar_arrive_expect_tx(mbar, (uint32_t)kBytes);
+#pragma unroll
+        for (int c = 0; c < CHUNKS; ++c)
+            bulk_g2s(dst + c * 512, block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+        if (HAS_META) bulk_g2s(dst + kMetaOff, block + meta_off + (size_t)tk0 * 4, 128u, mbar);
+        bulk_g2s(dst + kVOff, block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes, mbar);
+    }
+};
+
+}  // namespace sa
