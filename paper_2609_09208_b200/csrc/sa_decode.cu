@@ -36,7 +36,7 @@ struct DecodeSmem {
 };
 
 template <int D, int KB, bool NIB, int GT>
-__global__ void __launch_bounds__(128, 4) decode_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeArgs a) {
     using SM = DecodeSmem<D, KB, NIB, GT>;
     using Stage = typename SM::Stage;
     constexpr int EPL = D / 32;

@@ -86,7 +86,7 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
 // One block per (sequence, query head): kMergeGroups groups of D threads each take every
 // kMergeGroups-th split (independent, unrolled loads), then the groups are combined in shared
 // memory and the result is normalised.
-constexpr int kMergeGroups = 4;
+constexpr int kMergeGroups = 8;
 
 template <int D>
 __global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __restrict__ partials,
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __
 #pragma unroll
     for (int w = 0; w < D * kMergeGroups / 32; ++w) Ms = max(Ms, m_s[w]);
     float l = 0.0f, o = 0.0f;
-#pragma unroll 4
+#pragma unroll 8
     for (int s = grp; s < n_splits; s += kMergeGroups) {
         const float* p = base + s * stride;
         const int M = __float_as_int(p[0]);
