@@ -315,13 +315,16 @@ def measured_hbm_peak():
 
 
 def recorded_traffic(variant):
-    """DRAM bytes per main-kernel launch from the committed ncu capture, if one is recorded."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+    """DRAM bytes per main-kernel launch from the committed ncu capture (profiles/dram_traffic.txt)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     try:
-        with open(path) as f:
-            return json.load(f).get(variant)
+        for line in open(path):
+            parts = line.split("#")[0].split()
+            if len(parts) == 2 and parts[0] == variant:
+                return int(parts[1])
     except Exception:
-        return None
+        pass
+    return None
 
 
 def time_steps(fn, n, dev):
@@ -407,7 +410,10 @@ def run_ours(args):
     alg_bytes = wl.algorithmic_bytes_per_main_launch()
     achieved = alg_bytes / (main_us * 1e-6) / 1e9
     peak, peak_kind = measured_hbm_peak()
+    # the capture is of one batch-1, T = 32768 launch; traffic grows with the keys a launch reads
     traffic = recorded_traffic(args.variant)
+    if traffic is not None:
+        traffic = int(traffic * (wl.batch * wl.T) / 32768.0)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_kind": "of %s copy bandwidth" % peak_kind,
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
