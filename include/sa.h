@@ -38,9 +38,8 @@
  *                in the high nibble, nibble = sign << 3 | g.
  *     meta_off : 64 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.
  *     v_off    : vhat, int8, row-major [64][head_dim].
- *   For code = SA_KV_FP16 the block holds unquantised binary16 data: K in 16-byte chunks of 8
- *   elements (chunk c of token t at (c * 64 + t) * 16), no metadata, then V row-major
- *   [64][head_dim].
+ *   For code = SA_KV_FP16 the block holds unquantised binary16 data: K and then V, each in
+ *   16-byte chunks of 8 elements (chunk c of token t at (c * 64 + t) * 16), no metadata.
  */
 #ifndef SA_H_
 #define SA_H_

@@ -38,6 +38,26 @@ SA_D void load_q(const int32_t* src, int32_t (&q)[GT]) {
     }
 }
 
+// red_s[w][g] = {M (int bits), l, O[D]} of warp w -> the block's partial in the workspace.
+template <int D, int GT>
+SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], int b, int h0, int split) {
+    for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 128) {
+        const int g = idx / (D + 1), c = idx % (D + 1);       // c = 0: l, c >= 1: O[c - 1]
+        int Ms = kMNone;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) Ms = max(Ms, __float_as_int(red_s[w][g][0]));
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const int Mw = __float_as_int(red_s[w][g][0]);
+            if (Mw != kMNone) v += red_s[w][g][1 + c] * pow2i_neg(Mw - Ms);
+        }
+        float* dst = a.partials + (((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2);
+        dst[1 + c] = v;
+        if (c == 0) dst[0] = __int_as_float(Ms);
+    }
+}
+
 // Per-warp states (M, l, O) -> one partial per block.  acc[g][j] holds output dims
 // dc*2*NJ + 2j, dc*2*NJ + 2j + 1 summed over this lane's token group; token groups sit LPT lanes apart.
 template <int D, int GT, int NJ>
@@ -66,21 +86,7 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
         }
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 128) {
-        const int g = idx / (D + 1), c = idx % (D + 1);       // c = 0: l, c >= 1: O[c - 1]
-        int Ms = kMNone;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) Ms = max(Ms, __float_as_int(red_s[w][g][0]));
-        float v = 0.0f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            const int Mw = __float_as_int(red_s[w][g][0]);
-            if (Mw != kMNone) v += red_s[w][g][1 + c] * pow2i_neg(Mw - Ms);
-        }
-        float* dst = a.partials + (((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2);
-        dst[1 + c] = v;
-        if (c == 0) dst[0] = __int_as_float(Ms);
-    }
+    block_combine_and_store<D, GT>(a, red_s, b, h0, split);
 }
 
 // One block per (sequence, query head): kMergeGroups groups of D threads each take every

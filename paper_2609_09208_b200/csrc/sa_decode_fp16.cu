@@ -1,161 +1,268 @@
-// Decode attention over an unquantised binary16 cache: softmax(Q K^T / sqrt(d)) V of eq. (1)
-// with FP32 accumulation.  Same grid, tiling, online softmax and merges as the quantised kernel,
-// so that the throughput ratio between the two isolates the key/value representation.
+// Decode attention over an unquantised binary16 cache: softmax(Q K^T / sqrt(d)) V of eq. (1) with
+// FP32 accumulation — the like-for-like baseline of the power-of-two kernels (the paper's three
+// levels of comparison put FP16 attention on tensor cores, section III).
+//
+// Same grid, split and merge as the quantised kernel; each warp streams its own 32-key tiles
+// through a two-stage shared-memory ring filled by bulk-async copies.  Per tile:
+//   S^T = Q K^T   as  mma.m16n8k16: rows = the block's (up to 8) query heads padded to 16,
+//                     k = head dims, n = 8 keys;  Q fragments live in registers for the whole kernel,
+//                     K fragments are 32-bit shared-memory loads from the 16-byte chunk layout;
+//   online softmax with an integer running maximum (the 4 lanes of a row share its 32 keys);
+//   O += P V      as  mma.m16n8k16: the S^T accumulators, converted to binary16, are exactly the
+//                     A fragments of P; V fragments come from ldmatrix.trans on 8 x 8 blocks
+//                     (8 keys x one 16-byte chunk), which the chunk layout stores contiguously.
 #include "sa_common.cuh"
 #include "sa_decode_common.cuh"
 #include "sa_quant.cuh"
+#include "sa_stage.cuh"
 
 namespace sa {
 
+SA_D void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+SA_D void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr)
+                 : "memory");
+}
+SA_D uint32_t pack_half2(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// Stage buffer of one 32-key tile: K chunks [D/8][32 keys][16 B], then V chunks [D/8][32 keys][16 B].
+template <int D>
+struct Fp16Stage {
+    static constexpr int kChunks = D / 8;
+    static constexpr int kVOff = kChunks * 512;
+    static constexpr int kBytes = 2 * kChunks * 512;
+    SA_D static void issue(uint32_t dst, const uint8_t* block, size_t k_off, size_t v_off, int tk0, uint32_t mbar) {
+        mbar_arrive_expect_tx(mbar, (uint32_t)kBytes);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c)
+            bulk_g2s(dst + c * 512, block + k_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c)
+            bulk_g2s(dst + kVOff + c * 512, block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+    }
+};
+
 template <int D, int GT>
-__global__ void __launch_bounds__(128) decode_fp16_kernel(DecodeArgs a) {
-    constexpr int EPL = D / 32;
-    constexpr int CH = D / 8;                      // 16-byte chunks (8 binary16) per key
-    constexpr int LPT = D / 8;
-    constexpr int TS = 32 / LPT;
-    constexpr int TPL = 32 / TS;
-    __shared__ __align__(16) float q_s[D][GT];     // query times log2(e) / sqrt(d)
-    __shared__ __align__(16) float2 p_s[4][32][GT];
-    __shared__ __align__(16) float red_s[4][GT][D + 2];
+struct Fp16Smem {
+    using Stage = Fp16Stage<D>;
+    static constexpr int kStageOff = 0;
+    static constexpr int kMbarOff = 4 * kStages * Stage::kBytes;
+    static constexpr int kBytes = kMbarOff + 128;
+    static_assert(4 * GT * (D + 2) * 4 <= 4 * kStages * Stage::kBytes, "merge scratch must fit in the stage buffers");
+};
+
+template <int D, int GT>
+__global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
+    using SM = Fp16Smem<D, GT>;
+    using Stage = typename SM::Stage;
+    constexpr int KB16 = D / 16;                   // 16-dim blocks of the QK product
+    constexpr int NB8 = D / 8;                     // 8-dim blocks of the output
+    extern __shared__ __align__(128) uint8_t smem[];
+    float (*red_s)[GT][D + 2] = reinterpret_cast<float (*)[GT][D + 2]>(smem + SM::kStageOff);
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int row = lane >> 2, quad = lane & 3;    // fragment row (query) and column pair
     const int chunks = a.G / GT;
     const int kvh = blockIdx.y / chunks;
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;
     const int b = blockIdx.z;
     const int split = blockIdx.x;
+    const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
+    const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
+    const uint8_t* stage_ptr0 = smem + SM::kStageOff + warp * kStages * Stage::kBytes;
 
-    for (int g = warp; g < GT; g += 4) {
-        uint32_t bits[EPL];
-        load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
+    if (lane == 0) {
 #pragma unroll
-        for (int i = 0; i < EPL; ++i) q_s[lane * EPL + i][g] = half_bits_to_float(bits[i]) * a.zscale;
+        for (int s = 0; s < kStages; ++s) mbar_init(mbar0 + s * 8, 1u);
+        fence_mbar_init();
+        fence_proxy_async();
     }
-    __syncthreads();
+    __syncwarp();
 
     const int len = a.seq_lens[b];
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
     const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
     const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int first = tile0 + warp;
+    const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
+    auto issue = [&](int i) {
+        const int tile = first + 4 * i;
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int s = i % kStages;
+        if (pidx < 0 || pidx >= a.n_pages) {
+            mbar_arrive(mbar0 + s * 8);
+        } else {
+            const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.v_off, (tile & 1) * 32, mbar0 + s * 8);
+        }
+    };
+    if (lane == 0)
+        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
 
-    int M[GT];
-    float l[GT];
-    unsigned long long acc[GT][4];
+    // Q fragments (A operand, rows = query heads; rows >= GT are zero): for 16-dim block kb the lane
+    // holds dims 16kb + 2*quad + {0,1} and + 8 of query `row`.
+    uint32_t qa[KB16][2];
 #pragma unroll
-    for (int g = 0; g < GT; ++g) {
-        M[g] = kMNone;
-        l[g] = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[g][j] = 0ull;
+    for (int kb = 0; kb < KB16; ++kb) {
+        qa[kb][0] = qa[kb][1] = 0u;
+        if (row < GT) {
+            const uint32_t* q32 = reinterpret_cast<const uint32_t*>(a.Q + ((size_t)b * a.Hq + h0 + row) * D);
+            qa[kb][0] = __ldg(q32 + kb * 8 + quad);
+            qa[kb][1] = __ldg(q32 + kb * 8 + 4 + quad);
+        }
     }
-    const int ts = lane / LPT, dc = lane % LPT;
 
-    for (int tile = tile0 + warp; tile < tile1; tile += 4) {
-        const int lp = tile >> 1;
-        const int tk0 = (tile & 1) * 32;
-        const int n_valid = min(32, len - tile * 32);
-        const int pidx = a.page_table[(size_t)b * a.max_pages + lp];
-        if (pidx < 0 || pidx >= a.n_pages) continue;
-        const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+    int M = kMNone;                                // running maximum of this lane's query row
+    float l = 0.0f;                                // this lane's share of the row's weight sum
+    float o[NB8][4];
+#pragma unroll
+    for (int nb = 0; nb < NB8; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.0f;
+    bool failed = false;
 
-        // ---- scores, lane = key ----
-        float z[GT];
+    for (int i = 0; i < n_my; ++i) {
+        const int tile = first + 4 * i;
+        const int s = i % kStages;
+        const uint32_t parity = (uint32_t)(i / kStages) & 1u;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(mbar0 + s * 8, parity))) {
+            failed = true;
+            if (i + 1 < n_my) (void)mbar_wait_bounded(mbar0 + ((i + 1) % kStages) * 8, (uint32_t)((i + 1) / kStages) & 1u);
+            break;
+        }
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        if (pidx >= 0 && pidx < a.n_pages) {
+            const int n_valid = min(32, len - tile * 32);
+            const uint8_t* st = stage_ptr0 + s * Stage::kBytes;
+            const uint32_t st_addr = stage0 + s * Stage::kBytes;
+
+            // ---- S^T = Q K^T: four 8-key blocks ----
+            float sc[4][4];
 #pragma unroll
-        for (int g = 0; g < GT; ++g) z[g] = 0.0f;
-#pragma unroll 4
-        for (int c = 0; c < CH; ++c) {
-            const uint4 w = __ldg(reinterpret_cast<const uint4*>(block + a.kcode_off + ((size_t)c * kPageTokens + tk0 + lane) * 16));
-            const uint32_t w4[4] = {w.x, w.y, w.z, w.w};
+            for (int nb = 0; nb < 4; ++nb) {
+                sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.0f;
+                // key nb*8 + row, dims 2*quad + {0,1} of every 16-byte chunk
+                const uint32_t* kw = reinterpret_cast<const uint32_t*>(st) + (nb * 8 + row) * 4 + quad;
 #pragma unroll
-            for (int wi = 0; wi < 4; ++wi) {
-                const float2 kf = __half22float2(*reinterpret_cast<const __half2*>(&w4[wi]));
-                const int m = c * 8 + wi * 2;
-                const float4* q0 = reinterpret_cast<const float4*>(&q_s[m][0]);
-                const float4* q1 = reinterpret_cast<const float4*>(&q_s[m + 1][0]);
-                if constexpr (GT >= 4) {
-#pragma unroll
-                    for (int i = 0; i < GT / 4; ++i) {
-                        const float4 a0 = q0[i], a1 = q1[i];
-                        z[4 * i + 0] = fmaf(a0.x, kf.x, z[4 * i + 0]); z[4 * i + 0] = fmaf(a1.x, kf.y, z[4 * i + 0]);
-                        z[4 * i + 1] = fmaf(a0.y, kf.x, z[4 * i + 1]); z[4 * i + 1] = fmaf(a1.y, kf.y, z[4 * i + 1]);
-                        z[4 * i + 2] = fmaf(a0.z, kf.x, z[4 * i + 2]); z[4 * i + 2] = fmaf(a1.z, kf.y, z[4 * i + 2]);
-                        z[4 * i + 3] = fmaf(a0.w, kf.x, z[4 * i + 3]); z[4 * i + 3] = fmaf(a1.w, kf.y, z[4 * i + 3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int g = 0; g < GT; ++g) {
-                        z[g] = fmaf(q_s[m][g], kf.x, z[g]);
-                        z[g] = fmaf(q_s[m + 1][g], kf.y, z[g]);
-                    }
+                for (int kb = 0; kb < KB16; ++kb) {
+                    const uint32_t b0 = kw[(2 * kb) * 128];          // chunk 2kb: dims 16kb + 2*quad + {0,1}
+                    const uint32_t b1 = kw[(2 * kb + 1) * 128];      // chunk 2kb+1: dims 16kb + 8 + ...
+                    mma_f16_16816(sc[nb], qa[kb][0], 0u, qa[kb][1], 0u, b0, b1);
                 }
             }
-        }
 
-        // ---- online softmax with an integer running maximum ----
-        const bool valid = lane < n_valid;
-        bool changed = false;
-        float resc[GT];
+            // ---- online softmax, integer running maximum; this lane: row `row`, keys nb*8 + 2*quad + {0,1} ----
+            float zmax = -INFINITY;
 #pragma unroll
-        for (int g = 0; g < GT; ++g) {
-            const float zz = valid ? z[g] : -INFINITY;
-            const float zmax = warp_max_f32(zz);
+            for (int nb = 0; nb < 4; ++nb) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = nb * 8 + 2 * quad + e;
+                    sc[nb][e] = (key < n_valid) ? sc[nb][e] * a.zscale : -INFINITY;
+                    zmax = fmaxf(zmax, sc[nb][e]);
+                }
+            }
+            zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, 1));
+            zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, 2));
             const int Mt = (int)ceilf(fminf(fmaxf(zmax, -1.0e8f), 1.0e8f));
-            const int Mn = max(M[g], Mt);
-            resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);
-            changed |= (Mn != M[g]);
-            M[g] = Mn;
-            const float p = valid ? ex2_approx(zz - (float)Mn) : 0.0f;
-            l[g] = l[g] * resc[g] + p;
-            p_s[warp][lane][g] = make_float2(p, p);
-        }
-        if (changed) {
+            const int Mn = max(M, Mt);
+            const float resc = (M == kMNone) ? 0.0f : pow2i_neg(M - Mn);
+            if (Mn != M) {
 #pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const unsigned long long r2 = pack_f32x2(resc[g], resc[g]);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
+                for (int nb = 0; nb < NB8; ++nb) { o[nb][0] *= resc; o[nb][1] *= resc; }
             }
-        }
-        __syncwarp();
+            M = Mn;
+            l *= resc;
+            uint32_t pa[4];                                          // P as A fragments, one per 8-key block
+#pragma unroll
+            for (int nb = 0; nb < 4; ++nb) {
+                const float p0 = ex2_approx(sc[nb][0] - (float)Mn);  // exp2(-inf) = 0 for masked keys
+                const float p1 = ex2_approx(sc[nb][1] - (float)Mn);
+                // the weights enter the product rounded to binary16; the normaliser sums the same rounded
+                // values, so that the result stays an exact weighted mean of the value rows
+                const __half2 ph = __floats2half2_rn(p0, p1);
+                const float2 pr = __half22float2(ph);
+                l += pr.x + pr.y;
+                pa[nb] = *reinterpret_cast<const uint32_t*>(&ph);
+            }
 
-        // ---- O += p * V, lane = (token group, 8 dims) ----
-        const uint8_t* vbase = block + a.v_off + ((size_t)tk0 * D + dc * 8) * 2;
-#pragma unroll 4
-        for (int i = 0; i < TPL; ++i) {
-            const int t = ts + TS * i;
-            uint4 vv = __ldg(reinterpret_cast<const uint4*>(vbase + (size_t)t * D * 2));
-            if (t >= n_valid) vv = make_uint4(0u, 0u, 0u, 0u);   // unwritten slots may hold non-finite bit patterns
-            const uint32_t v4[4] = {vv.x, vv.y, vv.z, vv.w};
-            unsigned long long v2[4];
+            // ---- O += P V: two 16-key blocks x D/8 output blocks ----
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&v4[j]));
-                v2[j] = pack_f32x2(f.x, f.y);
-            }
+            for (int nb = 0; nb < NB8; ++nb) {
+                uint32_t vb[4];                                      // V^T fragments of chunk nb: keys 0-7, 8-15, 16-23, 24-31
+                ldmatrix_x4_trans(vb, st_addr + Stage::kVOff + (nb * 32 + lane) * 16);
+                if (n_valid < 32) {
+                    // slots past the sequence end may hold anything (even NaN patterns): their weight is
+                    // zero, but 0 * NaN is not, so the value halves of those keys are cleared
 #pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&p_s[warp][t][g]);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[g][j] = ffma2(v2[j], pp, acc[g][j]);
+                    for (int j = 0; j < 4; ++j) {
+                        const int key = j * 8 + 2 * quad;
+                        if (key >= n_valid) vb[j] = 0u;
+                        else if (key + 1 >= n_valid) vb[j] &= 0x0000ffffu;
+                    }
+                }
+                mma_f16_16816(o[nb], pa[0], 0u, pa[1], 0u, vb[0], vb[1]);
+                mma_f16_16816(o[nb], pa[2], 0u, pa[3], 0u, vb[2], vb[3]);
             }
         }
         __syncwarp();
+        if (lane == 0 && i + kStages < n_my) {
+            fence_proxy_async();
+            issue(i + kStages);
+        }
     }
+    if (failed) l = __int_as_float(0x7fc00000);    // a bounded wait expired: make it visible in the output
 
-    block_merge_and_store<D, GT, 4>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
+    // ---- per-warp state -> shared memory, merge the four warps, write the block's partial ----
+    __syncthreads();                               // the merge scratch re-uses the stage buffers
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (row < GT) {
+#pragma unroll
+        for (int nb = 0; nb < NB8; ++nb) {
+            red_s[warp][row][2 + nb * 8 + 2 * quad] = o[nb][0];
+            red_s[warp][row][2 + nb * 8 + 2 * quad + 1] = o[nb][1];
+        }
+        if (quad == 0) {
+            red_s[warp][row][0] = __int_as_float(M);
+            red_s[warp][row][1] = l;
+        }
+    }
+    __syncthreads();
+    block_combine_and_store<D, GT>(a, red_s, b, h0, split);
 }
 
 }  // namespace sa
 
 using namespace sa;
 
+template <int D, int GT>
+static void launch_fp16_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
+    constexpr int bytes = Fp16Smem<D, GT>::kBytes;
+    if (bytes > 48 * 1024) {
+        // opt in to more than 48 KB of dynamic shared memory (an attribute of the function; no allocation)
+        static const cudaError_t once = cudaFuncSetAttribute(decode_fp16_kernel<D, GT>,
+                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        (void)once;
+    }
+    decode_fp16_kernel<D, GT><<<grid, 128, bytes, s>>>(a);
+}
+
 template <int D>
 static void launch_fp16(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     switch (GT) {
-        case 8: decode_fp16_kernel<D, 8><<<grid, 128, 0, s>>>(a); break;
-        case 4: decode_fp16_kernel<D, 4><<<grid, 128, 0, s>>>(a); break;
-        case 2: decode_fp16_kernel<D, 2><<<grid, 128, 0, s>>>(a); break;
-        default: decode_fp16_kernel<D, 1><<<grid, 128, 0, s>>>(a); break;
+        case 8: launch_fp16_one<D, 8>(a, grid, s); break;
+        case 4: launch_fp16_one<D, 4>(a, grid, s); break;
+        case 2: launch_fp16_one<D, 2>(a, grid, s); break;
+        default: launch_fp16_one<D, 1>(a, grid, s); break;
     }
 }
 

@@ -115,9 +115,10 @@ SA_D void write_token_fp16(uint8_t* block, const CacheArgs& a, int t, int lane, 
     uint32_t kb[EPL], vb[EPL];
     load_vec_bits<EPL>(krow, lane, kb);
     load_vec_bits<EPL>(vrow, lane, vb);
-    const int m = lane * EPL;                        // chunk of 8 elements = 16 bytes
-    uint16_t* kdst = reinterpret_cast<uint16_t*>(block + a.kcode_off + ((size_t)(m >> 3) * kPageTokens + t) * 16) + (m & 7);
-    uint16_t* vdst = reinterpret_cast<uint16_t*>(block + a.v_off) + (size_t)t * D + m;
+    const int m = lane * EPL;                        // K and V both in 16-byte chunks of 8 elements
+    const size_t off = ((size_t)(m >> 3) * kPageTokens + t) * 16 + (size_t)(m & 7) * 2;
+    uint16_t* kdst = reinterpret_cast<uint16_t*>(block + a.kcode_off + off);
+    uint16_t* vdst = reinterpret_cast<uint16_t*>(block + a.v_off + off);
 #pragma unroll
     for (int i = 0; i < EPL; ++i) {
         kdst[i] = (uint16_t)kb[i];
