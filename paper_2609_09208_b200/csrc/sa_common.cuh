@@ -107,6 +107,12 @@ SA_D uint32_t shl_clamp(uint32_t x, uint32_t n) {
     return r;
 }
 
+// Programmatic dependent launch: a kernel launched with the attribute may start while its
+// predecessor in the stream is still draining; it must call pdl_wait() before it touches anything the
+// predecessor wrote.  Both are no-ops in a kernel launched the ordinary way.
+SA_D void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+SA_D void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 SA_D uint32_t warp_max_u32(uint32_t v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -182,5 +188,23 @@ SA_D float pow2i_neg(int e) { return e < -126 ? 0.0f : __int_as_float((e + 127) 
 
 SA_D float half_bits_to_float(uint32_t b) { return __half2float(__ushort_as_half((unsigned short)b)); }
 #endif  // __CUDACC__
+
+#ifdef __CUDACC__
+// Launch with programmatic stream serialisation allowed (see pdl_wait above).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+#endif
 
 }  // namespace sa

@@ -70,6 +70,8 @@ __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeAr
         fence_proxy_async();
     }
     __syncwarp();
+    pdl_wait();                 // everything below reads what earlier kernels in the stream wrote
+    pdl_launch_dependents();    // the split-K merge may be scheduled as soon as blocks of this grid retire
 
     // ---- this warp's tiles; start the first copies before the query is quantised ----
     const int len = a.seq_lens[b];
@@ -256,7 +258,7 @@ static void launch_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         (void)once;
     }
-    decode_kernel<D, KB, NIB, GT><<<grid, 128, bytes, s>>>(a);
+    (void)launch_pdl(decode_kernel<D, KB, NIB, GT>, grid, dim3(128), (size_t)bytes, s, a);
 }
 
 template <int D, int KB, bool NIB>

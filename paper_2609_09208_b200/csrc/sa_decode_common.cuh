@@ -99,6 +99,8 @@ __global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __
                                                                  float* __restrict__ O, int n_splits, int n_rows) {
     __shared__ int m_s[D * kMergeGroups / 32];
     __shared__ float o_s[kMergeGroups][D + 1];
+    pdl_wait();                                               // the partials come from the kernel before
+    pdl_launch_dependents();
     const int row = blockIdx.x;                               // b * Hq + h
     const int dd = threadIdx.x % D, grp = threadIdx.x / D;
     const size_t stride = (size_t)n_rows * (D + 2);
@@ -176,9 +178,12 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
 
 inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s) {
     const int rows = a.batch * a.Hq;
-    if (p.d == 64) merge_kernel<64><<<rows, 64 * kMergeGroups, 0, s>>>(a.partials, a.O, a.n_splits, rows);
-    else merge_kernel<128><<<rows, 128 * kMergeGroups, 0, s>>>(a.partials, a.O, a.n_splits, rows);
-    return cudaGetLastError() == cudaSuccess ? SA_OK : SA_ERR_CUDA;
+    cudaError_t err;
+    if (p.d == 64) err = launch_pdl(merge_kernel<64>, dim3(rows), dim3(64 * kMergeGroups), 0, s,
+                                    (const float*)a.partials, a.O, a.n_splits, rows);
+    else err = launch_pdl(merge_kernel<128>, dim3(rows), dim3(128 * kMergeGroups), 0, s,
+                          (const float*)a.partials, a.O, a.n_splits, rows);
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SA_OK : SA_ERR_CUDA;
 }
 
 }  // namespace sa

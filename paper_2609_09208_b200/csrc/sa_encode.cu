@@ -147,6 +147,8 @@ SA_D void write_token(uint8_t* block, const CacheArgs& a, int t, int lane, const
 template <int D, int MODE>
 __global__ void __launch_bounds__(128) append_kernel(CacheArgs a, const uint16_t* __restrict__ Knew,
                                                      const uint16_t* __restrict__ Vnew, int bump) {
+    pdl_wait();                 // earlier kernels in the stream may still be reading this cache
+    pdl_launch_dependents();
     const int b = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int len = a.seq_lens[b];
@@ -347,7 +349,7 @@ sa_status sa_append_kv(const sa_config* cfg, const sa_cache* cache, const uint16
     if (!K_new || !V_new) return SA_ERR_INVALID_ARG;
     if (!aligned(K_new, 16) || !aligned(V_new, 16)) return SA_ERR_ALIGNMENT;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-#define CALL(D, M) append_kernel<D, M><<<a.batch, 128, 0, s>>>(a, K_new, V_new, bump_lens)
+#define CALL(D, M) (void)launch_pdl(append_kernel<D, M>, dim3(a.batch), dim3(128), 0, s, a, K_new, V_new, bump_lens)
     SA_DISPATCH_D_MODE(p, CALL);
 #undef CALL
     return SA_LAUNCH_CHECK();
