@@ -22,22 +22,6 @@ struct DecodeArgs {
     uint32_t one;             // the value 1, opaque to the compiler (adds issued as multiply-add)
 };
 
-template <int GT>
-SA_D void load_q(const int32_t* src, int32_t (&q)[GT]) {
-    if constexpr (GT >= 4) {
-#pragma unroll
-        for (int i = 0; i < GT / 4; ++i) {
-            const int4 v = reinterpret_cast<const int4*>(src)[i];
-            q[4 * i] = v.x; q[4 * i + 1] = v.y; q[4 * i + 2] = v.z; q[4 * i + 3] = v.w;
-        }
-    } else if constexpr (GT == 2) {
-        const int2 v = *reinterpret_cast<const int2*>(src);
-        q[0] = v.x; q[1] = v.y;
-    } else {
-        q[0] = src[0];
-    }
-}
-
 // red_s[w][g] = {M (int bits), l, O[D]} of warp w -> the block's partial in the workspace.
 template <int D, int GT>
 SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], int b, int h0, int split) {
