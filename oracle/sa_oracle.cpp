@@ -301,9 +301,9 @@ int64_t ora_scores(const int8_t* qhat, const uint8_t* codes, int64_t T, int Hq, 
 // A [Hq, T]; delta [Hq]; scales [T, Hkv] binary16 bits; vhat [T, Hkv, d]; g [T, Hkv];
 // O [Hq, d].
 // ---------------------------------------------------------------------------------
-void ora_attention_twopass(const int64_t* A, const float* delta, const uint16_t* scales,
-                           const int8_t* vhat, const int8_t* g, int64_t T, int Hq, int Hkv,
-                           int d, int F, double* O) {
+static void twopass_core(const int64_t* A, const float* delta, const uint16_t* scales,
+                         const int8_t* vhat, const int8_t* g, int64_t T, int Hq, int Hkv,
+                         int d, double unit, double* O) {
     const int G = Hq / Hkv;
     const double log2e = 1.4426950408889634074;
     std::vector<double> z(static_cast<size_t>(T));
@@ -312,7 +312,7 @@ void ora_attention_twopass(const int64_t* A, const float* delta, const uint16_t*
         double* out = O + static_cast<int64_t>(h) * d;
         for (int m = 0; m < d; ++m) out[m] = 0.0;
         if (T == 0) continue;
-        const double qf = static_cast<double>(delta[h]) * std::ldexp(1.0, -F) * log2e /
+        const double qf = static_cast<double>(delta[h]) * unit * log2e /
                           std::sqrt(static_cast<double>(d));
         double zmax = -std::numeric_limits<double>::infinity();
         for (int64_t t = 0; t < T; ++t) {
@@ -330,6 +330,64 @@ void ora_attention_twopass(const int64_t* A, const float* delta, const uint16_t*
         }
         for (int m = 0; m < d; ++m) out[m] /= wsum;
     }
+}
+
+void ora_attention_twopass(const int64_t* A, const float* delta, const uint16_t* scales,
+                           const int8_t* vhat, const int8_t* g, int64_t T, int Hq, int Hkv,
+                           int d, int F, double* O) {
+    twopass_core(A, delta, scales, vhat, g, T, Hq, Hkv, d, std::ldexp(1.0, -F), O);
+}
+
+// ---------------------------------------------------------------------------------
+// Uniform INT8 key code: the comparison datapath of section III and section VI (an INT8
+// multiply-accumulate kernel "built on the same tiling"; Table II lists the uniform INT8
+// quantiser as an accuracy baseline).  Per key vector: scale = largest magnitude (binary16),
+// khat = clamp(round-half-even(K * 127 / amax), -127, 127), decided in binary32 exactly like
+// the query quantiser; K ~ (scale / 127) * khat.  Scores are plain integer dot products
+// A_ij = sum_m qhat_im * khat_jm; logits z = A * Delta * (scale / 127) * log2(e) / sqrt(d).
+// ---------------------------------------------------------------------------------
+void ora_encode_keys_int8(const uint16_t* K, int64_t n_vec, int d, int8_t* codes, uint16_t* scales) {
+    for (int64_t v = 0; v < n_vec; ++v) {
+        const uint16_t* row = K + v * d;
+        uint16_t smax_bits = 0;
+        for (int m = 0; m < d; ++m) {
+            const uint16_t mag = row[m] & 0x7fff;
+            if (mag > smax_bits) smax_bits = mag;
+        }
+        scales[v] = smax_bits;
+        const float amax = static_cast<float>(half_bits_to_double(smax_bits));
+        if (amax == 0.0f) {
+            for (int m = 0; m < d; ++m) codes[v * d + m] = 0;
+            continue;
+        }
+        const float inv = 127.0f / amax;
+        for (int m = 0; m < d; ++m) {
+            const float x = static_cast<float>(half_bits_to_double(row[m]));
+            float r = std::nearbyintf(x * inv);
+            if (r > 127.0f) r = 127.0f;
+            if (r < -127.0f) r = -127.0f;
+            codes[v * d + m] = static_cast<int8_t>(r);
+        }
+    }
+}
+
+void ora_scores_int8(const int8_t* qhat, const int8_t* codes, int64_t T, int Hq, int Hkv, int d, int64_t* A) {
+    const int G = Hq / Hkv;
+    for (int h = 0; h < Hq; ++h) {
+        const int kv = h / G;
+        for (int64_t t = 0; t < T; ++t) {
+            const int8_t* c = codes + (t * Hkv + kv) * d;
+            int64_t acc = 0;
+            for (int m = 0; m < d; ++m) acc += static_cast<int64_t>(qhat[h * d + m]) * static_cast<int64_t>(c[m]);
+            A[static_cast<int64_t>(h) * T + t] = acc;
+        }
+    }
+}
+
+void ora_attention_twopass_int8(const int64_t* A, const float* delta, const uint16_t* scales,
+                                const int8_t* vhat, const int8_t* g, int64_t T, int Hq, int Hkv,
+                                int d, double* O) {
+    twopass_core(A, delta, scales, vhat, g, T, Hq, Hkv, d, 1.0 / 127.0, O);
 }
 
 // ---------------------------------------------------------------------------------
@@ -433,7 +491,8 @@ void ora_sdpa_fp16(const uint16_t* Q, const uint16_t* K, const uint16_t* V, int6
 // ---------------------------------------------------------------------------------
 // The whole decode step for a ragged batch, chaining the functions above in the
 // paper's order: [optional rotation of Q and K] -> query quantise -> key encode ->
-// value quantise -> integer scores -> two-pass softmax and A.V.
+// value quantise -> integer scores -> two-pass softmax and A.V.  k = 8 selects the uniform INT8
+// comparison code (F is then ignored).
 // Q [B, Hq, d]; K, V [sum_b T_b, Hkv, d] with sequence b occupying rows
 // cu_lens[b] .. cu_lens[b+1]; O [B, Hq, d] fp64; A_dbg (nullable) [B, Hq, max_T]
 // receives the integer scores (row stride max_T).  The independent units
@@ -480,15 +539,18 @@ int64_t ora_decode_attention(const uint16_t* Q, const uint16_t* K, const uint16_
             double c1 = now();
             std::vector<uint8_t> codes(static_cast<size_t>(T) * d);
             std::vector<uint16_t> scales(static_cast<size_t>(T));
-            ora_encode_keys(kk.data(), T, d, k, codes.data(), scales.data());
+            if (k == 8) ora_encode_keys_int8(kk.data(), T, d, reinterpret_cast<int8_t*>(codes.data()), scales.data());
+            else ora_encode_keys(kk.data(), T, d, k, codes.data(), scales.data());
             std::vector<int8_t> vhat(static_cast<size_t>(T) * d), g(static_cast<size_t>(T));
             ora_quantise_value(vv.data(), T, d, vhat.data(), g.data());
             double c2 = now();
             std::vector<int64_t> A(static_cast<size_t>(G) * T);
-            overflow[tid] += ora_scores(qhat.data(), codes.data(), T, G, 1, d, k, F, A.data());
+            if (k == 8) ora_scores_int8(qhat.data(), reinterpret_cast<const int8_t*>(codes.data()), T, G, 1, d, A.data());
+            else overflow[tid] += ora_scores(qhat.data(), codes.data(), T, G, 1, d, k, F, A.data());
             double c3 = now();
-            ora_attention_twopass(A.data(), delta.data(), scales.data(), vhat.data(), g.data(), T,
-                                  G, 1, d, F, O + (static_cast<int64_t>(b) * Hq + kv * G) * d);
+            double* Oh = O + (static_cast<int64_t>(b) * Hq + kv * G) * d;
+            if (k == 8) ora_attention_twopass_int8(A.data(), delta.data(), scales.data(), vhat.data(), g.data(), T, G, 1, d, Oh);
+            else ora_attention_twopass(A.data(), delta.data(), scales.data(), vhat.data(), g.data(), T, G, 1, d, F, Oh);
             double c4 = now();
             if (A_dbg)
                 for (int h = 0; h < G; ++h)

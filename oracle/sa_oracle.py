@@ -190,5 +190,40 @@ def decode_attention(Q, K, V, cu_lens, k: int, F: int, hadamard: bool = False,
     return dict(O=O, A=A, overflow=int(ov), stage_seconds=st)
 
 
+def encode_keys_int8(K):
+    """Uniform INT8 comparison code: K [..., d] float16 -> (codes int8 [..., d], scales float16 [...])."""
+    kb = _half_bits(K)
+    d = kb.shape[-1]
+    codes = np.empty(kb.shape, dtype=np.int8)
+    scales = np.empty(kb.shape[:-1], dtype=np.uint16)
+    lib().ora_encode_keys_int8(_p(kb), C.c_int64(kb.size // d), C.c_int(d), _p(codes), _p(scales))
+    return codes, scales.view(np.float16)
+
+
+def scores_int8(qhat, codes):
+    """qhat int8 [Hq, d]; codes int8 [T, Hkv, d] -> A int64 [Hq, T]."""
+    qhat = np.ascontiguousarray(qhat, dtype=np.int8)
+    codes = np.ascontiguousarray(codes, dtype=np.int8)
+    Hq, d = qhat.shape
+    T, Hkv, _ = codes.shape
+    A = np.empty((Hq, T), dtype=np.int64)
+    lib().ora_scores_int8(_p(qhat), _p(codes), C.c_int64(T), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _p(A))
+    return A
+
+
+def attention_twopass_int8(A, delta, scales, vhat, g):
+    A = np.ascontiguousarray(A, dtype=np.int64)
+    delta = np.ascontiguousarray(delta, dtype=np.float32)
+    sb = _half_bits(scales)
+    vhat = np.ascontiguousarray(vhat, dtype=np.int8)
+    g = np.ascontiguousarray(g, dtype=np.int8)
+    Hq, T = A.shape
+    _, Hkv, d = vhat.shape
+    O = np.empty((Hq, d), dtype=np.float64)
+    lib().ora_attention_twopass_int8(_p(A), _p(delta), _p(sb), _p(vhat), _p(g), C.c_int64(T), C.c_int(Hq),
+                                     C.c_int(Hkv), C.c_int(d), _p(O))
+    return O
+
+
 def hardware_threads() -> int:
     return int(lib().ora_hardware_threads())

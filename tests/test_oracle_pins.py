@@ -531,3 +531,49 @@ def test_quantised_attention_approaches_fp16_attention():
         O = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, k, E + k)["O"][0]
         err[k] = np.max(np.abs(O - ref))
     assert err[4] < err[1] < err[0] and err[4] < 0.03
+
+
+# ------------------------------------------------------------------ uniform INT8 comparison code
+def test_int8_key_code_hand_example_and_error_bound():
+    K = np.zeros((2, 64), dtype=np.float16)
+    K[0, :6] = [2.0, -1.0, 0.5, 1.0, -2.0, 0.015625]
+    codes, scales = ora.encode_keys_int8(K)
+    assert codes[0, :6].tolist() == [127, -64, 32, 64, -127, 1]      # 63.5 -> 64 and 31.75 -> 32: ties to even / nearest
+    assert float(scales[0]) == 2.0 and not codes[1].any() and float(scales[1]) == 0.0
+    rng = np.random.default_rng(90)
+    K = (rng.standard_normal((300, 64)) * np.exp(rng.standard_normal((1, 64)))).astype(np.float16)
+    codes, scales = ora.encode_keys_int8(K)
+    step = scales.astype(np.float64) / 127.0
+    assert np.all(np.abs(codes).max(axis=1) == 127)
+    assert np.all(np.abs(K.astype(np.float64) - step[:, None] * codes) <= 0.5 * step[:, None] * (1 + 1e-5))
+
+
+def test_int8_scores_are_integer_dot_products_and_softmax_matches_library():
+    from scipy.special import softmax
+    rng = np.random.default_rng(91)
+    Hq, Hkv, d, T = 8, 2, 64, 200
+    K = rng.standard_normal((T, Hkv, d)).astype(np.float16)
+    V = rng.standard_normal((T, Hkv, d)).astype(np.float16)
+    Q = rng.standard_normal((Hq, d)).astype(np.float16)
+    codes, scales = ora.encode_keys_int8(K)
+    qhat, delta = ora.quantise_query(Q)
+    vhat, g = ora.quantise_value(V)
+    A = ora.scores_int8(qhat, codes)
+    for h in range(Hq):
+        kv = h // 4
+        want = codes[:, kv].astype(np.int64) @ qhat[h].astype(np.int64)          # numpy integer matmul
+        assert np.array_equal(A[h], want)
+    O = ora.attention_twopass_int8(A, delta, scales, vhat, g)
+    for h in range(Hq):
+        kv = h // 4
+        logits = A[h] * float(delta[h]) * scales[:, kv].astype(np.float64) / 127.0 / math.sqrt(d)
+        w = softmax(logits)
+        want = w @ (vhat[:, kv].astype(np.float64) * 2.0 ** (-g[:, kv, None].astype(np.float64)))
+        assert np.max(np.abs(O[h] - want)) < 1e-12
+    # whole step with k = 8, and its accuracy next to the 8-bit power-of-two code (the paper: within ~2x)
+    case = synth.make_case("t", [400], 8, 2, 64, 4, seed=92)
+    ref = ora.sdpa_fp16(case.Q[0], case.K, case.V)
+    o8 = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, 8, 0)["O"][0]
+    o4 = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, 4, 10)["O"][0]
+    e8, e4 = np.max(np.abs(o8 - ref)), np.max(np.abs(o4 - ref))
+    assert e8 < 0.02 and e8 < e4 < 6 * e8
