@@ -51,6 +51,7 @@ VARIANTS = {
     "pot4_nibble": (0, True, False, False),
     "pot4_nibble_had": (0, True, True, False),
     "fp16": (0, False, False, True),
+    "int8mac": (8, False, False, False),      # uniform INT8 keys, dp4a scores: the paper's multiply-native comparison
 }
 
 

@@ -63,7 +63,12 @@ typedef enum {
 } sa_status;
 
 /* Key code family: the value is k, the number of mantissa bits (eq. (2), eq. (5)). */
-enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_KV_FP16 = 16 };
+enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_INT8 = 8, SA_KV_FP16 = 16 };
+/* SA_INT8 is the comparison code of section III / VI (an INT8 multiply-accumulate kernel "of
+ * identical structure"): uniform INT8 keys, khat = round(K * 127 / amax) with the row maximum as
+ * scale, stored one byte per element in the byte container (132 bytes per key at d = 64, the same
+ * as PoT-M4); scores are integer dot products evaluated with dp4a.  Everything else (query and
+ * value quantisers, softmax, A.V, merge, cache layout) is shared with the power-of-two codes. */
 /* How key codes are stored in a page. */
 enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1 };
 /* flags */
@@ -73,7 +78,7 @@ typedef struct {
     int head_dim;    /* 64 or 128 */
     int n_q_heads;   /* multiple of n_kv_heads */
     int n_kv_heads;
-    int code;        /* SA_POT4 / SA_POTM1 / SA_POTM2 / SA_POTM4, or SA_KV_FP16 for the FP16 baseline cache */
+    int code;        /* SA_POT4 / SA_POTM1 / SA_POTM2 / SA_POTM4, SA_INT8 (comparison), or SA_KV_FP16 (FP16 baseline cache) */
     int klayout;     /* SA_KLAYOUT_BYTE, or SA_KLAYOUT_NIBBLE (only with SA_POT4) */
     int headroom_F;  /* fixed-point head-room F of eq. (3); 0 selects the default E + k = 6 + k.
                         Must satisfy F >= 6 + k (eq. (4): every shift is a left shift) and

@@ -13,7 +13,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsa.so")
 
-SA_POT4, SA_POTM1, SA_POTM2, SA_POTM4, SA_KV_FP16 = 0, 1, 2, 4, 16
+SA_POT4, SA_POTM1, SA_POTM2, SA_POTM4, SA_INT8, SA_KV_FP16 = 0, 1, 2, 4, 8, 16
 SA_KLAYOUT_BYTE, SA_KLAYOUT_NIBBLE = 0, 1
 SA_FLAG_HADAMARD = 1
 PAGE_TOKENS = 64

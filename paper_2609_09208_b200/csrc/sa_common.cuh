@@ -23,7 +23,7 @@ constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no k
 // ---------------------------------------------------------------------------------------------
 struct Plan {
     int d, Hq, Hkv, G, k;     // k = mantissa bits (0 for SA_KV_FP16)
-    bool fp16, nibble, hadamard;
+    bool fp16, nibble, hadamard, int8;   // int8: the uniform INT8 comparison code
     int F;                    // head-room actually used
     int f_extra;              // F - (6 + k): applied as one final left shift of the INT32 sum
     sa_layout lay;

@@ -74,10 +74,14 @@ SA_HD uint32_t add_fma(uint32_t a, uint32_t b, uint32_t one) {
 #endif
 }
 
-// NP consecutive 32-bit words (NP = 1, 2 or 4; 4 * NP-byte aligned) with one vector load.
+// NP consecutive 32-bit words (NP = 1, 2, 4 or 8; min(16, 4 * NP)-byte aligned) with vector loads.
 template <int NP>
 SA_HD void load_np(const uint32_t* src, uint32_t (&q)[NP]) {
-    if constexpr (NP == 4) {
+    if constexpr (NP == 8) {
+        const uint4 v0 = reinterpret_cast<const uint4*>(src)[0], v1 = reinterpret_cast<const uint4*>(src)[1];
+        q[0] = v0.x; q[1] = v0.y; q[2] = v0.z; q[3] = v0.w;
+        q[4] = v1.x; q[5] = v1.y; q[6] = v1.z; q[7] = v1.w;
+    } else if constexpr (NP == 4) {
         const uint4 v = *reinterpret_cast<const uint4*>(src);
         q[0] = v.x; q[1] = v.y; q[2] = v.z; q[3] = v.w;
     } else if constexpr (NP == 2) {

@@ -22,7 +22,7 @@ namespace sa {
 //   buffers once every warp has left its tile loop.
 template <int D, int KB, bool NIB, int GT>
 struct DecodeSmem {
-    static constexpr int NP = (GT + 1) / 2;
+    static constexpr int NP = (GT + 1) / 2;        // (KB == 8: the same area holds D/4 x GT words of four INT8 queries)
     static constexpr int CH = NIB ? D / 32 : D / 16;
     using Stage = TileStage<CH, true, D>;
     static constexpr int kStageOff = 0;
@@ -37,6 +37,7 @@ struct DecodeSmem {
 
 template <int D, int KB, bool NIB, int GT>
 __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeArgs a) {
+    // KB = 0, 1, 2, 4: power-of-two codes (shift datapath); KB = 8: uniform INT8 comparison code (dp4a)
     using SM = DecodeSmem<D, KB, NIB, GT>;
     using Stage = typename SM::Stage;
     constexpr int EPL = D / 32;
@@ -108,18 +109,39 @@ __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeAr
         if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
     }
     __syncthreads();
-    uint32_t qp_reg[(D * NP + 127) / 128];
+    if constexpr (KB != 8) {
+        uint32_t qp_reg[(D * NP + 127) / 128];
 #pragma unroll
-    for (int k = 0; k < (D * NP + 127) / 128; ++k) {
-        const int idx = threadIdx.x + k * 128;
-        const int m = idx / NP, p = idx % NP;
-        qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
-    }
-    __syncthreads();                                           // q_s is about to be re-used as p_s
+        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+            const int idx = threadIdx.x + k * 128;
+            const int m = idx / NP, p = idx % NP;
+            qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
+        }
+        __syncthreads();                                       // q_s is about to be re-used as p_s
 #pragma unroll
-    for (int k = 0; k < (D * NP + 127) / 128; ++k) {
-        const int idx = threadIdx.x + k * 128;
-        if (idx < D * NP) qp_s[idx / NP][idx % NP] = qp_reg[k];
+        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+            const int idx = threadIdx.x + k * 128;
+            if (idx < D * NP) qp_s[idx / NP][idx % NP] = qp_reg[k];
+        }
+    } else {
+        // four consecutive elements of one query per word, in the byte order of the key words
+        uint32_t* q4_s = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
+        uint32_t q4_reg[(D / 4 * GT + 127) / 128];
+#pragma unroll
+        for (int k = 0; k < (D / 4 * GT + 127) / 128; ++k) {
+            const int idx = threadIdx.x + k * 128;
+            const int w = idx / GT, g = idx % GT;
+            q4_reg[k] = 0u;
+            if (idx < D / 4 * GT)
+                q4_reg[k] = (uint32_t)(q_s[4 * w][g] & 0xff) | ((uint32_t)(q_s[4 * w + 1][g] & 0xff) << 8) |
+                            ((uint32_t)(q_s[4 * w + 2][g] & 0xff) << 16) | ((uint32_t)(q_s[4 * w + 3][g] & 0xff) << 24);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < (D / 4 * GT + 127) / 128; ++k) {
+            const int idx = threadIdx.x + k * 128;
+            if (idx < D / 4 * GT) q4_s[idx] = q4_reg[k];
+        }
     }
     __syncthreads();
 
@@ -156,14 +178,32 @@ __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeAr
 
             // ---- phase 1: integer scores, lane = key; one 32-bit code word (4 or 8 elements) per
             // iteration, kept rolled so that the loop body stays in the instruction cache ----
-            PackedPlanes<KB, NP> pl;
-            pl.begin(a.one);
+            int32_t A[GT];
             const uint32_t* cw = reinterpret_cast<const uint32_t*>(st) + lane * 4;
+            if constexpr (KB != 8) {
+                PackedPlanes<KB, NP> pl;
+                pl.begin(a.one);
 #pragma unroll 1
-            for (int wq = 0; wq < WORDS; ++wq) {
-                const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
-                if constexpr (!NIB) accumulate_word_bytes<KB, NP>(pl, w, &qp_s[wq * 4][0], NP);
-                else accumulate_word_nibbles<NP>(pl, w, &qp_s[wq * 8][0], NP);
+                for (int wq = 0; wq < WORDS; ++wq) {
+                    const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
+                    if constexpr (!NIB) accumulate_word_bytes<KB, NP>(pl, w, &qp_s[wq * 4][0], NP);
+                    else accumulate_word_nibbles<NP>(pl, w, &qp_s[wq * 8][0], NP);
+                }
+#pragma unroll
+                for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
+            } else {
+                // comparison datapath: four INT8 multiply-accumulates per instruction
+                const uint32_t* q4_s = reinterpret_cast<const uint32_t*>(smem + SM::kQpOff);
+#pragma unroll
+                for (int g = 0; g < GT; ++g) A[g] = 0;
+#pragma unroll 4
+                for (int wq = 0; wq < D / 4; ++wq) {
+                    const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
+                    uint32_t q4[GT];
+                    load_np<GT>(q4_s + wq * GT, q4);
+#pragma unroll
+                    for (int g = 0; g < GT; ++g) A[g] = __dp4a((int)q4[g], (int)w, A[g]);
+                }
             }
             const uint32_t meta = reinterpret_cast<const uint32_t*>(st + Stage::kMetaOff)[lane];
 
@@ -176,10 +216,9 @@ __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeAr
             float resc[GT];
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
-                const int32_t A = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
                 if (a.dbg_scores && valid)
-                    a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A;
-                const float z = valid ? (float)A * qscale_s[g] * s_j : -INFINITY;
+                    a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
+                const float z = valid ? (float)A[g] * qscale_s[g] * s_j : -INFINITY;
                 const float zmax = warp_max_f32(z);
                 const int Mt = (int)ceilf(fminf(fmaxf(zmax, -1.0e8f), 1.0e8f));
                 const int Mn = max(M[g], Mt);
@@ -274,6 +313,7 @@ static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
 template <int D>
 static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     if (p.nibble) { launch_gt<D, 0, true>(a, GT, grid, s); return; }
+    if (p.int8) { launch_gt<D, 8, false>(a, GT, grid, s); return; }
     switch (p.k) {
         case 0: launch_gt<D, 0, false>(a, GT, grid, s); break;
         case 1: launch_gt<D, 1, false>(a, GT, grid, s); break;
@@ -299,6 +339,7 @@ extern "C" sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_c
     a.dbg_scores = dbg_scores;
     // logits in the log2 domain: A * Delta * s * 2^-F * log2(e) / sqrt(d)
     a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / (double)(1LL << p.F));
+    if (p.int8) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / 127.0);   // key unit = scale / 127
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (stages & 1) {
         const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);

@@ -20,7 +20,9 @@ __global__ void __launch_bounds__(128) encode_keys_kernel(const uint16_t* __rest
     uint32_t bits[EPL];
     load_vec_bits<EPL>(Kin + v * D, lane, bits);
     uint8_t c[EPL];
-    const uint32_t smax = encode_key_vec<EPL, K>(bits, lane, hadamard != 0, c);
+    uint32_t smax;
+    if constexpr (K == 8) smax = encode_key_int8_vec<EPL>(bits, lane, hadamard != 0, c);
+    else smax = encode_key_vec<EPL, K>(bits, lane, hadamard != 0, c);
     store_bytes<EPL>(codes + v * D + lane * EPL, c);
     if (lane == 0) scales[v] = (uint16_t)smax;
 }
@@ -86,11 +88,16 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
     load_vec_bits<EPL>(krow, lane, kb);
     load_vec_bits<EPL>(vrow, lane, vb);
     uint8_t kc[EPL], vc[EPL];
-    const uint32_t smax = encode_key_vec<EPL, K>(kb, lane, a.hadamard != 0, kc);
-    const int gg = quantise_value_vec<EPL>(vb, vc);
-    // physical exponent field g = 7 - e (0 for the zero code): canonical byte ^ 0x70
+    uint32_t smax;
+    if constexpr (K == 8) {
+        smax = encode_key_int8_vec<EPL>(kb, lane, a.hadamard != 0, kc);      // uniform INT8: stored as is
+    } else {
+        smax = encode_key_vec<EPL, K>(kb, lane, a.hadamard != 0, kc);
+        // physical exponent field g = 7 - e (0 for the zero code): canonical byte ^ 0x70
 #pragma unroll
-    for (int i = 0; i < EPL; ++i) kc[i] ^= 0x70;
+        for (int i = 0; i < EPL; ++i) kc[i] ^= 0x70;
+    }
+    const int gg = quantise_value_vec<EPL>(vb, vc);
     uint8_t* kdst = block + a.kcode_off;
     if (!NIB) {
         const int m = lane * EPL;                   // first element of this lane
@@ -134,12 +141,14 @@ SA_D uint8_t* page_block(const CacheArgs& a, int b, int lp, int h) {
     return a.pages + ((size_t)pidx * a.Hkv + h) * a.page_bytes;
 }
 
-// MODE: 0..4 = quantised with K mantissa bits (byte container), 8 = PoT-4 nibble, 16 = FP16
+// MODE: 0..4 = power-of-two code with K mantissa bits (byte container), 8 = PoT-4 nibble, 16 = FP16,
+// 32 = uniform INT8 comparison code
 template <int D, int MODE>
 SA_D void write_token(uint8_t* block, const CacheArgs& a, int t, int lane, const uint16_t* krow,
                       const uint16_t* vrow) {
     if constexpr (MODE == 16) write_token_fp16<D>(block, a, t, lane, krow, vrow);
     else if constexpr (MODE == 8) write_token_quant<D, 0, true>(block, a, t, lane, krow, vrow);
+    else if constexpr (MODE == 32) write_token_quant<D, 8, false>(block, a, t, lane, krow, vrow);
     else write_token_quant<D, MODE, false>(block, a, t, lane, krow, vrow);
 }
 
@@ -181,7 +190,7 @@ __global__ void __launch_bounds__(128) fill_kernel(CacheArgs a, const uint16_t* 
 
 // sa_debug_unpack
 template <int D, bool NIB>
-__global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, uint8_t* __restrict__ codes,
+__global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, uint8_t xor_mask, uint8_t* __restrict__ codes,
                                                      uint16_t* __restrict__ scales, int8_t* __restrict__ vhat,
                                                      int8_t* __restrict__ g) {
     constexpr int EPL = D / 32;
@@ -198,7 +207,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
         if (!NIB) {
             const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) c[i] = src[i] ^ 0x70;
+            for (int i = 0; i < EPL; ++i) c[i] = src[i] ^ xor_mask;      // 0x70 for the power-of-two codes, 0 for INT8
         } else {
             const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 5) * kPageTokens + t) * 16 + ((m & 31) >> 1);
 #pragma unroll
@@ -245,7 +254,7 @@ static sa_status check_cache(const Plan& p, const sa_cache* c, CacheArgs* a) {
     return SA_OK;
 }
 
-static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.nibble ? 8 : p.k); }
+static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.int8 ? 32 : (p.nibble ? 8 : p.k)); }
 
 #define SA_LAUNCH_CHECK() (cudaGetLastError() == cudaSuccess ? SA_OK : SA_ERR_CUDA)
 
@@ -260,6 +269,7 @@ static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.nibble ? 8 : p.k); }
                 case 2: CALL(64, 2); break;                                             \
                 case 4: CALL(64, 4); break;                                             \
                 case 8: CALL(64, 8); break;                                             \
+                case 32: CALL(64, 32); break;                                           \
                 default: CALL(64, 16); break;                                           \
             }                                                                           \
         } else {                                                                        \
@@ -269,6 +279,7 @@ static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.nibble ? 8 : p.k); }
                 case 2: CALL(128, 2); break;                                            \
                 case 4: CALL(128, 4); break;                                            \
                 case 8: CALL(128, 8); break;                                            \
+                case 32: CALL(128, 32); break;                                          \
                 default: CALL(128, 16); break;                                          \
             }                                                                           \
         }                                                                               \
@@ -295,7 +306,10 @@ sa_status sa_encode_keys(const sa_config* cfg, const uint16_t* K, int64_t n, uin
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int had = p.hadamard ? 1 : 0;
 #define CALL(D, KK) encode_keys_kernel<D, KK><<<grid, 128, 0, s>>>(K, n_vec, codes, scales, had)
-    if (p.d == 64) {
+    if (p.int8) {
+        if (p.d == 64) CALL(64, 8);
+        else CALL(128, 8);
+    } else if (p.d == 64) {
         switch (p.k) { case 0: CALL(64, 0); break; case 1: CALL(64, 1); break; case 2: CALL(64, 2); break; default: CALL(64, 4); }
     } else {
         switch (p.k) { case 0: CALL(128, 0); break; case 1: CALL(128, 1); break; case 2: CALL(128, 2); break; default: CALL(128, 4); }
@@ -401,12 +415,13 @@ sa_status sa_debug_unpack(const sa_config* cfg, const sa_cache* cache, int b, in
     if (n_tokens == 0) return SA_OK;
     const unsigned grid = (unsigned)(((int64_t)n_tokens * a.Hkv + 3) / 4);
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const uint8_t xm = p.int8 ? 0x00 : 0x70;
     if (p.d == 64) {
-        if (p.nibble) unpack_kernel<64, true><<<grid, 128, 0, s>>>(a, b, n_tokens, codes, scales, v_hat, g);
-        else unpack_kernel<64, false><<<grid, 128, 0, s>>>(a, b, n_tokens, codes, scales, v_hat, g);
+        if (p.nibble) unpack_kernel<64, true><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
+        else unpack_kernel<64, false><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
     } else {
-        if (p.nibble) unpack_kernel<128, true><<<grid, 128, 0, s>>>(a, b, n_tokens, codes, scales, v_hat, g);
-        else unpack_kernel<128, false><<<grid, 128, 0, s>>>(a, b, n_tokens, codes, scales, v_hat, g);
+        if (p.nibble) unpack_kernel<128, true><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
+        else unpack_kernel<128, false><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
     }
     return SA_LAUNCH_CHECK();
 }

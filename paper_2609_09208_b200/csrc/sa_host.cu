@@ -33,6 +33,20 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
         *out = p;
         return SA_OK;
     }
+    if (cfg->code == SA_INT8) {
+        if (cfg->klayout != SA_KLAYOUT_BYTE || cfg->headroom_F != 0) return SA_ERR_UNSUPPORTED;
+        p.int8 = true;
+        p.k = 0;
+        p.F = 0;
+        p.f_extra = 0;
+        p.lay.kcode_off = 0;
+        p.lay.meta_off = (size_t)kPageTokens * p.d;
+        p.lay.v_off = p.lay.meta_off + (size_t)kPageTokens * 4;
+        p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d;
+        p.lay.align = 256;
+        *out = p;
+        return SA_OK;
+    }
     if (cfg->code != SA_POT4 && cfg->code != SA_POTM1 && cfg->code != SA_POTM2 && cfg->code != SA_POTM4)
         return SA_ERR_UNSUPPORTED;
     p.k = cfg->code;

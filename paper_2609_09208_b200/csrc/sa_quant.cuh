@@ -53,6 +53,32 @@ SA_D uint32_t encode_key_vec(uint32_t (&bits)[EPL], int lane, bool hadamard, uin
     return smax;
 }
 
+// Key vector -> uniform INT8 codes (the comparison code of section III / VI); returns the scale's
+// binary16 bits (the largest magnitude).  Same rounding rule as the query quantiser.
+template <int EPL>
+SA_D uint32_t encode_key_int8_vec(uint32_t (&bits)[EPL], int lane, bool hadamard, uint8_t (&codes)[EPL]) {
+    float x[EPL];
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) x[i] = half_bits_to_float(bits[i]);
+    if (hadamard) {
+        hadamard_warp<EPL>(x, bits, lane);
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) x[i] = half_bits_to_float(bits[i]);
+    }
+    uint32_t smax = 0;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) smax = max(smax, bits[i] & 0x7fffu);
+    smax = warp_max_u32(smax);
+    const float amax = half_bits_to_float(smax);
+    const float inv = (amax == 0.0f) ? 0.0f : __fdiv_rn(127.0f, amax);
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+        const int r = __float2int_rn(__fmul_rn(x[i], inv));
+        codes[i] = (uint8_t)(int8_t)max(-127, min(127, r));
+    }
+    return smax;
+}
+
 // Query vector -> integers in [-127, 127]; returns the step Delta = amax / 127 (eq. (2)).
 // The rounding decision is taken in FP32 with IEEE divide and multiply, no contraction.
 template <int EPL>

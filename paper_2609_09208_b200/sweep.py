@@ -101,12 +101,12 @@ def main():
         del c
         torch.cuda.empty_cache()
 
-    names = {0: "pot4", 1: "potm1", 2: "potm2", 4: "potm4", 16: "fp16"}
+    names = {0: "pot4", 1: "potm1", 2: "potm2", 4: "potm4", 8: "int8mac", 16: "fp16"}
     cell("cfg1 single head T=1024 pot4", [1024], 1, 1, 64, 0, outliers=False)
     cell("cfg2 llama-1.1B T=4096 potm1 outliers", [4096], 32, 4, 64, 1)
     for B in ([1] if quick else [1, 8, 32]):
         for code, nib, had in [(0, True, False), (0, True, True), (0, False, False), (1, False, False), (2, False, False),
-                               (4, False, False), (4, False, True), (16, False, False)]:
+                               (4, False, False), (4, False, True), (8, False, False), (16, False, False)]:
             cell("cfg3 T=32768 B=%d %s%s%s" % (B, names[code], "_nibble" if nib else "", "+hadamard" if had else ""),
                  [32768] * B, 32, 4, 64, code, nibble=nib, hadamard=had, outliers=False)
     lens4 = np.random.Generator(np.random.PCG64(4001)).integers(2048, 16385, size=16)

@@ -369,3 +369,38 @@ def test_decode_step_from_host_buffers(dev, code):
         else:
             ref = ora.decode_attention(full.Q[b:b + 1], K, V, np.array([0, len(K)]), 4, 10)["O"][0]
         assert np.max(np.abs(Oh.numpy()[b] - ref)) <= TOL_O
+
+
+# ------------------------------------------------------------------------------- INT8 comparison code
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("hadamard", [False, True])
+def test_int8_encode_keys_bit_exact(dev, d, hadamard):
+    import torch
+    rng = np.random.default_rng(2100 + d)
+    Hkv, n = 2, 999
+    K = synth.outlier_keys_fp16(rng, n, Hkv, d)
+    K[3, 1, :] = 0
+    cfg = sa.make_config(d, Hkv, Hkv, sa.SA_INT8, hadamard=hadamard)
+    codes = torch.zeros((n, Hkv, d), dtype=torch.int8, device=dev)
+    scales = torch.zeros((n, Hkv), dtype=torch.int16, device=dev)
+    sa.encode_keys(cfg, t16(K, dev), codes, scales)
+    torch.cuda.synchronize()
+    want_c, want_s = ora.encode_keys_int8(ora.hadamard_fp16(K) if hadamard else K)
+    assert np.array_equal(scales.cpu().numpy().view(np.uint16), want_s.view(np.uint16))
+    assert np.array_equal(codes.cpu().numpy(), want_c)
+
+
+@pytest.mark.parametrize("lens,Hq,Hkv,d,hadamard", [([32768], 32, 4, 64, False), ([0, 1, 33, 700, 64], 8, 2, 64, True),
+                                                    ([4096, 100], 32, 8, 128, False), ([1024], 1, 1, 64, False)])
+def test_int8_decode_matches_oracle(dev, lens, Hq, Hkv, d, hadamard):
+    case = synth.make_case("int8", lens, Hq, Hkv, d, 8, outliers=True, hadamard=hadamard, seed=2200 + d + len(lens))
+    O, dbg, cache = run_decode(case, dev, permute_seed=8)
+    check_against_oracle(case, O, dbg)
+    # the cache holds the oracle's codes
+    for b, T in enumerate(lens):
+        if T == 0:
+            continue
+        K = case.K[case.cu_lens[b]:case.cu_lens[b + 1]]
+        want_c, want_s = ora.encode_keys_int8(ora.hadamard_fp16(K) if hadamard else K)
+        codes, scales, _, _ = _unpack(cfg_of(case), cache, b, T, case, dev)
+        assert np.array_equal(codes.view(np.int8), want_c) and np.array_equal(scales, want_s.view(np.uint16))
