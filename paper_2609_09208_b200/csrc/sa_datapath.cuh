@@ -238,4 +238,67 @@ SA_HD void accumulate_word_nibbles(PackedPlanes<0, NP>& pl, uint32_t w, const ui
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Table datapath for the mantissa codes (KB >= 1).
+//
+// The mantissa factor (2^KB + j) depends only on the key element, the query only on the block:
+// the block prepares U[m][pair][mu] = {q_lo, q_hi}[m] * (2^KB + mu) for mu = 0 .. 2^KB - 1 once, by
+// repeated addition (no multiplication), in shared memory.  The row of one (element, query pair)
+// holds 2^KB entries of 8 bytes — 128 bytes for KB = 4, exactly the 32 banks — so the 32 lanes of
+// a warp, each fetching the entry of ITS key's mantissa, never conflict (equal entries broadcast).
+// Per (query, element) the work is then: half a 64-bit gather, one shift by r = 6 - e, one
+// complement for the sign and one add; the +1 of the two's complement is restored per key from the
+// population count of the sign bits.  The term is at most 127 * 31 * 2^6 < 2^18, the sum of 128 of
+// them fits INT32 (the host checks the bound with the head-room).
+// ---------------------------------------------------------------------------------------------
+template <int KB, int NGP>
+struct TableScore {
+    static constexpr int kRowBytes = 8 << KB;              // one (element, query pair) row
+    static constexpr int kElemBytes = NGP * kRowBytes;     // all query pairs of one element
+    uint32_t acc[2 * NGP];
+    uint32_t corr;
+    uint32_t one;
+    SA_HD void begin(uint32_t one_) {
+        one = one_;
+        corr = 0;
+#pragma unroll
+        for (int g = 0; g < 2 * NGP; ++g) acc[g] = 0;
+    }
+    // one 32-bit word of the byte container = 4 elements; `tab` = table row of the word's first element
+    SA_HD void accumulate_word(uint32_t w, const uint8_t* tab) {
+        const uint32_t gw = (w >> 4) & 0x07070707u;
+        const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;       // shift amounts g - 1; 0xff for the zero code
+        corr += (uint32_t)popc_hd(w & 0x80808080u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);
+            const uint32_t S = prmt_hd(w, 0u, 0x8888u | (0x1111u * i));
+            // byte offset of the mantissa's entry: mu * 8, mu = the byte's low nibble >> (4 - KB)
+            const int sh = 8 * i + 4 - KB - 3;                           // moves mu to bits 3 .. 3 + KB - 1 (folds after unrolling)
+            const uint32_t off = (sh >= 0 ? (w >> (sh >= 0 ? sh : 0)) : (w << (sh < 0 ? -sh : 0))) & (((1u << KB) - 1u) << 3);
+            const uint8_t* row = tab + i * kElemBytes + off;
+#pragma unroll
+            for (int gp = 0; gp < NGP; ++gp) {
+                const uint2 u = *reinterpret_cast<const uint2*>(row + gp * kRowBytes);
+                acc[2 * gp] = add_fma(shl_clamp_hd(u.x, r) ^ S, acc[2 * gp], one);
+                acc[2 * gp + 1] = add_fma(shl_clamp_hd(u.y, r) ^ S, acc[2 * gp + 1], one);
+            }
+        }
+    }
+    SA_HD int32_t score(int g) const { return (int32_t)(acc[g] + corr); }
+};
+
+// Fill the table rows of element m for query pair gp: entry mu = {q_lo, q_hi} * (2^KB + mu).
+template <int KB>
+SA_HD void fill_table_row(uint8_t* row, int q_lo, int q_hi) {
+    uint32_t a = (uint32_t)q_lo << KB, b = (uint32_t)q_hi << KB;
+#pragma unroll
+    for (int mu = 0; mu < (1 << KB); ++mu) {
+        reinterpret_cast<uint32_t*>(row)[2 * mu] = a;
+        reinterpret_cast<uint32_t*>(row)[2 * mu + 1] = b;
+        a += (uint32_t)q_lo;
+        b += (uint32_t)q_hi;
+    }
+}
+
 }  // namespace sa

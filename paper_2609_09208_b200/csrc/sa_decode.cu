@@ -22,22 +22,28 @@ namespace sa {
 //   buffers once every warp has left its tile loop.
 template <int D, int KB, bool NIB, int GT>
 struct DecodeSmem {
-    static constexpr int NP = (GT + 1) / 2;        // (KB == 8: the same area holds D/4 x GT words of four INT8 queries)
+    static constexpr int NP = (GT + 1) / 2;        // query pairs
+    static constexpr bool kTable = (KB == 1 || KB == 2 || KB == 4);   // mantissa codes: table datapath
     static constexpr int CH = NIB ? D / 32 : D / 16;
     using Stage = TileStage<CH, true, D>;
     static constexpr int kStageOff = 0;
     static constexpr int kMbarOff = 4 * kStages * Stage::kBytes;
+    // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
+    // the table of query multiples [D][NP][2^KB] x 8 bytes
     static constexpr int kQpOff = kMbarOff + 128;
-    static constexpr int kQscaleOff = kQpOff + D * NP * 4;
+    static constexpr int kQpBytes = kTable ? D * NP * (8 << KB) : D * NP * 4;
+    static constexpr int kQscaleOff = kQpOff + kQpBytes;
     static constexpr int kPOff = kQscaleOff + 128;
     static constexpr int kPBytes = (4 * 32 * GT * 8 > D * GT * 4) ? 4 * 32 * GT * 8 : D * GT * 4;
     static constexpr int kBytes = kPOff + kPBytes;
+    static constexpr int kBlocksPerSM = kTable ? (KB == 4 ? 3 : 4) : 5;
     static_assert(4 * GT * (D + 2) * 4 <= 4 * kStages * Stage::kBytes, "merge scratch must fit in the stage buffers");
 };
 
 template <int D, int KB, bool NIB, int GT>
-__global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeArgs a) {
-    // KB = 0, 1, 2, 4: power-of-two codes (shift datapath); KB = 8: uniform INT8 comparison code (dp4a)
+__global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM)) decode_kernel(DecodeArgs a) {
+    // KB = 0: PoT-4 (packed shift datapath); KB = 1, 2, 4: mantissa codes (table datapath);
+    // KB = 8: uniform INT8 comparison code (dp4a)
     using SM = DecodeSmem<D, KB, NIB, GT>;
     using Stage = typename SM::Stage;
     constexpr int EPL = D / 32;
@@ -109,7 +115,25 @@ __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeAr
         if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
     }
     __syncthreads();
-    if constexpr (KB != 8) {
+    if constexpr (SM::kTable) {
+        // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
+        using TS = TableScore<KB, NP>;
+        uint8_t* tab = smem + SM::kQpOff;
+        int qlo[(D * NP + 127) / 128], qhi[(D * NP + 127) / 128];
+#pragma unroll
+        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+            const int idx = threadIdx.x + k * 128;
+            const int m = idx / NP, p = idx % NP;
+            qlo[k] = (idx < D * NP) ? q_s[m][2 * p] : 0;
+            qhi[k] = (idx < D * NP && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
+        }
+        __syncthreads();                                       // q_s is about to be re-used as p_s
+#pragma unroll
+        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+            const int idx = threadIdx.x + k * 128;
+            if (idx < D * NP) fill_table_row<KB>(tab + (idx / NP) * TS::kElemBytes + (idx % NP) * TS::kRowBytes, qlo[k], qhi[k]);
+        }
+    } else if constexpr (KB != 8) {
         uint32_t qp_reg[(D * NP + 127) / 128];
 #pragma unroll
         for (int k = 0; k < (D * NP + 127) / 128; ++k) {
@@ -180,7 +204,17 @@ __global__ void __launch_bounds__(128, (KB == 4) ? 4 : 5) decode_kernel(DecodeAr
             // iteration, kept rolled so that the loop body stays in the instruction cache ----
             int32_t A[GT];
             const uint32_t* cw = reinterpret_cast<const uint32_t*>(st) + lane * 4;
-            if constexpr (KB != 8) {
+            if constexpr (SM::kTable) {
+                using TS = TableScore<KB, NP>;
+                const uint8_t* tab = smem + SM::kQpOff;
+                TS ts;
+                ts.begin(a.one);
+#pragma unroll 4
+                for (int wq = 0; wq < WORDS; ++wq)
+                    ts.accumulate_word(cw[(wq >> 2) * 128 + (wq & 3)], tab + wq * 4 * TS::kElemBytes);
+#pragma unroll
+                for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)ts.score(g) << a.f_extra);   // exact: the true sum fits INT32
+            } else if constexpr (KB != 8) {
                 PackedPlanes<KB, NP> pl;
                 pl.begin(a.one);
 #pragma unroll 1

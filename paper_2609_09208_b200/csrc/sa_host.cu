@@ -80,7 +80,7 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
     // One thread block per (split, KV head x query chunk, sequence).  Aim for a few blocks per
     // SM; every block should still own at least one 32-key tile per warp.
     const long long units = (long long)batch * p.Hkv * (p.G / GT);
-    const long long target = (long long)kNumSMs * (p.fp16 ? 3 : (p.k == 4 ? 4 : 5));   // resident blocks per SM of the kernel that will run: one full wave
+    const long long target = (long long)kNumSMs * (p.fp16 ? 3 : (p.k == 4 ? 3 : (p.k >= 1 ? 4 : 5)));   // resident blocks per SM of the kernel that will run: one full wave
     long long S = (target + units - 1) / units;
     const long long max_tiles = (long long)max_pages * (kPageTokens / 32);
     long long cap = max_tiles / 4;

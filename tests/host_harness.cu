@@ -30,7 +30,32 @@ static void score8(const uint8_t* canon, const int8_t* q8, int d, bool nibble_pa
     for (int g = 0; g < 8; ++g) out[g] = pl.score(g);
 }
 
+// The same scores through the table datapath of the mantissa codes.
+template <int K>
+static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
+    using TS = TableScore<K, 4>;
+    alignas(16) static uint8_t tab[128 * TS::kElemBytes];
+    for (int m = 0; m < d; ++m)
+        for (int gp = 0; gp < 4; ++gp)
+            fill_table_row<K>(tab + m * TS::kElemBytes + gp * TS::kRowBytes, q8[(2 * gp) * d + m], q8[(2 * gp + 1) * d + m]);
+    TS ts;
+    ts.begin(1u);
+    for (int m0 = 0; m0 < d; m0 += 4) {
+        uint32_t w = 0;
+        for (int i = 0; i < 4; ++i) w |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * i);
+        ts.accumulate_word(w, tab + m0 * TS::kElemBytes);
+    }
+    for (int g = 0; g < 8; ++g) out[g] = ts.score(g);
+}
+
 extern "C" {
+void hh_score8_table(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
+    switch (k) {
+        case 1: score8_table<1>(canon, q8, d, out); break;
+        case 2: score8_table<2>(canon, q8, d, out); break;
+        default: score8_table<4>(canon, q8, d, out); break;
+    }
+}
 int hh_encode_element(int k, unsigned a_bits, unsigned s_bits) {
     switch (k) {
         case 0: return encode_element<0>(a_bits, s_bits);

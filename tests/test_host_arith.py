@@ -100,3 +100,8 @@ def test_packed_plane_datapath_equals_oracle_scores(hh, k, d):
             hh.hh_score8(C.c_int(0), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
                          C.c_int(1), out.ctypes.data_as(C.c_void_p))
             assert np.array_equal(out.astype(np.int64), want[:, 0]), ("nibble", trial)
+        else:
+            # the table datapath of the mantissa codes gives the same integers
+            hh.hh_score8_table(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
+                               out.ctypes.data_as(C.c_void_p))
+            assert np.array_equal(out.astype(np.int64), want[:, 0]), ("table", trial, out, want[:, 0])
