@@ -119,19 +119,29 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
         // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
         using TS = TableScore<KB, NP>;
         uint8_t* tab = smem + SM::kQpOff;
-        int qlo[(D * NP + 127) / 128], qhi[(D * NP + 127) / 128];
+        // One thread per table entry and pass: consecutive threads write consecutive 8-byte entries
+        // (no bank conflicts).  The factor 2^KB + mu is applied by shift-and-add over the bits of mu.
+        constexpr int ENT = D * NP * (1 << KB);                // entries of {q_lo, q_hi} * (2^KB + mu)
+        constexpr int PASSES = (ENT + 127) / 128;
+        uint2 ent[PASSES];
 #pragma unroll
-        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
-            const int idx = threadIdx.x + k * 128;
-            const int m = idx / NP, p = idx % NP;
-            qlo[k] = (idx < D * NP) ? q_s[m][2 * p] : 0;
-            qhi[k] = (idx < D * NP && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
+        for (int k = 0; k < PASSES; ++k) {
+            const int idx = threadIdx.x + k * 128;             // = (m * NP + p) * 2^KB + mu
+            const int mu = idx & ((1 << KB) - 1), row = idx >> KB;
+            const int m = row / NP, p = row % NP;
+            const int qlo = (idx < ENT) ? q_s[m][2 * p] : 0;
+            const int qhi = (idx < ENT && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
+            uint32_t a = (uint32_t)qlo << KB, b = (uint32_t)qhi << KB;
+#pragma unroll
+            for (int bit = 0; bit < KB; ++bit)
+                if (mu & (1 << bit)) { a += (uint32_t)qlo << bit; b += (uint32_t)qhi << bit; }
+            ent[k] = make_uint2(a, b);
         }
         __syncthreads();                                       // q_s is about to be re-used as p_s
 #pragma unroll
-        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
+        for (int k = 0; k < PASSES; ++k) {
             const int idx = threadIdx.x + k * 128;
-            if (idx < D * NP) fill_table_row<KB>(tab + (idx / NP) * TS::kElemBytes + (idx % NP) * TS::kRowBytes, qlo[k], qhi[k]);
+            if (idx < ENT) reinterpret_cast<uint2*>(tab)[idx] = ent[k];
         }
     } else if constexpr (KB != 8) {
         uint32_t qp_reg[(D * NP + 127) / 128];
