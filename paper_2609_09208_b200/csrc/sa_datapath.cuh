@@ -92,7 +92,8 @@ SA_HD void load_np(const uint32_t* src, uint32_t (&q)[NP]) {
     }
 }
 
-// a * w + c on the FMA pipe (w is a power of two held in a register: a shift-and-add).
+// a * w + c on the FMA pipe; w is either a power of two held in a register (a shift-and-add) or a
+// sign +1 / -1 (a sign flip and an add).
 SA_HD uint32_t mad_fma(uint32_t a, uint32_t w, uint32_t c) {
 #ifdef __CUDA_ARCH__
     uint32_t d;
@@ -246,21 +247,18 @@ SA_HD void accumulate_word_nibbles(PackedPlanes<0, NP>& pl, uint32_t w, const ui
 // repeated addition (no multiplication), in shared memory.  The row of one (element, query pair)
 // holds 2^KB entries of 8 bytes — 128 bytes for KB = 4, exactly the 32 banks — so the 32 lanes of
 // a warp, each fetching the entry of ITS key's mantissa, never conflict (equal entries broadcast).
-// Per (query, element) the work is then: half a 64-bit gather, one shift by r = 6 - e, one
-// complement for the sign and one add; the +1 of the two's complement is restored per key from the
-// population count of the sign bits.  The term is at most 127 * 31 * 2^6 < 2^18, the sum of 128 of
-// them fits INT32 (the host checks the bound with the head-room).
+// Per (query, element) the work is then: half a 64-bit gather, one shift by r = 6 - e on the ALU
+// pipe, and one multiply-add by sigma = +1 or -1 on the FMA pipe, which is the sign flip and the
+// accumulation in one instruction (the multiplier only ever sees +1 or -1: magnitudes are shifted,
+// never multiplied).  The term is at most 127 * 31 * 2^6 < 2^18, the sum of 128 of them fits
+// INT32 (the host checks the bound with the head-room).
 // ---------------------------------------------------------------------------------------------
 template <int KB, int NGP>
 struct TableScore {
     static constexpr int kRowBytes = 8 << KB;              // one (element, query pair) row
     static constexpr int kElemBytes = NGP * kRowBytes;     // all query pairs of one element
     uint32_t acc[2 * NGP];
-    uint32_t corr;
-    uint32_t one;
-    SA_HD void begin(uint32_t one_) {
-        one = one_;
-        corr = 0;
+    SA_HD void begin(uint32_t) {
 #pragma unroll
         for (int g = 0; g < 2 * NGP; ++g) acc[g] = 0;
     }
@@ -268,11 +266,10 @@ struct TableScore {
     SA_HD void accumulate_word(uint32_t w, const uint8_t* tab) {
         const uint32_t gw = (w >> 4) & 0x07070707u;
         const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;       // shift amounts g - 1; 0xff for the zero code
-        corr += (uint32_t)popc_hd(w & 0x80808080u);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);
-            const uint32_t S = prmt_hd(w, 0u, 0x8888u | (0x1111u * i));
+            const uint32_t sg = prmt_hd(w, 0u, 0x8888u | (0x1111u * i)) | 1u;   // sigma: +1 or -1
             // byte offset of the mantissa's entry: mu * 8, mu = the byte's low nibble >> (4 - KB)
             const int sh = 8 * i + 4 - KB - 3;                           // moves mu to bits 3 .. 3 + KB - 1 (folds after unrolling)
             const uint32_t off = (sh >= 0 ? (w >> (sh >= 0 ? sh : 0)) : (w << (sh < 0 ? -sh : 0))) & (((1u << KB) - 1u) << 3);
@@ -280,12 +277,12 @@ struct TableScore {
 #pragma unroll
             for (int gp = 0; gp < NGP; ++gp) {
                 const uint2 u = *reinterpret_cast<const uint2*>(row + gp * kRowBytes);
-                acc[2 * gp] = add_fma(shl_clamp_hd(u.x, r) ^ S, acc[2 * gp], one);
-                acc[2 * gp + 1] = add_fma(shl_clamp_hd(u.y, r) ^ S, acc[2 * gp + 1], one);
+                acc[2 * gp] = mad_fma(shl_clamp_hd(u.x, r), sg, acc[2 * gp]);
+                acc[2 * gp + 1] = mad_fma(shl_clamp_hd(u.y, r), sg, acc[2 * gp + 1]);
             }
         }
     }
-    SA_HD int32_t score(int g) const { return (int32_t)(acc[g] + corr); }
+    SA_HD int32_t score(int g) const { return (int32_t)acc[g]; }
 };
 
 // Fill the table rows of element m for query pair gp: entry mu = {q_lo, q_hi} * (2^KB + mu).
