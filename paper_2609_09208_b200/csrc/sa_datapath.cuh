@@ -1,25 +1,22 @@
 // The integer score datapath of the decode kernel (section II-B eq. (3), II-C eq. (4), II-D
-// eq. (5)): shifts, sign flips, masks and adds only.  Everything here also compiles for the host so
+// eq. (5)): shifts, sign flips and adds only.  Everything here also compiles for the host so
 // that the unit tests can run the very same arithmetic against the CPU oracle without a GPU.
 //
 // Term of element m at head-room F0 = 6 + KB:  sigma * (qhat << r) * (2^KB + j),  r = 6 - e >= 0.
 //
+// PoT-4 (KB = 0), packed datapath:
 // * Two queries share one 32-bit register: P = (q_hi << 16) + q_lo as a 32-bit integer (a negative
 //   q_lo borrows from the upper half; all arithmetic below is plain integer arithmetic on P, so
 //   the two halves stay exact as long as the lower half's running sum fits in 16 bits).  One
-//   shift, one logic op and one add then serve two (query, element) pairs.
-// * The mantissa is handled in KB + 1 "planes": plane KB takes sigma*(P << r) of every element,
-//   plane b < KB only of the elements whose mantissa bit b is set; score = sum_b plane_b << b.
-// * The sign flip is a bitwise complement fused with the plane mask into one logic op
-//   ((x ^ S) & m); the "+1" that a two's complement would add is restored per key from population
-//   counts of the sign bits (it only concerns the lower half: the upper half of ~x is exact).
-// * A window of 4 elements (4 * 127 * 2^6 + 4 < 2^15) is accumulated in the packed register,
-//   whose lower half is biased by 0x8000 so that it never borrows; then both halves are added
-//   into 32-bit totals, weighted by the plane's 2^b.
-// * Adds are written as multiply-add by a 1 the compiler cannot see, so that they issue on the
-//   FMA pipe while shifts and logic ops issue on the ALU pipe: on sm_100a the two pipes run side
-//   by side (64 + 64 thread-instructions per clock per SM), and the integer ALU pipe is what
-//   bounds this kernel.
+//   shift and one add then serve two (query, element) pairs.
+// * The sign flip and the add are one multiply-add by sigma = +1 or -1 (the multiplier only ever
+//   sees +1 or -1: magnitudes are shifted, never multiplied).  It issues on the FMA pipe while the
+//   shifts and byte permutes issue on the ALU pipe: on sm_100a the two pipes run side by side
+//   (64 + 64 thread-instructions per clock per SM).
+// * A window of 4 elements (4 * 127 * 2^6 < 2^15) is accumulated in the packed register, whose
+//   lower half is biased by 0x8000 so that it never borrows; then both halves are added into
+//   32-bit totals.
+// Mantissa codes (KB = 1, 2, 4): table datapath, see TableScore below.
 //
 // Physical code format inside a page (differs from the canonical byte only in the exponent field):
 // byte = sign << 7 | g << 4 | mantissa, g = 7 - e for a non-zero element and 0 for the zero code,
@@ -106,134 +103,88 @@ SA_HD uint32_t mad_fma(uint32_t a, uint32_t w, uint32_t c) {
 
 SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (uint32_t)q_lo; }
 
-// Accumulators for 2 * NP queries against one key.
+// Accumulators for 2 * NP queries against one PoT-4 key.
 //
 // Flush of a window register W = h * 2^16 + l (l = biased lower half, 0 <= l < 2^16): instead of
 // separating both halves, two totals are kept modulo 2^32,
-//     tot += W << b        and        hit += h << b        (h = W >> 16, arithmetic),
-// and at the end  lower-query sum = tot - (hit << 16)  (exact: the true value is far below 2^32)
-// and  upper-query sum = hit.  That is one ALU instruction and two FMA-pipe multiply-adds (by the
-// plane weight 2^b held in a register) per window register.
-template <int KB, int NP>
-struct PackedPlanes {
-    uint32_t win[KB + 1][NP];   // window sums, lower half biased by 0x8000
+//     tot += W        and        hit += h        (h = W >> 16, arithmetic),
+// and at the end  lower-query sum = tot - (hit << 16) - bias  (exact: the true value is far below
+// 2^32) and  upper-query sum = hit.  That is one ALU instruction and two FMA-pipe adds per window
+// register.
+template <int NP>
+struct PackedShift {
+    uint32_t win[NP];           // window sums, lower half biased by 0x8000
     uint32_t tot[NP], hit[NP];  // running totals, see above
-    uint32_t corr;              // sum_b 2^b * (number of complemented terms in plane b)
     uint32_t n_windows;
-    uint32_t pw[KB + 1];        // plane weights 2^b as run-time values (pw[0] doubles as the opaque 1)
+    uint32_t one;               // 1, as a run-time value (keeps the adds on the FMA pipe)
 
-    SA_HD void begin(uint32_t one) {
-        corr = 0;
+    SA_HD void begin(uint32_t one_) {
+        one = one_;
         n_windows = 0;
-#pragma unroll
-        for (int b = 0; b <= KB; ++b) pw[b] = one << b;
 #pragma unroll
         for (int p = 0; p < NP; ++p) tot[p] = hit[p] = 0;
     }
-    // First element of a window: starts every plane from the bias; the mantissa planes take the
-    // term through a mask.  r: shift amount (>= 32 for the zero code); S: 0 or 0xffffffff;
-    // mask[b]: 0 or 0xffffffff.
-    SA_HD void element_first(uint32_t r, uint32_t S, const uint32_t* mask, const uint32_t* qp) {
+    // r: shift amount (>= 32 for the zero code); sg: +1 or -1
+    SA_HD void element_first(uint32_t r, uint32_t sg, const uint32_t* qp) {
 #pragma unroll
-        for (int p = 0; p < NP; ++p) {
-            const uint32_t t = shl_clamp_hd(qp[p], r) ^ S;
-            win[KB][p] = add_fma(t, 0x8000u, pw[0]);
-#pragma unroll
-            for (int b = 0; b < KB; ++b) win[b][p] = add_fma(t & mask[b], 0x8000u, pw[0]);
-        }
+        for (int p = 0; p < NP; ++p) win[p] = mad_fma(shl_clamp_hd(qp[p], r), sg, 0x8000u);
     }
-    // Later elements: a mantissa plane receives the term only if its bit is set.  The condition is
-    // the same for all queries, so it costs one predicate per (element, bit) instead of one logic
-    // op per (query pair, element, bit); the adds under it are predicated.
-    SA_HD void element_next(uint32_t r, uint32_t S, const bool* on, const uint32_t* qp) {
-        uint32_t t[NP];
+    SA_HD void element_next(uint32_t r, uint32_t sg, const uint32_t* qp) {
 #pragma unroll
-        for (int p = 0; p < NP; ++p) {
-            t[p] = shl_clamp_hd(qp[p], r) ^ S;
-            win[KB][p] = add_fma(t[p], win[KB][p], pw[0]);
-        }
-#pragma unroll
-        for (int b = 0; b < KB; ++b)
-            if (on[b]) {
-#pragma unroll
-                for (int p = 0; p < NP; ++p) win[b][p] = add_fma(t[p], win[b][p], pw[0]);
-            }
+        for (int p = 0; p < NP; ++p) win[p] = mad_fma(shl_clamp_hd(qp[p], r), sg, win[p]);
     }
     SA_HD void window_end() {
         ++n_windows;
 #pragma unroll
-        for (int b = 0; b <= KB; ++b)
-#pragma unroll
-            for (int p = 0; p < NP; ++p) {
-                const uint32_t h = (uint32_t)((int32_t)win[b][p] >> 16);      // exact upper half
-                tot[p] = mad_fma(win[b][p], pw[b], tot[p]);
-                hit[p] = mad_fma(h, pw[b], hit[p]);
-            }
+        for (int p = 0; p < NP; ++p) {
+            const uint32_t h = (uint32_t)((int32_t)win[p] >> 16);      // exact upper half
+            tot[p] = add_fma(win[p], tot[p], one);
+            hit[p] = add_fma(h, hit[p], one);
+        }
     }
     // score of query g (g even: lower half of register g / 2), before the final head-room shift
     SA_HD int32_t score(int g) const {
-        const uint32_t bias = n_windows * 0x8000u * ((2u << KB) - 1u);
-        return (g & 1) ? (int32_t)hit[g >> 1] : (int32_t)(tot[g >> 1] - (hit[g >> 1] << 16) - bias + corr);
+        return (g & 1) ? (int32_t)hit[g >> 1] : (int32_t)(tot[g >> 1] - (hit[g >> 1] << 16) - n_windows * 0x8000u);
     }
 };
 
 // One 32-bit word of the byte container = 4 elements.  qp points at the packed queries of the
 // word's first element; consecutive elements are `stride` words apart.
-template <int KB, int NP>
-SA_HD void accumulate_word_bytes(PackedPlanes<KB, NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
+template <int NP>
+SA_HD void accumulate_word_bytes(PackedShift<NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
     // shift amounts g - 1 per byte: 0..6, and 0xff for the zero code (g = 0)
     const uint32_t gw = (w >> 4) & 0x07070707u;
     const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;
-    const uint32_t neg = w & 0x80808080u;
-    uint32_t wb[KB > 0 ? KB : 1];
-    pl.corr += (uint32_t)popc_hd(neg) << KB;
-#pragma unroll
-    for (int b = 0; b < KB; ++b) {
-        wb[b] = w << (3 + KB - b);              // mantissa bit b of every byte moved to the byte's top bit
-        pl.corr += (uint32_t)popc_hd(neg & wb[b]) << b;
-    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const uint32_t rep = 0x8888u | (0x1111u * i);          // replicate the top bit of byte i
-        const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);       // byte i, zero-extended
-        const uint32_t S = prmt_hd(w, 0u, rep);
+        const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);                          // byte i, zero-extended
+        const uint32_t sg = prmt_hd(w, 0u, 0x8888u | (0x1111u * i)) | 1u;         // top bit of byte i replicated, | 1
         uint32_t q[NP];
         load_np<NP>(qp + i * stride, q);
-        if (i == 0) {
-            uint32_t mask[KB > 0 ? KB : 1];
-#pragma unroll
-            for (int b = 0; b < KB; ++b) mask[b] = prmt_hd(wb[b], 0u, rep);
-            pl.element_first(r, S, mask, q);
-        } else {
-            bool on[KB > 0 ? KB : 1];
-#pragma unroll
-            for (int b = 0; b < KB; ++b) on[b] = (wb[b] & (0x80u << (8 * i))) != 0u;
-            pl.element_next(r, S, on, q);
-        }
+        if (i == 0) pl.element_first(r, sg, q);
+        else pl.element_next(r, sg, q);
     }
     pl.window_end();
 }
 
-// One 32-bit word of the nibble container (PoT-4 only) = 8 elements, two windows.
+// One 32-bit word of the nibble container = 8 elements, two windows.
 template <int NP>
-SA_HD void accumulate_word_nibbles(PackedPlanes<0, NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
+SA_HD void accumulate_word_nibbles(PackedShift<NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
     const uint32_t ge = w & 0x07070707u, go = (w >> 4) & 0x07070707u;   // g of even / odd elements
     const uint32_t re = (ge + 0x7f7f7f7fu) ^ 0x80808080u, ro = (go + 0x7f7f7f7fu) ^ 0x80808080u;
     const uint32_t we = w << 4;                                         // even elements' sign at the byte's top bit
-    pl.corr += (uint32_t)popc_hd(w & 0x88888888u);
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int ni = half * 4 + i;                                // element within the word
             const int byte = ni >> 1;
-            const uint32_t rep = 0x8888u | (0x1111u * byte);
             const uint32_t r = prmt_hd((ni & 1) ? ro : re, 0u, 0x4440u | byte);
-            const uint32_t S = prmt_hd((ni & 1) ? w : we, 0u, rep);
+            const uint32_t sg = prmt_hd((ni & 1) ? w : we, 0u, 0x8888u | (0x1111u * byte)) | 1u;
             uint32_t q[NP];
             load_np<NP>(qp + ni * stride, q);
-            if (i == 0) pl.element_first(r, S, nullptr, q);
-            else pl.element_next(r, S, nullptr, q);
+            if (i == 0) pl.element_first(r, sg, q);
+            else pl.element_next(r, sg, q);
         }
         pl.window_end();
     }

@@ -225,12 +225,12 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)ts.score(g) << a.f_extra);   // exact: the true sum fits INT32
             } else if constexpr (KB != 8) {
-                PackedPlanes<KB, NP> pl;
+                PackedShift<NP> pl;
                 pl.begin(a.one);
 #pragma unroll 1
                 for (int wq = 0; wq < WORDS; ++wq) {
                     const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
-                    if constexpr (!NIB) accumulate_word_bytes<KB, NP>(pl, w, &qp_s[wq * 4][0], NP);
+                    if constexpr (!NIB) accumulate_word_bytes<NP>(pl, w, &qp_s[wq * 4][0], NP);
                     else accumulate_word_nibbles<NP>(pl, w, &qp_s[wq * 8][0], NP);
                 }
 #pragma unroll

@@ -5,22 +5,21 @@
 
 using namespace sa;
 
-// Scores of one key (canonical code bytes) against 8 queries, through the same packed plane
+// Scores of one PoT-4 key (canonical code bytes) against 8 queries, through the same packed
 // datapath and word decoders the decode kernel uses (physical codes = canonical ^ 0x70).
-template <int K>
-static void score8(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
+static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
     alignas(16) static uint32_t qp[128][4];
     for (int m = 0; m < d; ++m)
         for (int p = 0; p < 4; ++p) qp[m][p] = pack_pair(q8[(2 * p) * d + m], q8[(2 * p + 1) * d + m]);
-    PackedPlanes<K, 4> pl;
+    PackedShift<4> pl;
     pl.begin(1u);
     if (!nibble_path) {
         for (int m0 = 0; m0 < d; m0 += 4) {
             uint32_t w = 0;
             for (int i = 0; i < 4; ++i) w |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * i);
-            accumulate_word_bytes<K, 4>(pl, w, &qp[m0][0], 4);
+            accumulate_word_bytes<4>(pl, w, &qp[m0][0], 4);
         }
-    } else if constexpr (K == 0) {
+    } else {
         for (int m0 = 0; m0 < d; m0 += 8) {
             uint32_t w = 0;
             for (int i = 0; i < 8; ++i) w |= (uint32_t)((canon[m0 + i] ^ 0x70) >> 4) << (4 * i);
@@ -30,6 +29,7 @@ static void score8(const uint8_t* canon, const int8_t* q8, int d, bool nibble_pa
     for (int g = 0; g < 8; ++g) out[g] = pl.score(g);
 }
 
+// The scores of a mantissa code (k = 1, 2, 4) through the table datapath.
 // The same scores through the table datapath of the mantissa codes.
 template <int K>
 static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
@@ -69,11 +69,7 @@ void hh_encode_many(int k, const uint16_t* a_bits, int64_t n, unsigned s_bits, u
 }
 int hh_value_exponent(unsigned amax_bits) { return value_exponent(amax_bits); }
 void hh_score8(int k, const uint8_t* canon, const int8_t* q8, int d, int nibble_path, int32_t* out) {
-    switch (k) {
-        case 0: score8<0>(canon, q8, d, nibble_path != 0, out); break;
-        case 1: score8<1>(canon, q8, d, false, out); break;
-        case 2: score8<2>(canon, q8, d, false, out); break;
-        default: score8<4>(canon, q8, d, false, out); break;
-    }
+    if (k == 0) score8_packed(canon, q8, d, nibble_path != 0, out);
+    else hh_score8_table(k, canon, q8, d, out);
 }
 }

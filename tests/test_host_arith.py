@@ -1,6 +1,6 @@
 """The library's exact-arithmetic functions, compiled for the host, against the CPU oracle.
 
-The key-element encoder, the value exponent and the plane-accumulator score datapath are plain
+The key-element encoder, the value exponent and the packed-shift and table score datapaths are plain
 integer code that nvcc also compiles for the host; this checks them exhaustively / on random
 inputs without a GPU.  (The same functions run on the device in the -m gpu parity tests.)"""
 import ctypes as C
@@ -62,9 +62,9 @@ def test_value_exponent_all_magnitudes(hh):
 
 @pytest.mark.parametrize("k", [0, 1, 2, 4])
 @pytest.mark.parametrize("d", [64, 128])
-def test_packed_plane_datapath_equals_oracle_scores(hh, k, d):
+def test_score_datapaths_equal_oracle_scores(hh, k, d):
     """Eight queries (two per 32-bit register) against one key through the kernel's word decoders
-    and packed plane accumulators, including the cases that stress the 16-bit halves: every term
+    and packed accumulators, including the cases that stress the 16-bit halves: every term
     negative at the largest shift, extreme queries, zero codes with and without a sign bit."""
     rng = np.random.default_rng(100 + k + d)
     out = np.zeros(8, dtype=np.int32)
