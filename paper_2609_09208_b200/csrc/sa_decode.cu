@@ -4,13 +4,16 @@
 // heads into shared memory, then each of its four warps walks its own 32-key tiles of the
 // block's slice of the key axis with a private online-softmax state, so the main loop has no
 // block-wide barrier.  Per tile: lane = key for the integer scores (section II-B eq. (3) with
-// the mantissa code of eq. (5)), warp-shuffle maxima and an integer running maximum in the log2
-// domain (section II-E), then lane = (token group, 8 output dims) for the floating-point A.V
-// over the INT8 values.  The four warps' states and then the blocks' partial results are merged
-// with exact power-of-two factors.
+// the mantissa code of eq. (5)), warp-wide maxima and an integer running maximum in the log2
+// domain (section II-E); then the floating-point A.V over the INT8 values as small tensor-core
+// products O^T[dims][queries] += V^T[dims][keys] P^T[keys][queries] (mma.m16n8k8, tf32 operands:
+// the INT8 values are exact, every weight is split into two tf32 terms, accumulation in FP32).
+// The four warps' states and then the blocks' partial results are merged with exact
+// power-of-two factors.
 #include "sa_common.cuh"
 #include "sa_datapath.cuh"
 #include "sa_decode_common.cuh"
+#include "sa_mma.cuh"
 #include "sa_quant.cuh"
 #include "sa_stage.cuh"
 
@@ -34,7 +37,8 @@ struct DecodeSmem {
     static constexpr int kQpBytes = kTable ? D * NP * (8 << KB) : D * NP * 4;
     static constexpr int kQscaleOff = kQpOff + kQpBytes;
     static constexpr int kPOff = kQscaleOff + 128;
-    static constexpr int kPBytes = (4 * 32 * GT * 8 > D * GT * 4) ? 4 * 32 * GT * 8 : D * GT * 4;
+    // weights: per warp two tf32 terms x 32 key rows x 8 query columns of FP32
+    static constexpr int kPBytes = (4 * 2 * 32 * 8 * 4 > D * GT * 4) ? 4 * 2 * 32 * 8 * 4 : D * GT * 4;
     static constexpr int kBytes = kPOff + kPBytes;
     static constexpr int kBlocksPerSM = kTable ? (KB == 4 ? 3 : 4) : 5;
     static_assert(4 * GT * (D + 2) * 4 <= 4 * kStages * Stage::kBytes, "merge scratch must fit in the stage buffers");
@@ -49,14 +53,11 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
     constexpr int EPL = D / 32;
     constexpr int NP = SM::NP;
     constexpr int WORDS = NIB ? D / 8 : D / 4;     // 32-bit code words per key
-    constexpr int NJ = 2;                          // output-dim pairs per lane in the A.V phase (4 dims)
-    constexpr int LPT = D / (2 * NJ);              // lanes covering one token's value row
-    constexpr int TS = 32 / LPT;                   // token groups in the A.V phase
-    constexpr int TPL = 32 / TS;                   // tokens per lane per tile
+    constexpr int MT = D / 16;                     // 16-dim row tiles of O^T in the A.V phase
     extern __shared__ __align__(128) uint8_t smem[];
     uint32_t (*qp_s)[NP] = reinterpret_cast<uint32_t (*)[NP]>(smem + SM::kQpOff);
     float* qscale_s = reinterpret_cast<float*>(smem + SM::kQscaleOff);
-    float2 (*p_s)[32][GT] = reinterpret_cast<float2 (*)[32][GT]>(smem + SM::kPOff);
+    float (*p_s)[2][32][8] = reinterpret_cast<float (*)[2][32][8]>(smem + SM::kPOff);   // [warp][term][key row][query]
     int32_t (*q_s)[GT] = reinterpret_cast<int32_t (*)[GT]>(smem + SM::kPOff);      // prologue only
     float (*red_s)[GT][D + 2] = reinterpret_cast<float (*)[GT][D + 2]>(smem + SM::kStageOff);
 
@@ -177,19 +178,25 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
             if (idx < D / 4 * GT) q4_s[idx] = q4_reg[k];
         }
     }
+    // query columns beyond GT stay zero for the whole kernel (q_s, which shared this space, is no longer read)
+    for (int idx = threadIdx.x; idx < 4 * 2 * 32 * 8; idx += 128) (&p_s[0][0][0][0])[idx] = 0.0f;
     __syncthreads();
 
     int M[GT];
     float l[GT];
-    unsigned long long acc[GT][NJ];
+    float acc[MT][4];        // O^T tiles: lane (gq, t4) holds dims 16 mt + 2 gq (+1) of queries 2 t4 (+1)
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         M[g] = kMNone;
         l[g] = 0.0f;
-#pragma unroll
-        for (int j = 0; j < NJ; ++j) acc[g][j] = 0ull;
     }
-    const int ts = lane / LPT, dc = lane % LPT;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[mt][c] = 0.0f;
+    const int gq = lane >> 2, t4 = lane & 3;
+    // row of this lane's key in the weight buffer: within a group of 8 keys the even keys come first
+    const int prow = (lane & 24) | ((lane & 1) << 2) | ((lane & 7) >> 1);
     bool failed = false;
 
     for (int i = 0; i < n_my; ++i) {
@@ -257,56 +264,82 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
             const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
             const float vscale = valid ? pow2i(-g_j) : 0.0f;  // 2^-g_j; g_j in [-10, 30] for written tokens
             bool changed = false;
-            float resc[GT];
+            float resc[GT], p_hi[GT], p_lo[GT];
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 if (a.dbg_scores && valid)
                     a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
                 const float z = valid ? (float)A[g] * qscale_s[g] * s_j : -INFINITY;
-                const float zmax = warp_max_f32(z);
-                const int Mt = (int)ceilf(fminf(fmaxf(zmax, -1.0e8f), 1.0e8f));
+                // ceil of the tile's largest logit: ceil is monotone, so take the integer maximum
+                const int Mt = warp_max_s32(__float2int_ru(fminf(fmaxf(z, -1.0e8f), 1.0e8f)));
                 const int Mn = max(M[g], Mt);
                 resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);          // exact power of two
                 changed |= (Mn != M[g]);
                 M[g] = Mn;
                 const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
                 l[g] = l[g] * resc[g] + p;
+                // weight times 2^-g_j, as two tf32 terms (low 13 mantissa bits zero)
                 const float pv = p * vscale;
-                p_s[warp][lane][g] = make_float2(pv, pv);
+                p_hi[g] = __uint_as_float(__float_as_uint(pv) & 0xffffe000u);
+                p_lo[g] = __uint_as_float(__float_as_uint(pv - p_hi[g]) & 0xffffe000u);
             }
-            if (changed) {                                    // warp-uniform
+            if constexpr (GT == 8) {
+                float4* ph = reinterpret_cast<float4*>(&p_s[warp][0][prow][0]);
+                float4* pl = reinterpret_cast<float4*>(&p_s[warp][1][prow][0]);
+                ph[0] = make_float4(p_hi[0], p_hi[1], p_hi[2], p_hi[3]);
+                ph[1] = make_float4(p_hi[4], p_hi[5], p_hi[6], p_hi[7]);
+                pl[0] = make_float4(p_lo[0], p_lo[1], p_lo[2], p_lo[3]);
+                pl[1] = make_float4(p_lo[4], p_lo[5], p_lo[6], p_lo[7]);
+            } else {
 #pragma unroll
                 for (int g = 0; g < GT; ++g) {
-                    const unsigned long long r2 = pack_f32x2(resc[g], resc[g]);
+                    p_s[warp][0][prow][g] = p_hi[g];
+                    p_s[warp][1][prow][g] = p_lo[g];
+                }
+            }
+            if (changed) {                                    // warp-uniform
+                float r0 = 0.0f, r1 = 0.0f;                   // factors of this lane's queries 2 t4, 2 t4 + 1
 #pragma unroll
-                    for (int j = 0; j < NJ; ++j) acc[g][j] = ffma2(acc[g][j], r2, 0ull);
+                for (int g = 0; g < GT; g += 2)
+                    if (t4 == g / 2) {
+                        r0 = resc[g];
+                        r1 = (g + 1 < GT) ? resc[g + 1] : 0.0f;
+                    }
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    acc[mt][0] *= r0;
+                    acc[mt][1] *= r1;
+                    acc[mt][2] *= r0;
+                    acc[mt][3] *= r1;
                 }
             }
             __syncwarp();
 
-            // ---- phase 3: O += p * vhat * 2^-g, lane = (token group, 4 dims) ----
-            const uint8_t* vbase = st + Stage::kVOff + dc * (2 * NJ);
-#pragma unroll 4
-            for (int k = 0; k < TPL; ++k) {
-                const int t = ts + TS * k;
-                const uint32_t vv = *reinterpret_cast<const uint32_t*>(vbase + t * D);
-                unsigned long long v2[NJ];
-                v2[0] = pack_f32x2((float)(int8_t)(vv), (float)(int8_t)(vv >> 8));
-                v2[1] = pack_f32x2((float)(int8_t)(vv >> 16), (float)(int8_t)(vv >> 24));
-                if constexpr (GT % 2 == 0) {
+            // ---- phase 3: O^T += V^T P^T on the tensor cores.  One 8 x 8 block of 16-bit pairs
+            // (8 keys x 16 dims of INT8), transposed by ldmatrix, is the A fragment of one product:
+            // column t of the product is key 2t of the block, column t + 4 is key 2t + 1; row gq is
+            // dim 2 gq, row gq + 8 is dim 2 gq + 1.  The weight rows are stored in the same key order. ----
+            uint32_t bh[4][2], bl[4][2];
 #pragma unroll
-                    for (int g = 0; g < GT; g += 2) {         // two queries' duplicated weights per 128-bit load
-                        const ulonglong2 pp = *reinterpret_cast<const ulonglong2*>(&p_s[warp][t][g]);
+            for (int j = 0; j < 4; ++j) {
+                bh[j][0] = __float_as_uint(p_s[warp][0][8 * j + t4][gq]);
+                bh[j][1] = __float_as_uint(p_s[warp][0][8 * j + 4 + t4][gq]);
+                bl[j][0] = __float_as_uint(p_s[warp][1][8 * j + t4][gq]);
+                bl[j][1] = __float_as_uint(p_s[warp][1][8 * j + 4 + t4][gq]);
+            }
+            const uint32_t vaddr = stage0 + s * Stage::kBytes + Stage::kVOff + lane * D;
 #pragma unroll
-                        for (int j = 0; j < NJ; ++j) {
-                            acc[g][j] = ffma2(v2[j], pp.x, acc[g][j]);
-                            acc[g + 1][j] = ffma2(v2[j], pp.y, acc[g + 1][j]);
-                        }
-                    }
-                } else {
-                    const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&p_s[warp][t][0]);
+            for (int mt = 0; mt < MT; ++mt) {
+                uint32_t x[4];
+                ldmatrix_x4_trans(x, vaddr + mt * 16);
 #pragma unroll
-                    for (int j = 0; j < NJ; ++j) acc[0][j] = ffma2(v2[j], pp, acc[0][j]);
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t a0 = __float_as_uint((float)(int8_t)(x[j]));
+                    const uint32_t a1 = __float_as_uint((float)(int8_t)(x[j] >> 8));
+                    const uint32_t a2 = __float_as_uint((float)(int8_t)(x[j] >> 16));
+                    const uint32_t a3 = __float_as_uint((float)(int8_t)(x[j] >> 24));
+                    mma_tf32_1688(acc[mt], a0, a1, a2, a3, bh[j][0], bh[j][1]);
+                    mma_tf32_1688(acc[mt], a0, a1, a2, a3, bl[j][0], bl[j][1]);
                 }
             }
         }
@@ -325,7 +358,7 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
 
     // ---- merge the four warps of the block, write the block's partial ----
     __syncthreads();                                           // the merge scratch re-uses the stage buffers
-    block_merge_and_store<D, GT, NJ>(a, red_s, M, l, acc, lane, warp, ts, dc, LPT, b, h0, split);
+    block_merge_and_store<D, GT>(a, red_s, M, l, acc, lane, warp, b, h0, split);
 }
 
 }  // namespace sa

@@ -42,31 +42,32 @@ SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2]
     }
 }
 
-// Per-warp states (M, l, O) -> one partial per block.  acc[g][j] holds output dims
-// dc*2*NJ + 2j, dc*2*NJ + 2j + 1 summed over this lane's token group; token groups sit LPT lanes apart.
-template <int D, int GT, int NJ>
+// Per-warp states (M, l, O) -> one partial per block.  acc[mt] is the 16 x 8 tile (dims x queries)
+// of O^T in the accumulator layout of mma.m16n8k8: lane (gq, t4) holds dims 16 mt + 2 gq (c0, c1)
+// and 16 mt + 2 gq + 1 (c2, c3) of queries 2 t4 (c0, c2) and 2 t4 + 1 (c1, c3).
+template <int D, int GT>
 SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], const int (&M)[GT],
-                                float (&l)[GT], unsigned long long (&acc)[GT][NJ], int lane, int warp,
-                                int ts, int dc, int LPT, int b, int h0, int split) {
+                                float (&l)[GT], float (&acc)[D / 16][4], int lane, int warp, int b, int h0,
+                                int split) {
+    const int gq = lane >> 2, t4 = lane & 3;
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         const float lsum = warp_sum_f32(l[g]);
-#pragma unroll
-        for (int j = 0; j < NJ; ++j) {
-            float lo, hi;
-            unpack_f32x2(acc[g][j], &lo, &hi);
-            for (int off = LPT; off < 32; off <<= 1) {
-                lo += __shfl_xor_sync(0xffffffffu, lo, off);
-                hi += __shfl_xor_sync(0xffffffffu, hi, off);
-            }
-            if (ts == 0) {
-                red_s[warp][g][2 + dc * (2 * NJ) + 2 * j] = lo;
-                red_s[warp][g][2 + dc * (2 * NJ) + 2 * j + 1] = hi;
-            }
-        }
         if (lane == 0) {
             red_s[warp][g][0] = __int_as_float(M[g]);
             red_s[warp][g][1] = lsum;
+        }
+    }
+#pragma unroll
+    for (int mt = 0; mt < D / 16; ++mt) {
+        const int dim = 16 * mt + 2 * gq;
+        if (2 * t4 < GT) {
+            red_s[warp][2 * t4][2 + dim] = acc[mt][0];
+            red_s[warp][2 * t4][2 + dim + 1] = acc[mt][2];
+        }
+        if (2 * t4 + 1 < GT) {
+            red_s[warp][2 * t4 + 1][2 + dim] = acc[mt][1];
+            red_s[warp][2 * t4 + 1][2 + dim + 1] = acc[mt][3];
         }
     }
     __syncthreads();
