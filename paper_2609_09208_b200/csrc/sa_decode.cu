@@ -20,45 +20,47 @@
 namespace sa {
 
 // Shared-memory plan of one block (dynamic shared memory, 128-byte aligned):
-//   [4 warps x kStages stage buffers][mbarriers][packed queries][query scales][weights p (also the
-//   scratch for the unpacked queries during the prologue)]; the block-merge scratch re-uses the stage
-//   buffers once every warp has left its tile loop.
+//   [NW warps x kStages stage buffers][mbarriers][packed queries or table][query scales]; the
+//   block-merge scratch re-uses the stage buffers once every warp has left its tile loop.
 template <int D, int KB, bool NIB, int GT>
 struct DecodeSmem {
     static constexpr int NP = (GT + 1) / 2;        // query pairs
     static constexpr bool kTable = (KB == 1 || KB == 2 || KB == 4);   // mantissa codes: table datapath
+    static constexpr int NW = decode_shape(D, KB).warps;
     static constexpr int CH = NIB ? D / 32 : D / 16;
     using Stage = TileStage<CH, true, D>;
     static constexpr int kStageOff = 0;
-    static constexpr int kMbarOff = 4 * kStages * Stage::kBytes;
+    static constexpr int kMbarOff = NW * kStages * Stage::kBytes;
     // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
     // the table of query multiples [D][NP][2^KB] x 8 bytes
     static constexpr int kQpOff = kMbarOff + 128;
-    static constexpr int kQpBytes = kTable ? D * NP * (8 << KB) : D * NP * 4;
+    // (the prologue's scratch for the unpacked queries, D x GT words, uses the same space first)
+    static constexpr int kQpData = kTable ? D * NP * (8 << KB) : D * NP * 4;
+    static constexpr int kQpBytes = kQpData > D * GT * 4 ? kQpData : D * GT * 4;
     static constexpr int kQscaleOff = kQpOff + kQpBytes;
-    static constexpr int kPOff = kQscaleOff + 128;
-    // weights: per warp two tf32 terms x 32 key rows x 8 query columns of FP32
-    static constexpr int kPBytes = (4 * 2 * 32 * 8 * 4 > D * GT * 4) ? 4 * 2 * 32 * 8 * 4 : D * GT * 4;
-    static constexpr int kBytes = kPOff + kPBytes;
-    static constexpr int kBlocksPerSM = kTable ? (KB == 4 ? 3 : 4) : 5;
-    static_assert(4 * GT * (D + 2) * 4 <= 4 * kStages * Stage::kBytes, "merge scratch must fit in the stage buffers");
+    // (The softmax weights of a tile need no space of their own: they overwrite the tile's key
+    // codes in the stage buffer, which are dead by then.)
+    static constexpr int kBytes = kQscaleOff + 128;
+    static constexpr int kBlocksPerSM = decode_shape(D, KB).blocks_per_sm;
+    static_assert(NW * GT * (D + 2) * 4 <= NW * kStages * Stage::kBytes && NW * kStages * 8 <= 128, "merge scratch must fit in the stage buffers");
+    static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
 };
 
 template <int D, int KB, bool NIB, int GT>
-__global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM)) decode_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM)) decode_kernel(DecodeArgs a) {
     // KB = 0: PoT-4 (packed shift datapath); KB = 1, 2, 4: mantissa codes (table datapath);
     // KB = 8: uniform INT8 comparison code (dp4a)
     using SM = DecodeSmem<D, KB, NIB, GT>;
     using Stage = typename SM::Stage;
     constexpr int EPL = D / 32;
     constexpr int NP = SM::NP;
+    constexpr int NW = SM::NW, NT = 32 * NW;       // warps and threads per block
     constexpr int WORDS = NIB ? D / 8 : D / 4;     // 32-bit code words per key
     constexpr int MT = D / 16;                     // 16-dim row tiles of O^T in the A.V phase
     extern __shared__ __align__(128) uint8_t smem[];
     uint32_t (*qp_s)[NP] = reinterpret_cast<uint32_t (*)[NP]>(smem + SM::kQpOff);
     float* qscale_s = reinterpret_cast<float*>(smem + SM::kQscaleOff);
-    float (*p_s)[2][32][8] = reinterpret_cast<float (*)[2][32][8]>(smem + SM::kPOff);   // [warp][term][key row][query]
-    int32_t (*q_s)[GT] = reinterpret_cast<int32_t (*)[GT]>(smem + SM::kPOff);      // prologue only
+    int32_t (*q_s)[GT] = reinterpret_cast<int32_t (*)[GT]>(smem + SM::kQpOff);     // prologue only
     float (*red_s)[GT][D + 2] = reinterpret_cast<float (*)[GT][D + 2]>(smem + SM::kStageOff);
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -87,11 +89,11 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
     const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
     const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
     const int first = tile0 + warp;
-    const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
+    const int n_my = first < tile1 ? (tile1 - first + NW - 1) / NW : 0;
     // Lane 0: start the copies of my i-th tile into stage i % kStages.  A tile whose page is not
     // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
     auto issue = [&](int i) {
-        const int tile = first + 4 * i;
+        const int tile = first + NW * i;
         const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
         const int s = i % kStages;
         if (pidx < 0 || pidx >= a.n_pages) {
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
         for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
 
     // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register ----
-    for (int g = warp; g < GT; g += 4) {
+    for (int g = warp; g < GT; g += NW) {
         uint32_t bits[EPL];
         load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
         int q[EPL];
@@ -123,11 +125,11 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
         // One thread per table entry and pass: consecutive threads write consecutive 8-byte entries
         // (no bank conflicts).  The factor 2^KB + mu is applied by shift-and-add over the bits of mu.
         constexpr int ENT = D * NP * (1 << KB);                // entries of {q_lo, q_hi} * (2^KB + mu)
-        constexpr int PASSES = (ENT + 127) / 128;
+        constexpr int PASSES = (ENT + NT - 1) / NT;
         uint2 ent[PASSES];
 #pragma unroll
         for (int k = 0; k < PASSES; ++k) {
-            const int idx = threadIdx.x + k * 128;             // = (m * NP + p) * 2^KB + mu
+            const int idx = threadIdx.x + k * NT;             // = (m * NP + p) * 2^KB + mu
             const int mu = idx & ((1 << KB) - 1), row = idx >> KB;
             const int m = row / NP, p = row % NP;
             const int qlo = (idx < ENT) ? q_s[m][2 * p] : 0;
@@ -138,48 +140,46 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
                 if (mu & (1 << bit)) { a += (uint32_t)qlo << bit; b += (uint32_t)qhi << bit; }
             ent[k] = make_uint2(a, b);
         }
-        __syncthreads();                                       // q_s is about to be re-used as p_s
+        __syncthreads();                                       // q_s is about to be overwritten
 #pragma unroll
         for (int k = 0; k < PASSES; ++k) {
-            const int idx = threadIdx.x + k * 128;
+            const int idx = threadIdx.x + k * NT;
             if (idx < ENT) reinterpret_cast<uint2*>(tab)[idx] = ent[k];
         }
     } else if constexpr (KB != 8) {
-        uint32_t qp_reg[(D * NP + 127) / 128];
+        uint32_t qp_reg[(D * NP + NT - 1) / NT];
 #pragma unroll
-        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
-            const int idx = threadIdx.x + k * 128;
+        for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
+            const int idx = threadIdx.x + k * NT;
             const int m = idx / NP, p = idx % NP;
             qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
         }
-        __syncthreads();                                       // q_s is about to be re-used as p_s
+        __syncthreads();                                       // q_s is about to be overwritten
 #pragma unroll
-        for (int k = 0; k < (D * NP + 127) / 128; ++k) {
-            const int idx = threadIdx.x + k * 128;
+        for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
+            const int idx = threadIdx.x + k * NT;
             if (idx < D * NP) qp_s[idx / NP][idx % NP] = qp_reg[k];
         }
     } else {
         // four consecutive elements of one query per word, in the byte order of the key words
         uint32_t* q4_s = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
-        uint32_t q4_reg[(D / 4 * GT + 127) / 128];
+        uint32_t q4_reg[(D / 4 * GT + NT - 1) / NT];
 #pragma unroll
-        for (int k = 0; k < (D / 4 * GT + 127) / 128; ++k) {
-            const int idx = threadIdx.x + k * 128;
+        for (int k = 0; k < (D / 4 * GT + NT - 1) / NT; ++k) {
+            const int idx = threadIdx.x + k * NT;
             const int w = idx / GT, g = idx % GT;
             q4_reg[k] = 0u;
             if (idx < D / 4 * GT)
                 q4_reg[k] = (uint32_t)(q_s[4 * w][g] & 0xff) | ((uint32_t)(q_s[4 * w + 1][g] & 0xff) << 8) |
                             ((uint32_t)(q_s[4 * w + 2][g] & 0xff) << 16) | ((uint32_t)(q_s[4 * w + 3][g] & 0xff) << 24);
         }
-        __syncthreads();
+        __syncthreads();                                       // q_s is about to be overwritten
 #pragma unroll
-        for (int k = 0; k < (D / 4 * GT + 127) / 128; ++k) {
-            const int idx = threadIdx.x + k * 128;
+        for (int k = 0; k < (D / 4 * GT + NT - 1) / NT; ++k) {
+            const int idx = threadIdx.x + k * NT;
             if (idx < D / 4 * GT) q4_s[idx] = q4_reg[k];
         }
     }
-    // query columns beyond GT stay zero for the whole kernel (q_s, which shared this space, is no longer read)
-    for (int idx = threadIdx.x; idx < 4 * 2 * 32 * 8; idx += 128) (&p_s[0][0][0][0])[idx] = 0.0f;
     __syncthreads();
 
     int M[GT];
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
     bool failed = false;
 
     for (int i = 0; i < n_my; ++i) {
-        const int tile = first + 4 * i;
+        const int tile = first + NW * i;
         const int s = i % kStages;
         const uint32_t parity = (uint32_t)(i / kStages) & 1u;
         // the decision is made warp-uniform: a lane must never leave the loop alone
@@ -263,8 +263,12 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
             const float s_j = half_bits_to_float(meta & 0xffffu);
             const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
             const float vscale = valid ? pow2i(-g_j) : 0.0f;  // 2^-g_j; g_j in [-10, 30] for written tokens
+            // The weights go where the tile's key codes were (every lane is done with them): row =
+            // key, 8 query columns of FP32.
+            __syncwarp();
+            float (*p_t)[8] = reinterpret_cast<float (*)[8]>(const_cast<uint8_t*>(st));
             bool changed = false;
-            float resc[GT], p_hi[GT], p_lo[GT];
+            float resc[GT];
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 if (a.dbg_scores && valid)
@@ -278,24 +282,11 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
                 M[g] = Mn;
                 const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
                 l[g] = l[g] * resc[g] + p;
-                // weight times 2^-g_j, as two tf32 terms (low 13 mantissa bits zero)
-                const float pv = p * vscale;
-                p_hi[g] = __uint_as_float(__float_as_uint(pv) & 0xffffe000u);
-                p_lo[g] = __uint_as_float(__float_as_uint(pv - p_hi[g]) & 0xffffe000u);
+                p_t[prow][g] = p * vscale;                                          // weight times 2^-g_j
             }
-            if constexpr (GT == 8) {
-                float4* ph = reinterpret_cast<float4*>(&p_s[warp][0][prow][0]);
-                float4* pl = reinterpret_cast<float4*>(&p_s[warp][1][prow][0]);
-                ph[0] = make_float4(p_hi[0], p_hi[1], p_hi[2], p_hi[3]);
-                ph[1] = make_float4(p_hi[4], p_hi[5], p_hi[6], p_hi[7]);
-                pl[0] = make_float4(p_lo[0], p_lo[1], p_lo[2], p_lo[3]);
-                pl[1] = make_float4(p_lo[4], p_lo[5], p_lo[6], p_lo[7]);
-            } else {
+            if constexpr (GT < 8) {
 #pragma unroll
-                for (int g = 0; g < GT; ++g) {
-                    p_s[warp][0][prow][g] = p_hi[g];
-                    p_s[warp][1][prow][g] = p_lo[g];
-                }
+                for (int g = GT; g < 8; ++g) p_t[prow][g] = 0.0f;                   // unused query columns
             }
             if (changed) {                                    // warp-uniform
                 float r0 = 0.0f, r1 = 0.0f;                   // factors of this lane's queries 2 t4, 2 t4 + 1
@@ -318,15 +309,18 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
             // ---- phase 3: O^T += V^T P^T on the tensor cores.  One 8 x 8 block of 16-bit pairs
             // (8 keys x 16 dims of INT8), transposed by ldmatrix, is the A fragment of one product:
             // column t of the product is key 2t of the block, column t + 4 is key 2t + 1; row gq is
-            // dim 2 gq, row gq + 8 is dim 2 gq + 1.  The weight rows are stored in the same key order. ----
+            // dim 2 gq, row gq + 8 is dim 2 gq + 1.  The weight rows are stored in the same key order.
+            // Every weight is split here into two tf32 terms (low 13 mantissa bits zero). ----
             uint32_t bh[4][2], bl[4][2];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                bh[j][0] = __float_as_uint(p_s[warp][0][8 * j + t4][gq]);
-                bh[j][1] = __float_as_uint(p_s[warp][0][8 * j + 4 + t4][gq]);
-                bl[j][0] = __float_as_uint(p_s[warp][1][8 * j + t4][gq]);
-                bl[j][1] = __float_as_uint(p_s[warp][1][8 * j + 4 + t4][gq]);
-            }
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const float pv = p_t[8 * j + 4 * c + t4][gq];
+                    const float hi = __uint_as_float(__float_as_uint(pv) & 0xffffe000u);
+                    bh[j][c] = __float_as_uint(hi);
+                    bl[j][c] = __float_as_uint(pv - hi) & 0xffffe000u;
+                }
             const uint32_t vaddr = stage0 + s * Stage::kBytes + Stage::kVOff + lane * D;
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
@@ -343,7 +337,7 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
                 }
             }
         }
-        __syncwarp();                                         // every lane is done with this stage and with p_s
+        __syncwarp();                                         // every lane is done with this stage
         if (lane == 0 && i + kStages < n_my) {
             fence_proxy_async();
             issue(i + kStages);
@@ -358,7 +352,7 @@ __global__ void __launch_bounds__(128, (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM
 
     // ---- merge the four warps of the block, write the block's partial ----
     __syncthreads();                                           // the merge scratch re-uses the stage buffers
-    block_merge_and_store<D, GT>(a, red_s, M, l, acc, lane, warp, b, h0, split);
+    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, b, h0, split);
 }
 
 }  // namespace sa
@@ -374,7 +368,7 @@ static void launch_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         (void)once;
     }
-    (void)launch_pdl(decode_kernel<D, KB, NIB, GT>, grid, dim3(128), (size_t)bytes, s, a);
+    (void)launch_pdl(decode_kernel<D, KB, NIB, GT>, grid, dim3(32 * DecodeSmem<D, KB, NIB, GT>::NW), (size_t)bytes, s, a);
 }
 
 template <int D, int KB, bool NIB>

@@ -22,17 +22,17 @@ struct DecodeArgs {
     uint32_t one;             // the value 1, opaque to the compiler (adds issued as multiply-add)
 };
 
-// red_s[w][g] = {M (int bits), l, O[D]} of warp w -> the block's partial in the workspace.
-template <int D, int GT>
+// red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace.
+template <int D, int GT, int NW = 4>
 SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], int b, int h0, int split) {
-    for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 128) {
+    for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 32 * NW) {
         const int g = idx / (D + 1), c = idx % (D + 1);       // c = 0: l, c >= 1: O[c - 1]
         int Ms = kMNone;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) Ms = max(Ms, __float_as_int(red_s[w][g][0]));
+        for (int w = 0; w < NW; ++w) Ms = max(Ms, __float_as_int(red_s[w][g][0]));
         float v = 0.0f;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
+        for (int w = 0; w < NW; ++w) {
             const int Mw = __float_as_int(red_s[w][g][0]);
             if (Mw != kMNone) v += red_s[w][g][1 + c] * pow2i_neg(Mw - Ms);
         }
@@ -45,7 +45,7 @@ SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2]
 // Per-warp states (M, l, O) -> one partial per block.  acc[mt] is the 16 x 8 tile (dims x queries)
 // of O^T in the accumulator layout of mma.m16n8k8: lane (gq, t4) holds dims 16 mt + 2 gq (c0, c1)
 // and 16 mt + 2 gq + 1 (c2, c3) of queries 2 t4 (c0, c2) and 2 t4 + 1 (c1, c3).
-template <int D, int GT>
+template <int D, int GT, int NW>
 SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], const int (&M)[GT],
                                 float (&l)[GT], float (&acc)[D / 16][4], int lane, int warp, int b, int h0,
                                 int split) {
@@ -71,7 +71,7 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
         }
     }
     __syncthreads();
-    block_combine_and_store<D, GT>(a, red_s, b, h0, split);
+    block_combine_and_store<D, GT, NW>(a, red_s, b, h0, split);
 }
 
 // One block per (sequence, query head): kMergeGroups groups of D threads each take every

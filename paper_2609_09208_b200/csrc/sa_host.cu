@@ -1,6 +1,10 @@
 // Host side of the C ABI: configuration validation, page layout, split plan, and the
 // host-buffer convenience entry.  No kernels live here.
 #include "sa_common.cuh"
+#include <cmath>
+#ifdef SA_TUNE
+#include <cstdlib>
+#endif
 
 namespace sa {
 
@@ -77,18 +81,48 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
     int GT = 1;
     for (int c = 8; c >= 1; c >>= 1)
         if (p.G % c == 0) { GT = c; break; }
-    // One thread block per (split, KV head x query chunk, sequence).  Aim for a few blocks per
-    // SM; every block should still own at least one 32-key tile per warp.
+    // One thread block per (split, KV head x query chunk, sequence); its warps take the 32-key
+    // tiles of the block's slice in turn.  S is chosen by a small cost model of the
+    // launch, fitted to measured sweeps over S, in units of one tile per warp on a full SM:
+    //   * a block lasts about  r + c_fix  with r between tiles / (warps S) and its ceiling (warps that
+    //     run out of tiles leave their issue slots to the others, but not all of the time), and
+    //     c_fix for the prologue (query quantisation, table) and the block merge;
+    //   * blocks run in waves of 148 x resident-blocks-per-SM; a last wave whose SMs hold only the
+    //     fraction f of that takes 0.1 + 0.9 f of a full wave's time, a single partial wave f^0.2
+    //     (an SM's throughput falls almost in proportion to its resident warps).
+    // The sequence lengths live on the device, so the model uses the cache's capacity.
     const long long units = (long long)batch * p.Hkv * (p.G / GT);
-    const long long target = (long long)kNumSMs * (p.fp16 ? 3 : (p.k == 4 ? 3 : (p.k >= 1 ? 4 : 5)));   // resident blocks per SM of the kernel that will run: one full wave
-    long long S = (target + units - 1) / units;
-    const long long max_tiles = (long long)max_pages * (kPageTokens / 32);
-    long long cap = max_tiles / 4;
+    const KernelShape shape = p.fp16 ? kFp16Shape : decode_shape(p.d, p.int8 ? 8 : p.k);
+    const int bps = shape.blocks_per_sm, nw = shape.warps;
+    const long long slots = (long long)kNumSMs * bps;
+    const long long tiles = (long long)max_pages * (kPageTokens / 32);
+    long long cap = tiles / nw;                     // every warp should own at least one tile
     if (cap < 1) cap = 1;
-    if (S > cap) S = cap;
-    if (S > 512) S = 512;
-    if (S < 1) S = 1;
-    *n_splits = (int)S;
+    if (cap > 512) cap = 512;
+    const double c_fix = 0.5;
+    double best = 0.0;
+    long long best_S = 1;
+    for (long long S = 1; S <= cap; ++S) {
+        const long long blocks = units * S;
+        const double per_warp = (double)tiles / (double)(nw * S);
+        const double block_time = 0.5 * (per_warp + (double)(((tiles + S - 1) / S + nw - 1) / nw)) + c_fix;
+        const long long full = blocks / slots, rest = blocks % slots;
+        double cost = (double)full * block_time;
+        if (rest) {
+            const double fill = (double)((rest + kNumSMs - 1) / kNumSMs) / (double)bps;
+            // behind full waves a partial one overlaps their stragglers; on its own it does not
+            cost += block_time * (full ? 0.1 + 0.9 * fill : pow(fill, 0.2));
+        }
+        if (S == 1 || cost < best * 0.999) {        // ties go to the smaller S (less merge work)
+            best = cost;
+            best_S = S;
+        }
+        if (blocks > 16 * slots) break;             // more waves than this never pay
+    }
+    *n_splits = (int)best_S;
+#ifdef SA_TUNE
+    if (const char* e = getenv("SA_SPLITS")) { long long v = atoll(e); if (v >= 1 && v <= cap) *n_splits = (int)v; }
+#endif
     *gt = GT;
 }
 
