@@ -203,35 +203,74 @@ SA_HD void accumulate_word_nibbles(PackedShift<NP>& pl, uint32_t w, const uint32
 // accumulation in one instruction (the multiplier only ever sees +1 or -1: magnitudes are shifted,
 // never multiplied).  The term is at most 127 * 31 * 2^6 < 2^18, the sum of 128 of them fits
 // INT32 (the host checks the bound with the head-room).
+//
+// Per key element, shared by all queries: one byte permute for the shift amount, one for the sign
+// (turned into +1 / -1 on the FMA pipe), and one that drops the mantissa's byte offset into the low
+// byte of the table address — which is why the table of a group of 16 elements starts on a
+// 256-byte boundary and the rest of the address is an immediate.
 // ---------------------------------------------------------------------------------------------
+// Entry {x, y} at (base with its low byte replaced by byte i of offs) + IMM.  The kernel passes a
+// shared-space address, the unit tests on the host a plain pointer.
+template <int IMM>
+SA_HD void table_gather(uint32_t base, uint32_t offs, int i, uint32_t& x, uint32_t& y) {
+#ifdef __CUDA_ARCH__
+    const uint32_t addr = prmt_hd(offs, base, 0x7650u | (uint32_t)i);
+    asm("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(x), "=r"(y) : "r"(addr), "n"(IMM));
+#else
+    (void)base; (void)offs; (void)i;
+    x = y = 0u;                      // shared-space addresses exist on the device only
+#endif
+}
+template <int IMM>
+SA_HD void table_gather(const uint8_t* base, uint32_t offs, int i, uint32_t& x, uint32_t& y) {
+    const uintptr_t addr = (reinterpret_cast<uintptr_t>(base) & ~(uintptr_t)0xff) | ((offs >> (8 * i)) & 0xffu);
+    const uint32_t* e = reinterpret_cast<const uint32_t*>(addr + IMM);
+    x = e[0];
+    y = e[1];
+}
+
 template <int KB, int NGP>
 struct TableScore {
     static constexpr int kRowBytes = 8 << KB;              // one (element, query pair) row
     static constexpr int kElemBytes = NGP * kRowBytes;     // all query pairs of one element
+    static constexpr int kGroupBytes = 16 * kElemBytes;    // 16 elements = 4 code words; a multiple of 256
     uint32_t acc[2 * NGP];
-    SA_HD void begin(uint32_t) {
+    uint32_t one, two;                                     // 1 and 2 as run-time values (FMA-pipe arithmetic)
+    SA_HD void begin(uint32_t one_) {
+        one = one_;
+        two = one_ + one_;
 #pragma unroll
         for (int g = 0; g < 2 * NGP; ++g) acc[g] = 0;
     }
-    // one 32-bit word of the byte container = 4 elements; `tab` = table row of the word's first element
-    SA_HD void accumulate_word(uint32_t w, const uint8_t* tab) {
+    // query pairs GP .. NGP - 1 of one element; IMM = byte offset of the element's rows within the group
+    template <int IMM, int GP, typename Base>
+    SA_HD void element_pairs(Base grp, uint32_t offs, int i, uint32_t r, uint32_t sg) {
+        if constexpr (GP < NGP) {
+            uint32_t x, y;
+            table_gather<IMM + GP * kRowBytes>(grp, offs, i, x, y);
+            acc[2 * GP] = mad_fma(shl_clamp_hd(x, r), sg, acc[2 * GP]);
+            acc[2 * GP + 1] = mad_fma(shl_clamp_hd(y, r), sg, acc[2 * GP + 1]);
+            element_pairs<IMM, GP + 1>(grp, offs, i, r, sg);
+        }
+    }
+    template <int W4, int I, typename Base>
+    SA_HD void elements(uint32_t w, uint32_t rw, uint32_t offs, Base grp) {
+        if constexpr (I < 4) {
+            const uint32_t r = prmt_hd(rw, 0u, 0x4440u | I);
+            const uint32_t sg = mad_fma(prmt_hd(w, 0u, 0x8888u | (0x1111u * I)), two, one);   // sigma: 0 / -1 -> +1 / -1
+            element_pairs<(W4 * 4 + I) * kElemBytes, 0>(grp, offs, I, r, sg);
+            elements<W4, I + 1>(w, rw, offs, grp);
+        }
+    }
+    // One 32-bit word of the byte container = 4 elements: word W4 (0..3) of a group of 16 elements
+    // whose table starts at grp (256-byte aligned).
+    template <int W4, typename Base>
+    SA_HD void accumulate_word(uint32_t w, Base grp) {
         const uint32_t gw = (w >> 4) & 0x07070707u;
         const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;       // shift amounts g - 1; 0xff for the zero code
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);
-            const uint32_t sg = prmt_hd(w, 0u, 0x8888u | (0x1111u * i)) | 1u;   // sigma: +1 or -1
-            // byte offset of the mantissa's entry: mu * 8, mu = the byte's low nibble >> (4 - KB)
-            const int sh = 8 * i + 4 - KB - 3;                           // moves mu to bits 3 .. 3 + KB - 1 (folds after unrolling)
-            const uint32_t off = (sh >= 0 ? (w >> (sh >= 0 ? sh : 0)) : (w << (sh < 0 ? -sh : 0))) & (((1u << KB) - 1u) << 3);
-            const uint8_t* row = tab + i * kElemBytes + off;
-#pragma unroll
-            for (int gp = 0; gp < NGP; ++gp) {
-                const uint2 u = *reinterpret_cast<const uint2*>(row + gp * kRowBytes);
-                acc[2 * gp] = mad_fma(shl_clamp_hd(u.x, r), sg, acc[2 * gp]);
-                acc[2 * gp + 1] = mad_fma(shl_clamp_hd(u.y, r), sg, acc[2 * gp + 1]);
-            }
-        }
+        // byte offsets mu * 8 of the mantissas' entries (mu = the byte's low nibble >> (4 - KB))
+        const uint32_t offs = KB == 4 ? (w << 3) & 0x78787878u : KB == 2 ? (w << 1) & 0x18181818u : w & 0x08080808u;
+        elements<W4, 0>(w, rw, offs, grp);
     }
     SA_HD int32_t score(int g) const { return (int32_t)acc[g]; }
 };

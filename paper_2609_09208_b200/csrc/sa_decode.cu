@@ -33,7 +33,7 @@ struct DecodeSmem {
     static constexpr int kMbarOff = NW * kStages * Stage::kBytes;
     // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
     // the table of query multiples [D][NP][2^KB] x 8 bytes
-    static constexpr int kQpOff = kMbarOff + 128;
+    static constexpr int kQpOff = (kMbarOff + 128 + 255) & ~255;   // the table datapath wants 256-byte alignment
     // (the prologue's scratch for the unpacked queries, D x GT words, uses the same space first)
     static constexpr int kQpData = kTable ? D * NP * (8 << KB) : D * NP * 4;
     static constexpr int kQpBytes = kQpData > D * GT * 4 ? kQpData : D * GT * 4;
@@ -57,7 +57,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     constexpr int NW = SM::NW, NT = 32 * NW;       // warps and threads per block
     constexpr int WORDS = NIB ? D / 8 : D / 4;     // 32-bit code words per key
     constexpr int MT = D / 16;                     // 16-dim row tiles of O^T in the A.V phase
-    extern __shared__ __align__(128) uint8_t smem[];
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint32_t (*qp_s)[NP] = reinterpret_cast<uint32_t (*)[NP]>(smem + SM::kQpOff);
     float* qscale_s = reinterpret_cast<float*>(smem + SM::kQscaleOff);
     int32_t (*q_s)[GT] = reinterpret_cast<int32_t (*)[GT]>(smem + SM::kQpOff);     // prologue only
@@ -223,12 +223,17 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             const uint32_t* cw = reinterpret_cast<const uint32_t*>(st) + lane * 4;
             if constexpr (SM::kTable) {
                 using TS = TableScore<KB, NP>;
-                const uint8_t* tab = smem + SM::kQpOff;
+                uint32_t grp = smem_addr(smem + SM::kQpOff);    // table of the next 16 elements (256-byte aligned)
                 TS ts;
                 ts.begin(a.one);
-#pragma unroll 4
-                for (int wq = 0; wq < WORDS; ++wq)
-                    ts.accumulate_word(cw[(wq >> 2) * 128 + (wq & 3)], tab + wq * 4 * TS::kElemBytes);
+#pragma unroll 1
+                for (int c = 0; c < WORDS / 4; ++c, grp += TS::kGroupBytes) {
+                    const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                    ts.template accumulate_word<0>(w4.x, grp);
+                    ts.template accumulate_word<1>(w4.y, grp);
+                    ts.template accumulate_word<2>(w4.z, grp);
+                    ts.template accumulate_word<3>(w4.w, grp);
+                }
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)ts.score(g) << a.f_extra);   // exact: the true sum fits INT32
             } else if constexpr (KB != 8) {
@@ -269,6 +274,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             float (*p_t)[8] = reinterpret_cast<float (*)[8]>(const_cast<uint8_t*>(st));
             bool changed = false;
             float resc[GT];
+            float pv[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};        // unused query columns stay zero
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 if (a.dbg_scores && valid)
@@ -282,12 +288,10 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 M[g] = Mn;
                 const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
                 l[g] = l[g] * resc[g] + p;
-                p_t[prow][g] = p * vscale;                                          // weight times 2^-g_j
+                pv[g] = p * vscale;                                                 // weight times 2^-g_j
             }
-            if constexpr (GT < 8) {
-#pragma unroll
-                for (int g = GT; g < 8; ++g) p_t[prow][g] = 0.0f;                   // unused query columns
-            }
+            reinterpret_cast<float4*>(&p_t[prow][0])[0] = make_float4(pv[0], pv[1], pv[2], pv[3]);
+            reinterpret_cast<float4*>(&p_t[prow][0])[1] = make_float4(pv[4], pv[5], pv[6], pv[7]);
             if (changed) {                                    // warp-uniform
                 float r0 = 0.0f, r1 = 0.0f;                   // factors of this lane's queries 2 t4, 2 t4 + 1
 #pragma unroll

@@ -34,16 +34,20 @@ static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool ni
 template <int K>
 static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
     using TS = TableScore<K, 4>;
-    alignas(16) static uint8_t tab[128 * TS::kElemBytes];
+    alignas(256) static uint8_t tab[128 * TS::kElemBytes];
     for (int m = 0; m < d; ++m)
         for (int gp = 0; gp < 4; ++gp)
             fill_table_row<K>(tab + m * TS::kElemBytes + gp * TS::kRowBytes, q8[(2 * gp) * d + m], q8[(2 * gp + 1) * d + m]);
     TS ts;
     ts.begin(1u);
-    for (int m0 = 0; m0 < d; m0 += 4) {
-        uint32_t w = 0;
-        for (int i = 0; i < 4; ++i) w |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * i);
-        ts.accumulate_word(w, tab + m0 * TS::kElemBytes);
+    for (int m0 = 0; m0 < d; m0 += 16) {
+        uint32_t w[4] = {0, 0, 0, 0};
+        for (int i = 0; i < 16; ++i) w[i / 4] |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * (i % 4));
+        const uint8_t* grp = tab + m0 * TS::kElemBytes;
+        ts.template accumulate_word<0>(w[0], grp);
+        ts.template accumulate_word<1>(w[1], grp);
+        ts.template accumulate_word<2>(w[2], grp);
+        ts.template accumulate_word<3>(w[3], grp);
     }
     for (int g = 0; g < 8; ++g) out[g] = ts.score(g);
 }
