@@ -122,29 +122,41 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
         using TS = TableScore<KB, NP>;
         uint8_t* tab = smem + SM::kQpOff;
-        // One thread per table entry and pass: consecutive threads write consecutive 8-byte entries
-        // (no bank conflicts).  The factor 2^KB + mu is applied by shift-and-add over the bits of mu.
-        constexpr int ENT = D * NP * (1 << KB);                // entries of {q_lo, q_hi} * (2^KB + mu)
-        constexpr int PASSES = (ENT + NT - 1) / NT;
-        uint2 ent[PASSES];
+        // One thread per row (element, query pair) and pass; it walks the row's 2^KB entries by
+        // repeated addition of the pair, starting at an entry that depends on its lane so that the
+        // lanes of a half-warp always write different banks, and wraps around once.
+        constexpr int ROWS = D * NP;
+        constexpr int PASSES = (ROWS + NT - 1) / NT;
+        constexpr uint32_t MASK = (1u << KB) - 1u;
+        int qlo[PASSES], qhi[PASSES];
 #pragma unroll
         for (int k = 0; k < PASSES; ++k) {
-            const int idx = threadIdx.x + k * NT;             // = (m * NP + p) * 2^KB + mu
-            const int mu = idx & ((1 << KB) - 1), row = idx >> KB;
+            const int row = threadIdx.x + k * NT;              // = m * NP + p
             const int m = row / NP, p = row % NP;
-            const int qlo = (idx < ENT) ? q_s[m][2 * p] : 0;
-            const int qhi = (idx < ENT && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
-            uint32_t a = (uint32_t)qlo << KB, b = (uint32_t)qhi << KB;
-#pragma unroll
-            for (int bit = 0; bit < KB; ++bit)
-                if (mu & (1 << bit)) { a += (uint32_t)qlo << bit; b += (uint32_t)qhi << bit; }
-            ent[k] = make_uint2(a, b);
+            qlo[k] = (row < ROWS) ? q_s[m][2 * p] : 0;
+            qhi[k] = (row < ROWS && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
         }
         __syncthreads();                                       // q_s is about to be overwritten
+        const uint32_t mu0 = ((uint32_t)lane >> (4 - KB)) & MASK;
 #pragma unroll
         for (int k = 0; k < PASSES; ++k) {
-            const int idx = threadIdx.x + k * NT;
-            if (idx < ENT) reinterpret_cast<uint2*>(tab)[idx] = ent[k];
+            const int row = threadIdx.x + k * NT;
+            if (row < ROWS) {
+                uint2* dst = reinterpret_cast<uint2*>(tab + (size_t)row * TS::kRowBytes);
+                const uint32_t lo = (uint32_t)qlo[k], hi = (uint32_t)qhi[k];
+                uint32_t x = lo << KB, y = hi << KB;           // entry mu0: (2^KB + mu0) times the pair, by shift-and-add
+#pragma unroll
+                for (int bit = 0; bit < KB; ++bit)
+                    if (mu0 & (1u << bit)) { x += lo << bit; y += hi << bit; }
+#pragma unroll
+                for (uint32_t st = 0; st <= MASK; ++st) {
+                    const uint32_t mu = (mu0 + st) & MASK;
+                    if (mu == 0u) { x = lo << KB; y = hi << KB; }
+                    dst[mu] = make_uint2(x, y);
+                    x += lo;
+                    y += hi;
+                }
+            }
         }
     } else if constexpr (KB != 8) {
         uint32_t qp_reg[(D * NP + NT - 1) / NT];
