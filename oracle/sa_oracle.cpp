@@ -13,7 +13,9 @@
 //
 // Parity status: every function here is pinned by tests that do not use the oracle
 // to check itself (exhaustive brute force, exact rational arithmetic, closed forms,
-// textbook special cases).  Nothing here is "parity unpinned".
+// textbook special cases).  One exception: ora_attention_shiftav (the paper's
+// non-default shift-based A.V) takes two constants, N and k_max, whose values the paper
+// does not print: its arithmetic is pinned, those two values are "parity unpinned".
 //
 // Plain loops, no SIMD, no blocking, no fusion.  Compile with
 //   g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared -pthread
@@ -453,6 +455,87 @@ void ora_attention_online(const int64_t* A, const float* delta, const uint16_t* 
             for (int m = 0; m < d; ++m) o[m] += p.o[m] * f;
         }
         for (int m = 0; m < d; ++m) O[static_cast<int64_t>(h) * d + m] = (l > 0.0f) ? o[m] / l : 0.0f;
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Log2-quantised attention weights and the shift-based A.V: section II-E, eq. (6) and
+// eq. (7) — the paper's non-default option ("both products multiplier-free").
+//
+//   M      = ceil(max_j z_j)                      (integer, log2 domain, z = logit * log2 e)
+//   k_j    = round(M - z_j) >= 0,  weight 2^-k_j                                   eq. (6)
+//   g_ref  = min_j g_j                            (value scales 2^-g_j, INT8 values vhat_j)
+//   O      = 2^(-N - g_ref) * sum_{j : k_j <= k_max} vhat_j << (N - k_j + g_ref - g_j)   eq. (7)
+//            divided by the sum of the kept weights, sum_{j : k_j <= k_max} 2^-k_j.
+//
+// Readings (the paper gives neither N nor k_max, and writes eq. (7) without the
+// normaliser and without saying what a negative shift index means):
+//   * k_j is evaluated as M - round(z_j): for an integer M and round-half-to-even this is
+//     the same number, and it makes the decision independent of M.  The rounding is an
+//     integer decision taken on a floating-point logit, so the logit is formed in binary32
+//     in one fixed order:  z_j = (float(A_j) (x) (Delta (x) c)) (x) s_j  with
+//     c = binary32(log2(e) / sqrt(d) / 2^F) and (x) the binary32 product; it is clamped to
+//     +-1e8 before ceil / round (as for the running maximum of the default path).
+//   * M and g_ref are those of the whole key range (the definition; a streaming kernel's
+//     running values converge to them).
+//   * a key with k_j > k_max is dropped from numerator and normaliser alike (its weight is
+//     below 2^-k_max); a key whose shift index N - k_j + g_ref - g_j is negative is dropped
+//     from the numerator only (its value is below one unit 2^(-N - g_ref) of the accumulator).
+//   * N and k_max are inputs; 0 <= k_max <= N.
+// Everything after the rounding is exact integer arithmetic here (int64 numerator in units
+// of 2^(-N - g_ref), int64 normaliser in units of 2^-N); the final division is fp64.
+// Parity: the arithmetic is pinned (rational sums, softmax of the rounded logits, hand
+// cases for both drop rules); the VALUES of N and k_max are not the paper's — "parity
+// unpinned" for those two constants.
+// A [Hq, T]; delta [Hq]; scales [T, Hkv] binary16 bits; vhat [T, Hkv, d]; g [T, Hkv];
+// O [Hq, d]; zr_out (optional) [Hq, T] rounded logits; M_out (optional) [Hq].
+// ---------------------------------------------------------------------------------
+void ora_attention_shiftav(const int64_t* A, const float* delta, const uint16_t* scales,
+                           const int8_t* vhat, const int8_t* g, int64_t T, int Hq, int Hkv,
+                           int d, int F, int N, int k_max, double* O, int32_t* zr_out,
+                           int32_t* M_out) {
+    const int G = Hq / Hkv;
+    const float c = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(d)) /
+                                       static_cast<double>(1LL << F));
+    std::vector<int32_t> zr(static_cast<size_t>(T));
+    std::vector<int64_t> num(static_cast<size_t>(d));
+    for (int h = 0; h < Hq; ++h) {
+        const int kv = h / G;
+        double* out = O + static_cast<int64_t>(h) * d;
+        for (int m = 0; m < d; ++m) out[m] = 0.0;
+        if (M_out) M_out[h] = 0;
+        if (T == 0) continue;
+        const float qscale = delta[h] * c;                       // binary32 product
+        int32_t M = INT32_MIN;
+        int g_ref = INT32_MAX;
+        for (int64_t t = 0; t < T; ++t) {
+            const float s_j = static_cast<float>(half_bits_to_double(scales[t * Hkv + kv]));
+            float z = static_cast<float>(A[static_cast<int64_t>(h) * T + t]);   // int -> binary32, nearest-even
+            z = z * qscale;
+            z = z * s_j;
+            z = std::fmin(std::fmax(z, -1.0e8f), 1.0e8f);
+            const int32_t up = static_cast<int32_t>(std::ceil(z));
+            zr[t] = static_cast<int32_t>(std::nearbyintf(z));    // round half to even
+            if (up > M) M = up;
+            const int gj = g[t * Hkv + kv];
+            if (gj < g_ref) g_ref = gj;
+            if (zr_out) zr_out[static_cast<int64_t>(h) * T + t] = zr[t];
+        }
+        if (M_out) M_out[h] = M;
+        int64_t norm = 0;                                        // units of 2^-N
+        for (int m = 0; m < d; ++m) num[m] = 0;                  // units of 2^(-N - g_ref)
+        for (int64_t t = 0; t < T; ++t) {
+            const int64_t k = static_cast<int64_t>(M) - zr[t];  // >= 0 because ceil >= round
+            if (k > k_max) continue;
+            norm += int64_t{1} << (N - k);
+            const int64_t sh = N - k + g_ref - g[t * Hkv + kv];
+            if (sh < 0) continue;
+            const int8_t* vr = vhat + (t * Hkv + kv) * d;
+            for (int m = 0; m < d; ++m) num[m] += static_cast<int64_t>(vr[m]) * (int64_t{1} << sh);
+        }
+        if (norm == 0) continue;
+        for (int m = 0; m < d; ++m)
+            out[m] = std::ldexp(static_cast<double>(num[m]), -g_ref) / static_cast<double>(norm);
     }
 }
 

@@ -157,6 +157,26 @@ def attention_online(A, delta, scales, vhat, g, F: int, tile: int = 128, splits:
     return O
 
 
+def attention_shiftav(A, delta, scales, vhat, g, F: int, N: int, k_max: int):
+    """Eq. (6), (7): log2-quantised weights and shift-based A.V.  Returns (O float64 [Hq, d],
+    zr int32 [Hq, T] rounded binary32 logits, M int32 [Hq])."""
+    A = np.ascontiguousarray(A, dtype=np.int64)
+    delta = np.ascontiguousarray(delta, dtype=np.float32)
+    sb = _half_bits(scales)
+    vhat = np.ascontiguousarray(vhat, dtype=np.int8)
+    g = np.ascontiguousarray(g, dtype=np.int8)
+    Hq, T = A.shape
+    T2, Hkv, d = vhat.shape
+    assert T == T2 and 0 <= k_max <= N <= 40
+    O = np.empty((Hq, d), dtype=np.float64)
+    zr = np.empty((Hq, max(T, 1)), dtype=np.int32)
+    M = np.empty(Hq, dtype=np.int32)
+    lib().ora_attention_shiftav(_p(A), _p(delta), _p(sb), _p(vhat), _p(g), C.c_int64(T), C.c_int(Hq),
+                                C.c_int(Hkv), C.c_int(d), C.c_int(F), C.c_int(N), C.c_int(k_max), _p(O),
+                                _p(zr), _p(M))
+    return O, zr[:, :T], M
+
+
 def sdpa_fp16(Q, K, V):
     """Q [Hq, d], K/V [T, Hkv, d] float16 -> O [Hq, d] float64."""
     qb, kb, vb = _half_bits(Q), _half_bits(K), _half_bits(V)

@@ -432,6 +432,90 @@ def test_softmax_special_cases():
     assert not ora.attention_online(A[:, :0], delta, scales[:0], vhat[:0], g[:0], F).any()
 
 
+# ------------------------------------------------------------------ eq. (6), (7): log2 weights, shift A.V
+def test_shiftav_rounded_logits_and_integer_maximum():
+    """The rounded logits are the nearest integers of the logit (formed in binary32, so compared
+    with the fp64 logit up to binary32 rounding), M is the ceiling of the largest one, k >= 0 and
+    the best key has k in {0, 1}."""
+    A, delta, scales, vhat, g, F = _attention_inputs(50, T=300)
+    Hq, T = A.shape
+    Hkv, d = vhat.shape[1], vhat.shape[2]
+    _, zr, M = ora.attention_shiftav(A, delta, scales, vhat, g, F, 15, 15)
+    for h in range(Hq):
+        kv = h // (Hq // Hkv)
+        z = A[h] * float(delta[h]) * scales[:, kv].astype(np.float64) / 2 ** F / math.sqrt(d) * math.log2(math.e)
+        tol = 1e-5 * (1 + np.abs(z))
+        assert np.all(np.abs(zr[h] - z) <= 0.5 + tol)
+        assert M[h] >= z.max() - tol.max() and M[h] < z.max() + 1 + tol.max()
+        k = M[h] - zr[h]
+        assert k.min() in (0, 1) and np.all(k >= 0)
+
+
+def test_shiftav_equals_exact_rational_softmax_of_rounded_logits():
+    """With N and k_max large enough that nothing is dropped, eq. (7) over eq. (6) is the softmax in
+    base 2 of the ROUNDED logits applied to the dequantised values: checked with exact rationals and
+    against the library softmax."""
+    from scipy.special import softmax
+    A, delta, scales, vhat, g, F = _attention_inputs(51, T=60)
+    Hq, T = A.shape
+    Hkv, d = vhat.shape[1], vhat.shape[2]
+    O, zr, M = ora.attention_shiftav(A, delta, scales, vhat, g, F, 40, 40)
+    assert int((M[:, None] - zr).max()) + int(g.max()) - int(g.min()) <= 40       # nothing is dropped
+    for h in range(Hq):
+        kv = h // (Hq // Hkv)
+        w = [Fraction(2) ** int(zr[h, t]) for t in range(T)]
+        den = sum(w)
+        for m in range(0, d, 7):
+            num = sum(w[t] * int(vhat[t, kv, m]) * Fraction(2) ** (-int(g[t, kv])) for t in range(T))
+            assert abs(float(num / den) - O[h, m]) <= 1e-12 * max(1.0, abs(O[h, m]))
+        wl = softmax(zr[h].astype(np.float64) * math.log(2.0))
+        want = wl @ (vhat[:, kv].astype(np.float64) * 2.0 ** (-g[:, kv, None].astype(np.float64)))
+        assert np.max(np.abs(O[h] - want)) < 1e-11
+
+
+def test_shiftav_hand_cases_for_both_drop_rules():
+    """One head, d = 1, F = 6, three keys with logits 0.2, -3.1, -19.8 (or -2.2): rounded logits
+    0, -3, -20 (-2), M = 1, k = 1, 4, 21 (3).  Worked by hand:
+      k_max = 15 drops the third key everywhere:  O = (10*2^14 - 20*2^11) / (2^14 + 2^11) * 2^-2 = 5/3;
+      g = (0, 0, 20) makes the third key's shift index 15 - 3 + 0 - 20 < 0: it leaves the numerator but
+      stays in the normaliser:  O = (10*2^14 - 20*2^11) / (2^14 + 2^11 + 2^12) = 60/11."""
+    c = math.log2(math.e) / 64.0
+    delta = np.array([1.0], dtype=np.float32)
+    scales = np.ones((3, 1), dtype=np.float16)
+    vhat = np.array([10, -20, 99], dtype=np.int8).reshape(3, 1, 1)
+    A = np.array([[round(0.2 / c), round(-3.1 / c), round(-19.8 / c)]], dtype=np.int64)
+    O, zr, M = ora.attention_shiftav(A, delta, scales, vhat, np.array([[2], [2], [5]], dtype=np.int8), 6, 15, 15)
+    assert zr.tolist() == [[0, -3, -20]] and M.tolist() == [1]
+    assert abs(O[0, 0] - 5.0 / 3.0) < 1e-12
+    A[0, 2] = round(-2.2 / c)
+    O, zr, M = ora.attention_shiftav(A, delta, scales, vhat, np.array([[0], [0], [20]], dtype=np.int8), 6, 15, 15)
+    assert zr.tolist() == [[0, -3, -2]] and M.tolist() == [1]
+    assert abs(O[0, 0] - 60.0 / 11.0) < 1e-12
+    # with room for the small value (N = 24) the third key comes back: 99 * 2^-20 * 2^-3 joins the numerator
+    O, _, _ = ora.attention_shiftav(A, delta, scales, vhat, np.array([[0], [0], [20]], dtype=np.int8), 6, 24, 24)
+    want = (10 * 2.0 ** -1 - 20 * 2.0 ** -4 + 99 * 2.0 ** -23) / (2.0 ** -1 + 2.0 ** -4 + 2.0 ** -3)
+    assert abs(O[0, 0] - want) < 1e-12
+
+
+def test_shiftav_special_cases_and_distance_to_the_unquantised_softmax():
+    A, delta, scales, vhat, g, F = _attention_inputs(52, T=64)
+    # one cached key: its dequantised value row, exactly; equal scores: the mean (equal value scales)
+    O1, _, _ = ora.attention_shiftav(A[:, :1], delta, scales[:1], vhat[:1], g[:1], F, 15, 15)
+    for h in range(A.shape[0]):
+        assert np.array_equal(O1[h], vhat[0, h // 4] * 2.0 ** (-float(g[0, h // 4])))
+    g0 = np.zeros_like(g)
+    Oz, _, _ = ora.attention_shiftav(np.zeros_like(A), delta, scales, vhat, g0, F, 15, 15)
+    assert np.max(np.abs(Oz[0] - vhat[:, 0].astype(np.float64).mean(axis=0))) < 1e-12
+    # empty cache
+    assert not ora.attention_shiftav(A[:, :0], delta, scales[:0], vhat[:0], g[:0], F, 15, 15)[0].any()
+    # every weight is within a factor sqrt(2) of the unquantised one, so the output stays near the
+    # two-pass softmax (a second quantisation: the paper reports +0.13 .. +0.15 perplexity for it)
+    Oq, _, _ = ora.attention_shiftav(A, delta, scales, vhat, g, F, 15, 15)
+    Or = ora.attention_twopass(A, delta, scales, vhat, g, F)
+    spread = (vhat.astype(np.float64) * 2.0 ** (-g[..., None].astype(np.float64))).std()
+    assert 0 < np.abs(Oq - Or).mean() < 0.25 * spread
+
+
 # ------------------------------------------------------------------ rotation
 @pytest.mark.parametrize("d", [64, 128])
 def test_hadamard_matches_library_matrix_and_is_an_involution(d):
