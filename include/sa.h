@@ -172,6 +172,27 @@ sa_status sa_decode_attention_fp16(const sa_config* cfg, const sa_cache* cache, 
                                    float* O, void* workspace, size_t workspace_bytes,
                                    sa_stream stream);
 
+/* The paper's non-default option: attention weights quantised to powers of two and the
+ * shift-based A.V (section II-E eq. (6), (7); section V-G), which makes the second product
+ * multiplier-free too:
+ *   M = ceil(max_j z_j), k_j = M - round(z_j) >= 0, weight 2^-k_j;
+ *   O = 2^(-N - g_ref) * sum_{j: k_j <= k_max} vhat_j << (N - k_j + g_ref - g_j), divided by the
+ *   sum of the kept weights; g_ref = min_j g_j.
+ * M and g_ref are those of the whole sequence: the call runs the decode kernel's score phase
+ * (rounded logits to the workspace), a second kernel with a per-tile INT32 accumulator, and the
+ * split-K merge.  A key with k_j > k_max is dropped from numerator and normaliser, one whose
+ * shift index is negative from the numerator only.  The paper prints no values for N (n_bits)
+ * and k_max: 1 <= n_bits <= 18 (INT32 accumulator over a 32-key tile), 0 <= k_max <= n_bits.
+ * Codes: SA_POT4 .. SA_POTM4 (not SA_INT8, not SA_KV_FP16).
+ * workspace: at least sa_shiftav_workspace_bytes, 256-byte aligned, no initialisation needed.
+ * dbg_scores (nullable) as in sa_decode_attention; dbg_rounded (nullable): int32 [batch, n_q_heads,
+ * max_pages_per_seq * 64], receives round(z_j) for every cached key (test hook). */
+sa_status sa_shiftav_workspace_bytes(const sa_config* cfg, int batch, int max_pages_per_seq, size_t* bytes);
+sa_status sa_decode_attention_shiftav(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                                      float* O, void* workspace, size_t workspace_bytes, int n_bits,
+                                      int k_max, int32_t* dbg_scores, int32_t* dbg_rounded,
+                                      sa_stream stream);
+
 /* The two decode entry points with their kernels selectable, for callers that want to time or
  * overlap them separately: stages is a bit mask, 1 = the main kernel (scores, softmax, A.V; writes
  * the split-K partials into the workspace), 2 = the merge of the partials into O.  stages = 3 is

@@ -22,7 +22,7 @@ EXPORTS = [
     "sa_version", "sa_status_string", "sa_get_layout", "sa_workspace_bytes", "sa_encode_keys",
     "sa_quantise_query", "sa_quantise_values", "sa_append_kv", "sa_fill_kv", "sa_decode_attention",
     "sa_decode_attention_fp16", "sa_decode_attention_stages", "sa_decode_attention_fp16_stages", "sa_debug_unpack", "sa_staging_bytes", "sa_decode_step_host",
-    "sa_decode_attention_static", "sa_pipe_microbench",
+    "sa_decode_attention_static", "sa_pipe_microbench", "sa_shiftav_workspace_bytes", "sa_decode_attention_shiftav",
 ]
 
 
@@ -166,6 +166,22 @@ def decode_attention_fp16(cfg, cache: SaCache, Q, O, workspace, stages: int = 3)
                                                    C.c_size_t(workspace.numel() * workspace.element_size()),
                                                    C.c_int(stages), _stream())
     _check(st, "sa_decode_attention_fp16")
+
+
+def shiftav_workspace_bytes(cfg: SaConfig, batch: int, max_pages_per_seq: int) -> int:
+    out = C.c_size_t()
+    _check(lib().sa_shiftav_workspace_bytes(C.byref(cfg), C.c_int(batch), C.c_int(max_pages_per_seq), C.byref(out)),
+           "sa_shiftav_workspace_bytes")
+    return out.value
+
+
+def decode_attention_shiftav(cfg, cache: SaCache, Q, O, workspace, n_bits: int = 15, k_max: int = 15,
+                             dbg_scores=None, dbg_rounded=None):
+    """Log2-quantised weights and shift-based A.V (eq. (6), (7)); workspace of shiftav_workspace_bytes."""
+    _check(lib().sa_decode_attention_shiftav(C.byref(cfg), C.byref(cache), _ptr(Q), _ptr(O), _ptr(workspace),
+                                             C.c_size_t(workspace.numel() * workspace.element_size()),
+                                             C.c_int(n_bits), C.c_int(k_max), _ptr(dbg_scores), _ptr(dbg_rounded),
+                                             _stream()), "sa_decode_attention_shiftav")
 
 
 PIPE_KINDS = ["shl", "lop3", "iadd3", "imad_by_one", "prmt", "shl+imad1", "lop3+imad1", "ffma", "ffma2",

@@ -101,7 +101,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         } else {
             const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
             Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
-                         mbar0 + s * 8);
+                         mbar0 + s * 8, true, a.zr == nullptr);   // the score pass of the shift-A.V option needs no values
         }
     };
     if (lane == 0)
@@ -206,6 +206,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[mt][c] = 0.0f;
+    int g_min = 0x7fffffff;                        // shift-A.V score pass only
     const int gq = lane >> 2, t4 = lane & 3;
     // row of this lane's key in the weight buffer: within a group of 8 keys the even keys come first
     const int prow = (lane & 24) | ((lane & 1) << 2) | ((lane & 7) >> 1);
@@ -280,6 +281,25 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             const float s_j = half_bits_to_float(meta & 0xffffu);
             const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
             const float vscale = valid ? pow2i(-g_j) : 0.0f;  // 2^-g_j; g_j in [-10, 30] for written tokens
+            if (a.zr) {
+                // Score pass of the shift-based A.V option (eq. (6)): store the rounded logits and keep
+                // the ceiling of the largest one and the smallest value exponent; no softmax, no A.V here.
+#pragma unroll
+                for (int g = 0; g < GT; ++g) {
+                    if (a.dbg_scores && valid)
+                        a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
+                    const float z = valid ? fminf(fmaxf((float)A[g] * qscale_s[g] * s_j, -1.0e8f), 1.0e8f) : -1.0e8f;
+                    M[g] = max(M[g], warp_max_s32(__float2int_ru(z)));
+                    if (valid) a.zr[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = __float2int_rn(z);
+                }
+                g_min = min(g_min, valid ? g_j : 0x7fffffff);
+                __syncwarp();
+                if (lane == 0 && i + kStages < n_my) {
+                    fence_proxy_async();
+                    issue(i + kStages);
+                }
+                continue;
+            }
             // The weights go where the tile's key codes were (every lane is done with them): row =
             // key, 8 query columns of FP32.
             __syncwarp();
@@ -366,8 +386,29 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         for (int g = 0; g < GT; ++g) l[g] = __int_as_float(0x7fc00000);
     }
 
-    // ---- merge the four warps of the block, write the block's partial ----
+    // ---- merge the warps of the block, write the block's partial ----
     __syncthreads();                                           // the merge scratch re-uses the stage buffers
+    if (a.zr) {
+        // score pass of the shift-A.V option: the block's statistics instead of a partial
+        int* stat_s = reinterpret_cast<int*>(smem + SM::kStageOff);           // [NW][GT + 1]
+        g_min = warp_min_s32(g_min);
+        if (lane == 0) {
+#pragma unroll
+            for (int g = 0; g < GT; ++g) stat_s[warp * (GT + 1) + g] = failed ? 0x7fffffff : M[g];
+            stat_s[warp * (GT + 1) + GT] = g_min;
+        }
+        __syncthreads();
+        if (threadIdx.x <= GT) {
+            int v = (threadIdx.x < GT) ? kMNone : 0x7fffffff;
+            for (int w = 0; w < NW; ++w) {
+                const int x = stat_s[w * (GT + 1) + threadIdx.x];
+                v = (threadIdx.x < GT) ? max(v, x) : min(v, x);
+            }
+            if (threadIdx.x < GT) a.stat_m[((size_t)split * a.batch + b) * a.Hq + h0 + threadIdx.x] = v;
+            else a.stat_g[((size_t)split * a.batch + b) * gridDim.y + blockIdx.y] = v;
+        }
+        return;
+    }
     block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, b, h0, split);
 }
 
@@ -409,6 +450,15 @@ static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, c
     }
 }
 
+namespace sa {
+// The decode kernel for these arguments (the score pass of the shift-A.V option when a.zr is set).
+void launch_decode_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s) {
+    const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
+    if (p.d == 64) launch_code<64>(p, a, GT, grid, s);
+    else launch_code<128>(p, a, GT, grid, s);
+}
+}  // namespace sa
+
 extern "C" sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_cache* cache,
                                                 const uint16_t* Q, float* O, void* workspace,
                                                 size_t workspace_bytes, int32_t* dbg_scores, int stages,
@@ -429,9 +479,7 @@ extern "C" sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_c
     if (p.int8) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / 127.0);   // key unit = scale / 127
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (stages & 1) {
-        const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
-        if (p.d == 64) launch_code<64>(p, a, GT, grid, s);
-        else launch_code<128>(p, a, GT, grid, s);
+        launch_decode_main(p, a, GT, s);
         if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
     }
     return (stages & 2) ? launch_merge(p, a, s) : SA_OK;

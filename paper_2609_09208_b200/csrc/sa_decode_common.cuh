@@ -20,6 +20,11 @@ struct DecodeArgs {
     size_t page_bytes, kcode_off, meta_off, v_off;
     float zscale;
     uint32_t one;             // the value 1, opaque to the compiler (adds issued as multiply-add)
+    // Shift-based A.V option (eq. (6), (7)); all null / 0 on the default path.
+    int32_t* zr;              // [batch][Hq][dbg_stride] rounded logits, written by the score pass
+    int32_t* stat_m;          // [n_splits][batch][Hq] ceil of the largest logit of the split
+    int32_t* stat_g;          // [n_splits][batch][gridDim.y] smallest value exponent g of the split
+    int n_bits, k_max;        // N and k_max of eq. (7)
 };
 
 // red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace.
@@ -157,6 +162,11 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->v_off = p.lay.v_off;
     a->zscale = 0.0f;
     a->one = 1u;
+    a->zr = nullptr;
+    a->stat_m = nullptr;
+    a->stat_g = nullptr;
+    a->n_bits = 0;
+    a->k_max = 0;
     *gt = GT;
     return SA_OK;
 }

@@ -38,4 +38,10 @@ SA_D int warp_max_s32(int v) {
     return r;
 }
 
+SA_D int warp_min_s32(int v) {
+    int r;
+    asm volatile("redux.sync.min.s32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v));
+    return r;
+}
+
 }  // namespace sa

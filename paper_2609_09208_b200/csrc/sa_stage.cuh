@@ -63,14 +63,17 @@ struct TileStage {
     static constexpr int kBytes = kVOff + kVBytes;            // a multiple of 128
 
     // Issued by one lane.  `block` is the (page, KV head) block, tk0 the tile's first token (0 or 32).
+    // with_codes / with_values: which parts of the tile the caller needs (at least one of them).
     SA_D static void issue(uint32_t dst, const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off,
-                           int tk0, uint32_t mbar) {
-        mbar_arrive_expect_tx(mbar, (uint32_t)kBytes);
+                           int tk0, uint32_t mbar, bool with_codes = true, bool with_values = true) {
+        mbar_arrive_expect_tx(mbar, (uint32_t)((with_codes ? kCodeBytes : 0) + kMetaBytes + (with_values ? kVBytes : 0)));
+        if (with_codes) {
 #pragma unroll
-        for (int c = 0; c < CHUNKS; ++c)
-            bulk_g2s(dst + c * 512, block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+            for (int c = 0; c < CHUNKS; ++c)
+                bulk_g2s(dst + c * 512, block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+        }
         if (HAS_META) bulk_g2s(dst + kMetaOff, block + meta_off + (size_t)tk0 * 4, 128u, mbar);
-        bulk_g2s(dst + kVOff, block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes, mbar);
+        if (with_values) bulk_g2s(dst + kVOff, block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes, mbar);
     }
 };
 

@@ -8,7 +8,8 @@ CUDA events, and prints keys/s and algorithmic GB/s.  Cells:
     T = 32768 for every code, with and without the Hadamard flag, batch 1 / 8 / 32, and the FP16 kernel;
   - ragged paged batch 16, lengths uniform in [2048, 16384], PoT-M2;
   - long-context grid (32 query / 8 KV heads, d = 128): T in {1k, 4k, 16k, 64k, 128k} x batch in {1, 8, 32},
-    PoT-4 / PoT-M1 / PoT-M4.
+    PoT-4 / PoT-M1 / PoT-M4;
+  - the shift-based A.V option (eq. (6), (7)) on the T = 32768 shape for PoT-4 nibble and PoT-M4.
 """
 from __future__ import annotations
 
@@ -25,13 +26,15 @@ def bytes_per_key(d, code, nibble):
 
 
 class Cell:
-    def __init__(self, dev, lens, Hq, Hkv, d, code, nibble=False, hadamard=False, outliers=True, seed=1, min_bytes=400e6):
+    def __init__(self, dev, lens, Hq, Hkv, d, code, nibble=False, hadamard=False, outliers=True, seed=1, min_bytes=400e6,
+                 shiftav=False):
         import torch
         from . import binding as sa
         from . import synth
         self.sa, self.torch = sa, torch
         self.cfg = sa.make_config(d, Hq, Hkv, code, nibble=nibble, hadamard=hadamard and code != 16)
         self.fp16 = code == 16
+        self.shiftav = shiftav                                # eq. (6), (7) option: N = k_max = 15
         lens = np.asarray(lens, dtype=np.int64)
         self.keys = int(lens.sum()) * Hkv
         self.bytes = self.keys * bytes_per_key(d, code, nibble)
@@ -59,12 +62,18 @@ class Cell:
             self.caches.append(cache)
             self.Q.append(torch.randn((len(lens), Hq, d), generator=gen, device=dev, dtype=torch.float32).half())
             self.O.append(torch.zeros((len(lens), Hq, d), dtype=torch.float32, device=dev))
+        if shiftav:
+            raw = torch.empty(sa.shiftav_workspace_bytes(self.cfg, len(lens), self.caches[0].max_pages) + 256,
+                              dtype=torch.uint8, device=dev)
+            self.shift_ws = raw[(-raw.data_ptr()) % 256:]
 
     def run_once(self):
         sa = self.sa
         for c, q, o in zip(self.caches, self.Q, self.O):
             if self.fp16:
                 sa.decode_attention_fp16(self.cfg, c.handle, q, o, c.workspace)
+            elif self.shiftav:
+                sa.decode_attention_shiftav(self.cfg, c.handle, q, o, self.shift_ws, 15, 15)
             else:
                 sa.decode_attention(self.cfg, c.handle, q, o, c.workspace)
 
@@ -109,6 +118,9 @@ def main():
                                (4, False, False), (4, False, True), (8, False, False), (16, False, False)]:
             cell("cfg3 T=32768 B=%d %s%s%s" % (B, names[code], "_nibble" if nib else "", "+hadamard" if had else ""),
                  [32768] * B, 32, 4, 64, code, nibble=nib, hadamard=had, outliers=False)
+        for code, nib in ([] if quick else [(0, True), (4, False)]):
+            cell("cfg3 T=32768 B=%d %s%s shift-based A.V (N = k_max = 15)" % (B, names[code], "_nibble" if nib else ""),
+                 [32768] * B, 32, 4, 64, code, nibble=nib, outliers=False, shiftav=True)
     lens4 = np.random.Generator(np.random.PCG64(4001)).integers(2048, 16385, size=16)
     cell("cfg4 ragged B=16 [2048,16384] potm2", lens4, 32, 4, 64, 2)
     cell("cfg4 ragged B=16 [2048,16384] fp16", lens4, 32, 4, 64, 16)

@@ -121,3 +121,23 @@ def test_entry_points_reject_bad_arguments_before_any_cuda_call():
     assert lib.sa_decode_attention_fp16(C.byref(cfg), C.byref(cache), one, one, one, C.c_size_t(1 << 30), null) == 2
     assert lib.sa_debug_unpack(C.byref(cfg), C.byref(cache), C.c_int(3), C.c_int(1), null, null, null, null, null) == 1
     assert lib.sa_debug_unpack(C.byref(cfg), C.byref(cache), C.c_int(0), C.c_int(4 * 64 + 1), null, null, null, null, null) == 4
+
+
+def test_shiftav_entry_validates_on_the_host():
+    """The shift-based A.V option: workspace = partials + rounded logits + per-split statistics; the
+    constants N and k_max, the code and the workspace are checked before anything is launched."""
+    lib = sa.lib()
+    cfg = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    base, full = sa.workspace_bytes(cfg, 2, 64), sa.shiftav_workspace_bytes(cfg, 2, 64)
+    assert full >= base + 2 * 32 * 64 * 64 * 4               # + int32 rounded logits for every (head, key slot)
+    assert full % 256 == 0
+    for code in (sa.SA_INT8, sa.SA_KV_FP16):
+        assert _status(sa.shiftav_workspace_bytes, sa.make_config(64, 32, 4, code), 2, 64) == 2
+    null, one = C.c_void_p(0), C.c_void_p(256)
+    cache = sa.SaCache(256, 256, 256, 2, 64, 128)
+    big = C.c_size_t(1 << 30)
+    call = lambda n, k, ws=one, nbytes=big: lib.sa_decode_attention_shiftav(
+        C.byref(cfg), C.byref(cache), one, one, ws, nbytes, C.c_int(n), C.c_int(k), null, null, null)
+    assert call(0, 0) == 1 and call(19, 3) == 1 and call(15, 16) == 1 and call(15, -1) == 1
+    assert call(15, 15, one, C.c_size_t(full - 1)) == 4
+    assert call(15, 15, C.c_void_p(256 + 16), big) == 3

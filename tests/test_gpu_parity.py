@@ -404,3 +404,84 @@ def test_int8_decode_matches_oracle(dev, lens, Hq, Hkv, d, hadamard):
         want_c, want_s = ora.encode_keys_int8(ora.hadamard_fp16(K) if hadamard else K)
         codes, scales, _, _ = _unpack(cfg_of(case), cache, b, T, case, dev)
         assert np.array_equal(codes.view(np.int8), want_c) and np.array_equal(scales, want_s.view(np.uint16))
+
+
+# ------------------------------------------------------------------------------- eq. (6), (7): shift-based A.V
+def oracle_shiftav(case, n_bits, k_max, F=0):
+    """The oracle's steps chained per sequence: (rotation,) key codes, query and value quantisers, integer
+    scores, then log2-quantised weights with the shift-based A.V.  Returns O [B, Hq, d] and the rounded
+    logits per sequence."""
+    F = F or E + case.code_k
+    O = np.zeros((case.batch, case.n_q_heads, case.head_dim))
+    rounded = []
+    for b in range(case.batch):
+        t0, t1 = int(case.cu_lens[b]), int(case.cu_lens[b + 1])
+        Q, K, V = case.Q[b], case.K[t0:t1], case.V[t0:t1]
+        if case.hadamard:
+            Q, K = ora.hadamard_fp16(Q), ora.hadamard_fp16(K)
+        codes, scales = ora.encode_keys(K, case.code_k)
+        qhat, delta = ora.quantise_query(Q)
+        vhat, g = ora.quantise_value(V)
+        A, ov = ora.scores(qhat, codes, case.code_k, F)
+        assert ov == 0
+        O[b], zr, _ = ora.attention_shiftav(A, delta, scales, vhat, g, F, n_bits, k_max)
+        rounded.append(zr)
+    return O, rounded
+
+
+@pytest.mark.parametrize("k,nibble,d,Hq,Hkv,hadamard", [
+    (0, False, 64, 32, 4, False), (0, True, 64, 32, 4, True), (1, False, 64, 32, 4, False),
+    (4, False, 64, 32, 4, False), (4, False, 128, 32, 8, False), (2, False, 64, 8, 8, False),
+])
+@pytest.mark.parametrize("n_bits,k_max", [(15, 15), (18, 9)])
+def test_shiftav_matches_oracle(dev, k, nibble, d, Hq, Hkv, hadamard, n_bits, k_max):
+    """Rounded logits bit-exact, O within 1e-3, on a ragged batch with an empty sequence, a ragged tail,
+    several tiles per warp and value rows of very different scales (so that both drop rules fire)."""
+    import torch
+    case = synth.make_case("shiftav", [1500, 0, 33, 2049, 64], Hq, Hkv, d, k, nibble=nibble, hadamard=hadamard,
+                           outliers=True, seed=900 + k + d)
+    rng = np.random.default_rng(5)
+    scale = np.exp2(rng.integers(-9, 3, size=(case.V.shape[0], Hkv, 1))).astype(np.float16)
+    case.V = (case.V * scale).astype(np.float16)             # value exponents g spread over 12 binades
+    cfg, cache = build_cache(case, dev, permute_seed=3)
+    ws = torch.empty(sa.shiftav_workspace_bytes(cfg, case.batch, cache.max_pages) + 256, dtype=torch.uint8, device=dev)
+    ws = ws[(-ws.data_ptr()) % 256:]
+    O = torch.full((case.batch, Hq, d), float("nan"), dtype=torch.float32, device=dev)
+    zr = torch.full((case.batch, Hq, cache.max_pages * 64), -7, dtype=torch.int32, device=dev)
+    sa.decode_attention_shiftav(cfg, cache.handle, t16(case.Q, dev), O, ws, n_bits, k_max, None, zr)
+    torch.cuda.synchronize()
+    want_O, want_zr = oracle_shiftav(case, n_bits, k_max)
+    zr = zr.cpu().numpy()
+    for b in range(case.batch):
+        T = int(case.lens[b])
+        assert np.array_equal(zr[b, :, :T], want_zr[b]), "rounded logits differ (sequence %d)" % b
+        assert np.all(zr[b, :, T:] == -7)
+    got = O.cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.max(np.abs(got - want_O)) <= TOL_O, np.max(np.abs(got - want_O))
+    # same result without the test hook (rounded logits in the workspace)
+    O2 = torch.full_like(O, float("nan"))
+    sa.decode_attention_shiftav(cfg, cache.handle, t16(case.Q, dev), O2, ws, n_bits, k_max)
+    torch.cuda.synchronize()
+    assert torch.equal(O, O2)
+
+
+def test_shiftav_long_sequence_and_host_checks(dev):
+    import torch
+    case = synth.make_case("shiftav_long", [32768], 32, 4, 64, 4, outliers=False, seed=77)
+    cfg, cache = build_cache(case, dev, permute_seed=1)
+    ws = torch.empty(sa.shiftav_workspace_bytes(cfg, 1, cache.max_pages) + 256, dtype=torch.uint8, device=dev)
+    ws = ws[(-ws.data_ptr()) % 256:]
+    O = torch.full((1, 32, 64), float("nan"), dtype=torch.float32, device=dev)
+    sa.decode_attention_shiftav(cfg, cache.handle, t16(case.Q, dev), O, ws, 15, 15)
+    torch.cuda.synchronize()
+    want_O, _ = oracle_shiftav(case, 15, 15)
+    assert np.max(np.abs(O.cpu().numpy() - want_O)) <= TOL_O
+    # a workspace that is too small, or constants outside the supported range, launch nothing
+    O.fill_(7.0)
+    for bad in (dict(ws=ws[:1024], n=15, k=15, status=4), dict(ws=ws, n=19, k=3, status=1), dict(ws=ws, n=15, k=16, status=1)):
+        with pytest.raises(sa.SaError) as err:
+            sa.decode_attention_shiftav(cfg, cache.handle, t16(case.Q, dev), O, bad["ws"], bad["n"], bad["k"])
+        assert err.value.status == bad["status"]
+    torch.cuda.synchronize()
+    assert bool((O == 7.0).all())
