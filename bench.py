@@ -50,6 +50,8 @@ VARIANTS = {
     "pot4": (0, False, False, False),
     "pot4_nibble": (0, True, False, False),
     "pot4_nibble_had": (0, True, True, False),
+    "potm1_planar": (1, True, False, False),  # dense 5-bit container: sign/exponent nibbles + one mantissa bit plane
+    "potm2_planar": (2, True, False, False),  # dense 6-bit container
     "fp16": (0, False, False, True),
     "int8mac": (8, False, False, False),      # uniform INT8 keys, dp4a scores: the paper's multiply-native comparison
 }
@@ -58,7 +60,7 @@ VARIANTS = {
 def bytes_per_key(d, code_k, nibble, fp16):
     if fp16:
         return 4 * d
-    return (d // 2 if nibble else d) + 4 + d
+    return (d // 2 + code_k * d // 8 if nibble else d) + 4 + d      # dense containers: nibbles + k mantissa bit planes
 
 
 class Workload:

@@ -69,8 +69,15 @@ enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_INT8 = 8, SA_KV
  * scale, stored one byte per element in the byte container (132 bytes per key at d = 64, the same
  * as PoT-M4); scores are integer dot products evaluated with dp4a.  Everything else (query and
  * value quantisers, softmax, A.V, merge, cache layout) is shared with the power-of-two codes. */
-/* How key codes are stored in a page. */
-enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1 };
+/* How key codes are stored in a page.
+ * SA_KLAYOUT_BYTE: one byte per element (any code).
+ * SA_KLAYOUT_NIBBLE: SA_POT4 only, two 4-bit codes (sign, exponent) per byte.
+ * SA_KLAYOUT_PLANAR: SA_POTM1 / SA_POTM2 only, the dense 5- and 6-bit form of section II-F (the
+ *   paper's 109-byte PoT-M1 record): the sign/exponent nibbles as in SA_KLAYOUT_NIBBLE, followed at
+ *   kcode_off + 64 * head_dim / 2 by k bit planes of the mantissa, plane b holding head_dim / 8
+ *   bytes per token (bit m % 8 of byte m / 8 = bit b of element m's mantissa), 64 tokens after one
+ *   another.  108 / 116 bytes per key at head_dim = 64 against 132 in the byte container. */
+enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1, SA_KLAYOUT_PLANAR = 2 };
 /* flags */
 #define SA_FLAG_HADAMARD 1u /* rotate Q and K by the normalised Walsh-Hadamard matrix before quantising */
 
@@ -79,7 +86,7 @@ typedef struct {
     int n_q_heads;   /* multiple of n_kv_heads */
     int n_kv_heads;
     int code;        /* SA_POT4 / SA_POTM1 / SA_POTM2 / SA_POTM4, SA_INT8 (comparison), or SA_KV_FP16 (FP16 baseline cache) */
-    int klayout;     /* SA_KLAYOUT_BYTE, or SA_KLAYOUT_NIBBLE (only with SA_POT4) */
+    int klayout;     /* SA_KLAYOUT_BYTE, SA_KLAYOUT_NIBBLE (only with SA_POT4) or SA_KLAYOUT_PLANAR (SA_POTM1 / SA_POTM2) */
     int headroom_F;  /* fixed-point head-room F of eq. (3); 0 selects the default E + k = 6 + k.
                         Must satisfy F >= 6 + k (eq. (4): every shift is a left shift) and
                         head_dim * 127 * (2^(k+1) - 1) * 2^(F - k) < 2^31 (INT32 accumulator) */

@@ -23,10 +23,12 @@ constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no k
 // ---------------------------------------------------------------------------------------------
 struct Plan {
     int d, Hq, Hkv, G, k;     // k = mantissa bits (0 for SA_KV_FP16)
-    bool fp16, nibble, hadamard, int8;   // int8: the uniform INT8 comparison code
+    bool fp16, nibble, hadamard, int8;   // nibble: 4-bit sign/exponent codes (PoT-4 nibble container, or with k = 1, 2
+                                         // the dense planar container); int8: the uniform INT8 comparison code
     int F;                    // head-room actually used
     int f_extra;              // F - (6 + k): applied as one final left shift of the INT32 sum
     sa_layout lay;
+    size_t plane_off;         // dense planar container: offset of the mantissa bit planes inside a block
 };
 
 sa_status make_plan(const sa_config* cfg, Plan* out);

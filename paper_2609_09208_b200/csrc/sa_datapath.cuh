@@ -272,6 +272,37 @@ struct TableScore {
         const uint32_t offs = KB == 4 ? (w << 3) & 0x78787878u : KB == 2 ? (w << 1) & 0x18181818u : w & 0x08080808u;
         elements<W4, 0>(w, rw, offs, grp);
     }
+    // Dense planar container (PoT-M1 / PoT-M2 only): one 32-bit word of sign/exponent nibbles = 8
+    // elements (low nibble = even element), with the elements' mantissa bits in KB separate bit
+    // planes: bit ni of planes[b] is bit b of element ni's mantissa.  W8 = position of the word in
+    // its group of 16 elements (0 or 1).
+    template <int W8, int NI, typename Base>
+    SA_HD void nibble_elements(uint32_t w, uint32_t we, uint32_t re, uint32_t ro, uint32_t offs_e, uint32_t offs_o, Base grp) {
+        if constexpr (NI < 8) {
+            constexpr int byte = NI >> 1;
+            const uint32_t r = prmt_hd((NI & 1) ? ro : re, 0u, 0x4440u | byte);
+            const uint32_t sg = mad_fma(prmt_hd((NI & 1) ? w : we, 0u, 0x8888u | (0x1111u * byte)), two, one);
+            element_pairs<(W8 * 8 + NI) * kElemBytes, 0>(grp, (NI & 1) ? offs_o : offs_e, byte, r, sg);
+            nibble_elements<W8, NI + 1>(w, we, re, ro, offs_e, offs_o, grp);
+        }
+    }
+    template <int W8, typename Base>
+    SA_HD void accumulate_nibble_word(uint32_t w, const uint32_t (&planes)[KB], Base grp) {
+        static_assert(KB == 1 || KB == 2, "the planar container holds PoT-M1 and PoT-M2");
+        const uint32_t ge = w & 0x07070707u, go = (w >> 4) & 0x07070707u;   // g of even / odd elements
+        const uint32_t re = (ge + 0x7f7f7f7fu) ^ 0x80808080u, ro = (go + 0x7f7f7f7fu) ^ 0x80808080u;
+        const uint32_t we = w << 4;                                         // even elements' sign at the byte's top bit
+        // Byte offsets mu * 8 of the table entries, one byte per element: bit 2i of a plane byte goes
+        // to bit 3 + b of byte i.  The product by 0x00208208 places copies of the byte at bit offsets
+        // 3, 9, 15, 21; the mask keeps the wanted copy of each bit (a bit spread, not arithmetic on data).
+        uint32_t offs_e = 0u, offs_o = 0u;
+#pragma unroll
+        for (int b = 0; b < KB; ++b) {
+            offs_e |= (((planes[b] & 0x55u) * 0x00208208u) & 0x08080808u) << b;
+            offs_o |= ((((planes[b] >> 1) & 0x55u) * 0x00208208u) & 0x08080808u) << b;
+        }
+        nibble_elements<W8, 0>(w, we, re, ro, offs_e, offs_o, grp);
+    }
     SA_HD int32_t score(int g) const { return (int32_t)acc[g]; }
 };
 

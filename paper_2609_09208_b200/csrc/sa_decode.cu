@@ -28,7 +28,8 @@ struct DecodeSmem {
     static constexpr bool kTable = (KB == 1 || KB == 2 || KB == 4);   // mantissa codes: table datapath
     static constexpr int NW = decode_shape(D, KB).warps;
     static constexpr int CH = NIB ? D / 32 : D / 16;
-    using Stage = TileStage<CH, true, D>;
+    static constexpr int PLANES = (NIB && kTable) ? KB : 0;           // dense planar container: mantissa bit planes
+    using Stage = TileStage<CH, true, D, PLANES, D / 8>;
     static constexpr int kStageOff = 0;
     static constexpr int kMbarOff = NW * kStages * Stage::kBytes;
     // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
@@ -101,7 +102,8 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         } else {
             const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
             Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
-                         mbar0 + s * 8, true, a.zr == nullptr);   // the score pass of the shift-A.V option needs no values
+                         mbar0 + s * 8, true, a.zr == nullptr,    // the score pass of the shift-A.V option needs no values
+                         a.plane_off);
         }
     };
     if (lane == 0)
@@ -239,13 +241,41 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 uint32_t grp = smem_addr(smem + SM::kQpOff);    // table of the next 16 elements (256-byte aligned)
                 TS ts;
                 ts.begin(a.one);
+                if constexpr (!NIB) {
 #pragma unroll 1
-                for (int c = 0; c < WORDS / 4; ++c, grp += TS::kGroupBytes) {
-                    const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
-                    ts.template accumulate_word<0>(w4.x, grp);
-                    ts.template accumulate_word<1>(w4.y, grp);
-                    ts.template accumulate_word<2>(w4.z, grp);
-                    ts.template accumulate_word<3>(w4.w, grp);
+                    for (int c = 0; c < WORDS / 4; ++c, grp += TS::kGroupBytes) {
+                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        ts.template accumulate_word<0>(w4.x, grp);
+                        ts.template accumulate_word<1>(w4.y, grp);
+                        ts.template accumulate_word<2>(w4.z, grp);
+                        ts.template accumulate_word<3>(w4.w, grp);
+                    }
+                } else {
+                    // dense planar container: 4 nibble words (32 elements) per 16-byte chunk, and per plane one
+                    // 32-bit word of mantissa bits for the same 32 elements
+                    const uint32_t* pw = reinterpret_cast<const uint32_t*>(st + Stage::kPlaneOff) + lane * (D / 32);
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        uint32_t pb[KB];
+#pragma unroll
+                        for (int bit = 0; bit < KB; ++bit) pb[bit] = pw[bit * (Stage::kPlaneBytes / 4) + c];
+                        uint32_t pl[KB];
+#pragma unroll
+                        for (int bit = 0; bit < KB; ++bit) pl[bit] = pb[bit] & 0xffu;
+                        ts.template accumulate_nibble_word<0>(w4.x, pl, grp);
+#pragma unroll
+                        for (int bit = 0; bit < KB; ++bit) pl[bit] = (pb[bit] >> 8) & 0xffu;
+                        ts.template accumulate_nibble_word<1>(w4.y, pl, grp);
+                        grp += TS::kGroupBytes;
+#pragma unroll
+                        for (int bit = 0; bit < KB; ++bit) pl[bit] = (pb[bit] >> 16) & 0xffu;
+                        ts.template accumulate_nibble_word<0>(w4.z, pl, grp);
+#pragma unroll
+                        for (int bit = 0; bit < KB; ++bit) pl[bit] = pb[bit] >> 24;
+                        ts.template accumulate_nibble_word<1>(w4.w, pl, grp);
+                        grp += TS::kGroupBytes;
+                    }
                 }
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)ts.score(g) << a.f_extra);   // exact: the true sum fits INT32
@@ -440,7 +470,12 @@ static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
 
 template <int D>
 static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
-    if (p.nibble) { launch_gt<D, 0, true>(a, GT, grid, s); return; }
+    if (p.nibble) {
+        if (p.k == 0) launch_gt<D, 0, true>(a, GT, grid, s);
+        else if (p.k == 1) launch_gt<D, 1, true>(a, GT, grid, s);       // dense planar container
+        else launch_gt<D, 2, true>(a, GT, grid, s);
+        return;
+    }
     if (p.int8) { launch_gt<D, 8, false>(a, GT, grid, s); return; }
     switch (p.k) {
         case 0: launch_gt<D, 0, false>(a, GT, grid, s); break;

@@ -17,7 +17,7 @@ struct DecodeArgs {
     int32_t* dbg_scores;
     size_t dbg_stride;
     int batch, Hq, Hkv, G, max_pages, n_pages, n_splits, f_extra, hadamard;
-    size_t page_bytes, kcode_off, meta_off, v_off;
+    size_t page_bytes, kcode_off, meta_off, v_off, plane_off;
     float zscale;
     uint32_t one;             // the value 1, opaque to the compiler (adds issued as multiply-add)
     // Shift-based A.V option (eq. (6), (7)); all null / 0 on the default path.
@@ -160,6 +160,7 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->kcode_off = p.lay.kcode_off;
     a->meta_off = p.lay.meta_off;
     a->v_off = p.lay.v_off;
+    a->plane_off = p.plane_off;
     a->zscale = 0.0f;
     a->one = 1u;
     a->zr = nullptr;

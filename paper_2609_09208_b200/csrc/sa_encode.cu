@@ -76,7 +76,7 @@ struct CacheArgs {
     const int32_t* page_table;
     int32_t* seq_lens;
     int batch, max_pages, n_pages, Hkv;
-    size_t page_bytes, kcode_off, meta_off, v_off;
+    size_t page_bytes, kcode_off, meta_off, v_off, plane_off;
     int hadamard;
 };
 
@@ -109,6 +109,25 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
         for (int i = 0; i < EPL / 2; ++i) nb[i] = (uint8_t)((kc[2 * i] >> 4) | (kc[2 * i + 1] & 0xf0));
         const int m = lane * EPL;
         store_bytes<EPL / 2>(kdst + ((size_t)(m >> 5) * kPageTokens + t) * 16 + ((m & 31) >> 1), nb);
+        if constexpr (K > 0 && K < 8) {
+            // dense planar container: mantissa bit b of element m goes to bit m % 8 of byte m / 8 of plane b.
+            // A lane holds EPL consecutive elements, so 8 / EPL lanes share a byte; lane B assembles byte B.
+            constexpr int LPB = 8 / EPL;                      // lanes per plane byte
+#pragma unroll
+            for (int bit = 0; bit < K; ++bit) {
+                uint32_t mask[EPL];
+#pragma unroll
+                for (int i = 0; i < EPL; ++i) mask[i] = __ballot_sync(0xffffffffu, (kc[i] >> (4 - K + bit)) & 1u);
+                if (lane < D / 8) {
+                    uint32_t byte = 0;
+#pragma unroll
+                    for (int l = 0; l < LPB; ++l)
+#pragma unroll
+                        for (int i = 0; i < EPL; ++i) byte |= ((mask[i] >> (LPB * lane + l)) & 1u) << (EPL * l + i);
+                    block[a.plane_off + ((size_t)bit * kPageTokens + t) * (D / 8) + lane] = (uint8_t)byte;
+                }
+            }
+        }
     }
     store_bytes<EPL>(block + a.v_off + (size_t)t * D + lane * EPL, vc);
     if (lane == 0)
@@ -141,13 +160,15 @@ SA_D uint8_t* page_block(const CacheArgs& a, int b, int lp, int h) {
     return a.pages + ((size_t)pidx * a.Hkv + h) * a.page_bytes;
 }
 
-// MODE: 0..4 = power-of-two code with K mantissa bits (byte container), 8 = PoT-4 nibble, 16 = FP16,
-// 32 = uniform INT8 comparison code
+// MODE: 0..4 = power-of-two code with K mantissa bits (byte container), 8 = PoT-4 nibble, 9 / 10 = PoT-M1 /
+// PoT-M2 in the dense planar container, 16 = FP16, 32 = uniform INT8 comparison code
 template <int D, int MODE>
 SA_D void write_token(uint8_t* block, const CacheArgs& a, int t, int lane, const uint16_t* krow,
                       const uint16_t* vrow) {
     if constexpr (MODE == 16) write_token_fp16<D>(block, a, t, lane, krow, vrow);
     else if constexpr (MODE == 8) write_token_quant<D, 0, true>(block, a, t, lane, krow, vrow);
+    else if constexpr (MODE == 9) write_token_quant<D, 1, true>(block, a, t, lane, krow, vrow);
+    else if constexpr (MODE == 10) write_token_quant<D, 2, true>(block, a, t, lane, krow, vrow);
     else if constexpr (MODE == 32) write_token_quant<D, 8, false>(block, a, t, lane, krow, vrow);
     else write_token_quant<D, MODE, false>(block, a, t, lane, krow, vrow);
 }
@@ -190,7 +211,7 @@ __global__ void __launch_bounds__(128) fill_kernel(CacheArgs a, const uint16_t* 
 
 // sa_debug_unpack
 template <int D, bool NIB>
-__global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, uint8_t xor_mask, uint8_t* __restrict__ codes,
+__global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, uint8_t xor_mask, int planes, uint8_t* __restrict__ codes,
                                                      uint16_t* __restrict__ scales, int8_t* __restrict__ vhat,
                                                      int8_t* __restrict__ g) {
     constexpr int EPL = D / 32;
@@ -214,6 +235,12 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
             for (int i = 0; i < EPL / 2; ++i) {
                 c[2 * i] = (uint8_t)((src[i] << 4) ^ 0x70);
                 c[2 * i + 1] = (uint8_t)((src[i] & 0xf0) ^ 0x70);
+            }
+            // dense planar container: the canonical mantissa is left-aligned in the low nibble
+            for (int bit = 0; bit < planes; ++bit) {
+                const uint8_t* pl = block + a.plane_off + ((size_t)bit * kPageTokens + t) * (D / 8);
+#pragma unroll
+                for (int i = 0; i < EPL; ++i) c[i] |= (uint8_t)(((pl[(m + i) >> 3] >> ((m + i) & 7)) & 1u) << (4 - planes + bit));
             }
         }
         store_bytes<EPL>(codes + (size_t)v * D + m, c);
@@ -250,11 +277,12 @@ static sa_status check_cache(const Plan& p, const sa_cache* c, CacheArgs* a) {
     a->kcode_off = p.lay.kcode_off;
     a->meta_off = p.lay.meta_off;
     a->v_off = p.lay.v_off;
+    a->plane_off = p.plane_off;
     a->hadamard = p.hadamard ? 1 : 0;
     return SA_OK;
 }
 
-static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.int8 ? 32 : (p.nibble ? 8 : p.k)); }
+static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.int8 ? 32 : (p.nibble ? 8 + p.k : p.k)); }
 
 #define SA_LAUNCH_CHECK() (cudaGetLastError() == cudaSuccess ? SA_OK : SA_ERR_CUDA)
 
@@ -269,6 +297,8 @@ static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.int8 ? 32 : (p.nibbl
                 case 2: CALL(64, 2); break;                                             \
                 case 4: CALL(64, 4); break;                                             \
                 case 8: CALL(64, 8); break;                                             \
+                case 9: CALL(64, 9); break;                                             \
+                case 10: CALL(64, 10); break;                                           \
                 case 32: CALL(64, 32); break;                                           \
                 default: CALL(64, 16); break;                                           \
             }                                                                           \
@@ -279,6 +309,8 @@ static int mode_of(const Plan& p) { return p.fp16 ? 16 : (p.int8 ? 32 : (p.nibbl
                 case 2: CALL(128, 2); break;                                            \
                 case 4: CALL(128, 4); break;                                            \
                 case 8: CALL(128, 8); break;                                            \
+                case 9: CALL(128, 9); break;                                            \
+                case 10: CALL(128, 10); break;                                          \
                 case 32: CALL(128, 32); break;                                          \
                 default: CALL(128, 16); break;                                          \
             }                                                                           \
@@ -416,12 +448,13 @@ sa_status sa_debug_unpack(const sa_config* cfg, const sa_cache* cache, int b, in
     const unsigned grid = (unsigned)(((int64_t)n_tokens * a.Hkv + 3) / 4);
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const uint8_t xm = p.int8 ? 0x00 : 0x70;
+    const int pl = p.nibble ? p.k : 0;                         // mantissa bit planes of the dense planar container
     if (p.d == 64) {
-        if (p.nibble) unpack_kernel<64, true><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
-        else unpack_kernel<64, false><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
+        if (p.nibble) unpack_kernel<64, true><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, pl, codes, scales, v_hat, g);
+        else unpack_kernel<64, false><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, pl, codes, scales, v_hat, g);
     } else {
-        if (p.nibble) unpack_kernel<128, true><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
-        else unpack_kernel<128, false><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, codes, scales, v_hat, g);
+        if (p.nibble) unpack_kernel<128, true><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, pl, codes, scales, v_hat, g);
+        else unpack_kernel<128, false><<<grid, 128, 0, s>>>(a, b, n_tokens, xm, pl, codes, scales, v_hat, g);
     }
     return SA_LAUNCH_CHECK();
 }

@@ -2,9 +2,6 @@
 // host-buffer convenience entry.  No kernels live here.
 #include "sa_common.cuh"
 #include <cmath>
-#ifdef SA_TUNE
-#include <cstdlib>
-#endif
 
 namespace sa {
 
@@ -57,6 +54,9 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
     if (cfg->klayout == SA_KLAYOUT_NIBBLE) {
         if (p.k != 0) return SA_ERR_UNSUPPORTED;
         p.nibble = true;
+    } else if (cfg->klayout == SA_KLAYOUT_PLANAR) {
+        if (p.k != 1 && p.k != 2) return SA_ERR_UNSUPPORTED;    // 5 and 6 bits per element; 4 and 8 are dense already
+        p.nibble = true;
     } else if (cfg->klayout != SA_KLAYOUT_BYTE) {
         return SA_ERR_UNSUPPORTED;
     }
@@ -69,7 +69,8 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
     p.f_extra = p.F - p.k - kEmax;
     const size_t kbytes = p.nibble ? (size_t)p.d / 2 : (size_t)p.d;
     p.lay.kcode_off = 0;
-    p.lay.meta_off = (size_t)kPageTokens * kbytes;
+    p.plane_off = (size_t)kPageTokens * kbytes;                 // k bit planes of d / 8 bytes per token (planar only)
+    p.lay.meta_off = p.plane_off + (p.nibble ? (size_t)p.k * kPageTokens * (p.d / 8) : 0);
     p.lay.v_off = p.lay.meta_off + (size_t)kPageTokens * 4;
     p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d;
     p.lay.align = 256;
@@ -120,9 +121,6 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
         if (blocks > 16 * slots) break;             // more waves than this never pay
     }
     *n_splits = (int)best_S;
-#ifdef SA_TUNE
-    if (const char* e = getenv("SA_SPLITS")) { long long v = atoll(e); if (v >= 1 && v <= cap) *n_splits = (int)v; }
-#endif
     *gt = GT;
 }
 

@@ -52,25 +52,34 @@ SA_D void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar)
                  : "memory");
 }
 
-// Layout of one stage buffer: [code chunks: CHUNKS x 512 B][metadata: 128 B or none][values: 32 rows].
-template <int CHUNKS, bool HAS_META, int VROW_BYTES>
+// Layout of one stage buffer: [code chunks: CHUNKS x 512 B][mantissa bit planes: PLANES x 32 rows of
+// PLANE_ROW bytes (dense planar container only)][metadata: 128 B or none][values: 32 rows].
+template <int CHUNKS, bool HAS_META, int VROW_BYTES, int PLANES = 0, int PLANE_ROW = 0>
 struct TileStage {
     static constexpr int kCodeBytes = CHUNKS * 512;
-    static constexpr int kMetaOff = kCodeBytes;
+    static constexpr int kPlaneOff = kCodeBytes;
+    static constexpr int kPlaneBytes = 32 * PLANE_ROW;          // one plane of one tile
+    static constexpr int kMetaOff = kPlaneOff + PLANES * kPlaneBytes;
     static constexpr int kMetaBytes = HAS_META ? 128 : 0;
-    static constexpr int kVOff = kCodeBytes + kMetaBytes;
+    static constexpr int kVOff = kMetaOff + kMetaBytes;
     static constexpr int kVBytes = 32 * VROW_BYTES;
     static constexpr int kBytes = kVOff + kVBytes;            // a multiple of 128
 
     // Issued by one lane.  `block` is the (page, KV head) block, tk0 the tile's first token (0 or 32).
     // with_codes / with_values: which parts of the tile the caller needs (at least one of them).
     SA_D static void issue(uint32_t dst, const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off,
-                           int tk0, uint32_t mbar, bool with_codes = true, bool with_values = true) {
-        mbar_arrive_expect_tx(mbar, (uint32_t)((with_codes ? kCodeBytes : 0) + kMetaBytes + (with_values ? kVBytes : 0)));
+                           int tk0, uint32_t mbar, bool with_codes = true, bool with_values = true,
+                           size_t plane_off = 0) {
+        mbar_arrive_expect_tx(mbar, (uint32_t)((with_codes ? kCodeBytes + PLANES * kPlaneBytes : 0) + kMetaBytes +
+                                               (with_values ? kVBytes : 0)));
         if (with_codes) {
 #pragma unroll
             for (int c = 0; c < CHUNKS; ++c)
                 bulk_g2s(dst + c * 512, block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+#pragma unroll
+            for (int b = 0; b < PLANES; ++b)
+                bulk_g2s(dst + kPlaneOff + b * kPlaneBytes, block + plane_off + ((size_t)b * kPageTokens + tk0) * PLANE_ROW,
+                         (uint32_t)kPlaneBytes, mbar);
         }
         if (HAS_META) bulk_g2s(dst + kMetaOff, block + meta_off + (size_t)tk0 * 4, 128u, mbar);
         if (with_values) bulk_g2s(dst + kVOff, block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes, mbar);

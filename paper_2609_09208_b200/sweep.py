@@ -22,7 +22,7 @@ import numpy as np
 def bytes_per_key(d, code, nibble):
     if code == 16:
         return 4 * d
-    return (d // 2 if nibble else d) + 4 + d
+    return (d // 2 + code * d // 8 if nibble else d) + 4 + d         # dense containers: nibbles + k mantissa bit planes
 
 
 class Cell:
@@ -114,9 +114,10 @@ def main():
     cell("cfg1 single head T=1024 pot4", [1024], 1, 1, 64, 0, outliers=False)
     cell("cfg2 llama-1.1B T=4096 potm1 outliers", [4096], 32, 4, 64, 1)
     for B in ([1] if quick else [1, 8, 32]):
-        for code, nib, had in [(0, True, False), (0, True, True), (0, False, False), (1, False, False), (2, False, False),
+        for code, nib, had in [(0, True, False), (0, True, True), (0, False, False), (1, False, False), (1, True, False),
+                               (2, False, False), (2, True, False),
                                (4, False, False), (4, False, True), (8, False, False), (16, False, False)]:
-            cell("cfg3 T=32768 B=%d %s%s%s" % (B, names[code], "_nibble" if nib else "", "+hadamard" if had else ""),
+            cell("cfg3 T=32768 B=%d %s%s%s" % (B, names[code], ("_nibble" if code == 0 else "_planar") if nib else "", "+hadamard" if had else ""),
                  [32768] * B, 32, 4, 64, code, nibble=nib, hadamard=had, outliers=False)
         for code, nib in ([] if quick else [(0, True), (4, False)]):
             cell("cfg3 T=32768 B=%d %s%s shift-based A.V (N = k_max = 15)" % (B, names[code], "_nibble" if nib else ""),

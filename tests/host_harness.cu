@@ -52,7 +52,39 @@ static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t*
     for (int g = 0; g < 8; ++g) out[g] = ts.score(g);
 }
 
+// The same through the dense planar container (k = 1, 2): sign/exponent nibbles, two per byte, and the
+// mantissa bits in k separate bit planes.
+template <int K>
+static void score8_planar(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
+    using TS = TableScore<K, 4>;
+    alignas(256) static uint8_t tab[128 * TS::kElemBytes];
+    for (int m = 0; m < d; ++m)
+        for (int gp = 0; gp < 4; ++gp)
+            fill_table_row<K>(tab + m * TS::kElemBytes + gp * TS::kRowBytes, q8[(2 * gp) * d + m], q8[(2 * gp + 1) * d + m]);
+    TS ts;
+    ts.begin(1u);
+    for (int m0 = 0; m0 < d; m0 += 16) {
+        const uint8_t* grp = tab + m0 * TS::kElemBytes;
+        for (int half = 0; half < 2; ++half) {
+            uint32_t w = 0, planes[K];
+            for (int b = 0; b < K; ++b) planes[b] = 0;
+            for (int i = 0; i < 8; ++i) {
+                const uint8_t phys = canon[m0 + 8 * half + i] ^ 0x70;
+                w |= (uint32_t)(phys >> 4) << (4 * i);
+                for (int b = 0; b < K; ++b) planes[b] |= (uint32_t)((phys >> (4 - K + b)) & 1u) << i;
+            }
+            if (half == 0) ts.template accumulate_nibble_word<0>(w, planes, grp);
+            else ts.template accumulate_nibble_word<1>(w, planes, grp);
+        }
+    }
+    for (int g = 0; g < 8; ++g) out[g] = ts.score(g);
+}
+
 extern "C" {
+void hh_score8_planar(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
+    if (k == 1) score8_planar<1>(canon, q8, d, out);
+    else score8_planar<2>(canon, q8, d, out);
+}
 void hh_score8_table(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
     switch (k) {
         case 1: score8_table<1>(canon, q8, d, out); break;

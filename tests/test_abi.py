@@ -32,7 +32,8 @@ def test_library_exports_every_declared_symbol():
 @pytest.mark.parametrize("d,code,nibble,want", [
     (64, sa.SA_POT4, True, 100), (64, sa.SA_POT4, False, 132), (64, sa.SA_POTM1, False, 132),
     (64, sa.SA_POTM4, False, 132), (128, sa.SA_POT4, True, 196), (128, sa.SA_POTM4, False, 260),
-    (64, sa.SA_KV_FP16, False, 256), (128, sa.SA_KV_FP16, False, 512)])
+    (64, sa.SA_KV_FP16, False, 256), (128, sa.SA_KV_FP16, False, 512),
+    (64, sa.SA_POTM1, True, 108), (64, sa.SA_POTM2, True, 116), (128, sa.SA_POTM1, True, 212), (128, sa.SA_POTM2, True, 228)])
 def test_layout_bytes_per_key(d, code, nibble, want):
     lay = sa.get_layout(sa.make_config(d, 32, 4, code, nibble=nibble))
     assert lay.page_bytes == want * 64
@@ -69,7 +70,13 @@ def test_config_validation():
     assert _status(sa.get_layout, sa.make_config(96, 32, 4, sa.SA_POTM4)) == 2          # head_dim
     assert _status(sa.get_layout, sa.make_config(64, 30, 4, sa.SA_POTM4)) == 1          # Hq % Hkv
     assert _status(sa.get_layout, sa.make_config(64, 32, 4, 3)) == 2                     # no 3-bit mantissa
-    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POTM1, nibble=True)) == 2
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POTM4, nibble=True)) == 2   # 8 bits are dense already
+    wrong = sa.make_config(64, 32, 4, sa.SA_POTM1)
+    wrong.klayout = sa.SA_KLAYOUT_NIBBLE                                                   # nibble container: PoT-4 only
+    assert _status(sa.get_layout, wrong) == 2
+    wrong = sa.make_config(64, 32, 4, sa.SA_POT4)
+    wrong.klayout = sa.SA_KLAYOUT_PLANAR                                                   # planar container: PoT-M1 / M2 only
+    assert _status(sa.get_layout, wrong) == 2
     assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_KV_FP16, hadamard=True)) == 2
     bad = sa.make_config(64, 32, 4, sa.SA_POTM4)
     bad.page_tokens = 32

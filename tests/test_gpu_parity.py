@@ -146,7 +146,8 @@ def _unpack(cfg, cache, b, T, case, dev):
 
 @pytest.mark.parametrize("d,k,nibble,hadamard", [(64, 0, True, False), (64, 0, False, True), (64, 1, False, False),
                                                  (64, 4, False, True), (128, 0, True, False), (128, 2, False, False),
-                                                 (128, 4, False, True)])
+                                                 (128, 4, False, True), (64, 1, True, False), (64, 2, True, True),
+                                                 (128, 1, True, True), (128, 2, True, False)])
 def test_fill_and_unpack_bit_exact(dev, d, k, nibble, hadamard):
     case = synth.make_case("fill", [130, 0, 64, 1, 257], 4, 2, d, k, outliers=True, nibble=nibble,
                            hadamard=hadamard, seed=1300 + d + k)
@@ -164,7 +165,7 @@ def test_fill_and_unpack_bit_exact(dev, d, k, nibble, hadamard):
         assert np.array_equal(vh, want_v) and np.array_equal(g, want_g)
 
 
-@pytest.mark.parametrize("d,k,nibble", [(64, 4, False), (64, 0, True), (128, 1, False)])
+@pytest.mark.parametrize("d,k,nibble", [(64, 4, False), (64, 0, True), (128, 1, False), (64, 1, True), (128, 2, True)])
 def test_append_matches_bulk_fill(dev, d, k, nibble):
     import torch
     lens = np.array([62, 0, 127])
@@ -214,7 +215,8 @@ def test_config2_llama_shape_potm1_outliers(dev):
 
 @pytest.mark.parametrize("k,nibble,hadamard,outliers", [
     (4, False, False, False), (4, False, True, False), (4, False, True, True),
-    (0, False, False, False), (0, True, False, False), (0, True, True, True)])
+    (0, False, False, False), (0, True, False, False), (0, True, True, True),
+    (1, True, False, True), (2, True, True, False)])                 # PoT-M1 / PoT-M2 in the dense planar container
 def test_config3_T32k_full_size(dev, k, nibble, hadamard, outliers):
     case = synth.config3(k, hadamard=hadamard, nibble=nibble, outliers=outliers)
     O, dbg, _ = run_decode(case, dev)
@@ -225,6 +227,17 @@ def test_config4_ragged_paged_batch_potm2(dev):
     case = synth.config4()
     O, dbg, _ = run_decode(case, dev, permute_seed=44)
     check_against_oracle(case, O, dbg)
+
+
+@pytest.mark.parametrize("d,Hq,Hkv,k", [(64, 32, 4, 1), (64, 32, 4, 2), (128, 32, 8, 1), (128, 32, 8, 2), (64, 6, 2, 2)])
+def test_planar_container_ragged_batch(dev, d, Hq, Hkv, k):
+    """PoT-M1 / PoT-M2 in the dense planar container (5 / 6 bits per element): the same integer scores and
+    outputs as the oracle, on a ragged paged batch with an empty sequence and shuffled pages."""
+    case = synth.make_case("planar", [3000, 0, 65, 1, 777], Hq, Hkv, d, k, nibble=True, outliers=True, seed=1700 + d + k)
+    O, dbg, cache = run_decode(case, dev, permute_seed=9)
+    check_against_oracle(case, O, dbg)
+    lay = sa.get_layout(cfg_of(case))
+    assert lay.page_bytes == 64 * (d // 2 + k * d // 8 + 4 + d)
 
 
 @pytest.mark.parametrize("T,B,k", [(1024, 1, 0), (1024, 8, 1), (4096, 8, 4), (16384, 1, 1), (4096, 32, 0)])
@@ -265,7 +278,7 @@ def test_config5_largest_cells_sampled_sequences(dev):
 
 
 @pytest.mark.parametrize("lens", [[0], [1], [31], [32], [33], [63], [64], [65], [127, 0, 129, 1], [4097]])
-@pytest.mark.parametrize("k,nibble", [(0, True), (4, False)])
+@pytest.mark.parametrize("k,nibble", [(0, True), (4, False), (2, True)])
 def test_edge_lengths(dev, lens, k, nibble):
     case = synth.make_case("edge", lens, 8, 2, 64, k, nibble=nibble, seed=1500 + sum(lens) + k)
     O, dbg, _ = run_decode(case, dev, permute_seed=3)
@@ -432,6 +445,7 @@ def oracle_shiftav(case, n_bits, k_max, F=0):
 @pytest.mark.parametrize("k,nibble,d,Hq,Hkv,hadamard", [
     (0, False, 64, 32, 4, False), (0, True, 64, 32, 4, True), (1, False, 64, 32, 4, False),
     (4, False, 64, 32, 4, False), (4, False, 128, 32, 8, False), (2, False, 64, 8, 8, False),
+    (1, True, 64, 32, 4, False),
 ])
 @pytest.mark.parametrize("n_bits,k_max", [(15, 15), (18, 9)])
 def test_shiftav_matches_oracle(dev, k, nibble, d, Hq, Hkv, hadamard, n_bits, k_max):

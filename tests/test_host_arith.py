@@ -105,3 +105,8 @@ def test_score_datapaths_equal_oracle_scores(hh, k, d):
             hh.hh_score8_table(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
                                out.ctypes.data_as(C.c_void_p))
             assert np.array_equal(out.astype(np.int64), want[:, 0]), ("table", trial, out, want[:, 0])
+            if k in (1, 2):
+                # ... and so does the dense planar container (nibbles + mantissa bit planes)
+                hh.hh_score8_planar(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
+                                    out.ctypes.data_as(C.c_void_p))
+                assert np.array_equal(out.astype(np.int64), want[:, 0]), ("planar", trial, out, want[:, 0])
