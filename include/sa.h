@@ -179,6 +179,21 @@ sa_status sa_decode_attention_fp16(const sa_config* cfg, const sa_cache* cache, 
                                    float* O, void* workspace, size_t workspace_bytes,
                                    sa_stream stream);
 
+/* One decode step of a layer in a single pass (section II-F: the cache stores only quantised data,
+ * and the step both extends it and attends over it): equivalent to
+ *   sa_append_kv(cfg, cache, K_new, V_new, 1, stream); sa_decode_attention(cfg, cache, Q, O, ...);
+ * The warp of the decode kernel that owns the new token's 32-key tile encodes and writes the token
+ * before it stages that tile, so the separate append kernel and its launch disappear from the
+ * step; seq_lens[b] is incremented by the split-K merge kernel, after every block has read it.
+ * As with sa_append_kv the token's page must already be mapped; if it is not, the token is not
+ * written, the length stays, and the step attends over the old cache.
+ * With a binary16 cache (SA_KV_FP16), or more than 8 query heads per KV head, the call runs the
+ * two kernels separately.  Same buffers, alignment and workspace as sa_decode_attention;
+ * K_new, V_new [batch, n_kv_heads, head_dim] binary16, 16-byte aligned. */
+sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                         const uint16_t* K_new, const uint16_t* V_new, float* O, void* workspace,
+                         size_t workspace_bytes, sa_stream stream);
+
 /* The paper's non-default option: attention weights quantised to powers of two and the
  * shift-based A.V (section II-E eq. (6), (7); section V-G), which makes the second product
  * multiplier-free too:

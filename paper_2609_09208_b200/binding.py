@@ -23,6 +23,7 @@ EXPORTS = [
     "sa_quantise_query", "sa_quantise_values", "sa_append_kv", "sa_fill_kv", "sa_decode_attention",
     "sa_decode_attention_fp16", "sa_decode_attention_stages", "sa_decode_attention_fp16_stages", "sa_debug_unpack", "sa_staging_bytes", "sa_decode_step_host",
     "sa_decode_attention_static", "sa_pipe_microbench", "sa_shiftav_workspace_bytes", "sa_decode_attention_shiftav",
+    "sa_decode_step",
 ]
 
 
@@ -170,6 +171,13 @@ def decode_attention_fp16(cfg, cache: SaCache, Q, O, workspace, stages: int = 3)
                                                    C.c_size_t(workspace.numel() * workspace.element_size()),
                                                    C.c_int(stages), _stream())
     _check(st, "sa_decode_attention_fp16")
+
+
+def decode_step(cfg, cache: SaCache, Q, K_new, V_new, O, workspace):
+    """Append the step's token and attend over the extended cache in one pass (sa_decode_step)."""
+    _check(lib().sa_decode_step(C.byref(cfg), C.byref(cache), _ptr(Q), _ptr(K_new), _ptr(V_new), _ptr(O),
+                                _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()),
+                                _stream()), "sa_decode_step")
 
 
 def shiftav_workspace_bytes(cfg: SaConfig, batch: int, max_pages_per_seq: int) -> int:

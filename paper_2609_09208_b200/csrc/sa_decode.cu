@@ -11,6 +11,7 @@
 // The four warps' states and then the blocks' partial results are merged with exact
 // power-of-two factors.
 #include "sa_common.cuh"
+#include "sa_cache_write.cuh"
 #include "sa_datapath.cuh"
 #include "sa_decode_common.cuh"
 #include "sa_mma.cuh"
@@ -81,35 +82,11 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         fence_proxy_async();
     }
     __syncwarp();
-    pdl_wait();                 // everything below reads what earlier kernels in the stream wrote
     pdl_launch_dependents();    // the split-K merge may be scheduled as soon as blocks of this grid retire
 
-    // ---- this warp's tiles; start the first copies before the query is quantised ----
-    const int len = a.seq_lens[b];
-    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
-    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
-    const int first = tile0 + warp;
-    const int n_my = first < tile1 ? (tile1 - first + NW - 1) / NW : 0;
-    // Lane 0: start the copies of my i-th tile into stage i % kStages.  A tile whose page is not
-    // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
-    auto issue = [&](int i) {
-        const int tile = first + NW * i;
-        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
-        const int s = i % kStages;
-        if (pidx < 0 || pidx >= a.n_pages) {
-            mbar_arrive(mbar0 + s * 8);
-        } else {
-            const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
-            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
-                         mbar0 + s * 8, true, a.zr == nullptr,    // the score pass of the shift-A.V option needs no values
-                         a.plane_off);
-        }
-    };
-    if (lane == 0)
-        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
-
-    // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register ----
+    // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register.  It reads
+    // only Q, which no kernel of a decode step writes, so it runs BEFORE the wait on the preceding
+    // kernel (the cache append) and overlaps it. ----
     for (int g = warp; g < GT; g += NW) {
         uint32_t bits[EPL];
         load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
@@ -195,6 +172,60 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
     }
     __syncthreads();
+
+    pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
+
+    // ---- this warp's tiles; start the first copies ----
+    int len = a.seq_lens[b];
+    int tile_new = -1, pidx_new = -1;
+    if (a.Knew) {
+        // Fused append: the step's new token goes to position len (if its page is mapped) and is part of
+        // this step's attention.  Every block takes the same decision; the split-K merge kernel bumps
+        // seq_lens once all blocks have read it.
+        const int lp = len / kPageTokens;
+        pidx_new = (len >= 0 && lp < a.max_pages) ? a.page_table[(size_t)b * a.max_pages + lp] : -1;
+        if (pidx_new >= 0 && pidx_new < a.n_pages) {
+            tile_new = len >> 5;
+            len += 1;
+        }
+    }
+    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
+    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
+    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int first = tile0 + warp;
+    const int n_my = first < tile1 ? (tile1 - first + NW - 1) / NW : 0;
+    if (tile_new >= first && tile_new < tile1 && (tile_new - first) % NW == 0) {      // warp-uniform: this warp owns that tile
+        // encode / quantise the token and write it into its page before the tile is copied to shared memory
+        constexpr int MODE = (KB == 8) ? 32 : (NIB ? 8 + KB : KB);
+        CacheArgs ca{};
+        ca.kcode_off = a.kcode_off;
+        ca.meta_off = a.meta_off;
+        ca.v_off = a.v_off;
+        ca.plane_off = a.plane_off;
+        ca.hadamard = a.hadamard;
+        uint8_t* block = const_cast<uint8_t*>(a.pages) + ((size_t)pidx_new * a.Hkv + kvh) * a.page_bytes;
+        const size_t row = ((size_t)b * a.Hkv + kvh) * D;
+        write_token<D, MODE>(block, ca, (len - 1) % kPageTokens, lane, a.Knew + row, a.Vnew + row);
+        fence_proxy_async_global();
+        __syncwarp();
+    }
+    // Lane 0: start the copies of my i-th tile into stage i % kStages.  A tile whose page is not
+    // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
+    auto issue = [&](int i) {
+        const int tile = first + NW * i;
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int s = i % kStages;
+        if (pidx < 0 || pidx >= a.n_pages) {
+            mbar_arrive(mbar0 + s * 8);
+        } else {
+            const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
+                         mbar0 + s * 8, true, a.zr == nullptr,    // the score pass of the shift-A.V option needs no values
+                         a.plane_off);
+        }
+    };
+    if (lane == 0)
+        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
 
     int M[GT];
     float l[GT];
@@ -518,6 +549,37 @@ extern "C" sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_c
         if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
     }
     return (stages & 2) ? launch_merge(p, a, s) : SA_OK;
+}
+
+extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
+                                    const uint16_t* K_new, const uint16_t* V_new, float* O, void* workspace,
+                                    size_t workspace_bytes, sa_stream stream) {
+    Plan p;
+    sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    if (!K_new || !V_new) return SA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(K_new) | reinterpret_cast<uintptr_t>(V_new)) & 15) return SA_ERR_ALIGNMENT;
+    int S, GT;
+    if (cache && cache->batch > 0 && cache->max_pages_per_seq > 0) split_plan(p, cache->batch, cache->max_pages_per_seq, &S, &GT);
+    else GT = 0;
+    if (p.fp16 || GT != p.G) {
+        // binary16 cache, or a query group wider than one block: the separate append kernel
+        st = sa_append_kv(cfg, cache, K_new, V_new, 1, stream);
+        if (st != SA_OK) return st;
+        return p.fp16 ? sa_decode_attention_fp16(cfg, cache, Q, O, workspace, workspace_bytes, stream)
+                      : sa_decode_attention(cfg, cache, Q, O, workspace, workspace_bytes, nullptr, stream);
+    }
+    DecodeArgs a;
+    st = make_decode_args(p, cache, Q, O, workspace, workspace_bytes, &a, &GT);
+    if (st != SA_OK) return st;
+    a.Knew = K_new;
+    a.Vnew = V_new;
+    a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / (double)(1LL << p.F));
+    if (p.int8) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / 127.0);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    launch_decode_main(p, a, GT, s);
+    if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
+    return launch_merge(p, a, s);
 }
 
 extern "C" sa_status sa_decode_attention(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,

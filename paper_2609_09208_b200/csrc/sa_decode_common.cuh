@@ -25,6 +25,9 @@ struct DecodeArgs {
     int32_t* stat_m;          // [n_splits][batch][Hq] ceil of the largest logit of the split
     int32_t* stat_g;          // [n_splits][batch][gridDim.y] smallest value exponent g of the split
     int n_bits, k_max;        // N and k_max of eq. (7)
+    // Fused cache append (sa_decode_step); null on the plain decode path.
+    const uint16_t* Knew;     // [batch][Hkv][D] binary16: the step's new token, written at position seq_lens[b]
+    const uint16_t* Vnew;
 };
 
 // red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace.
@@ -84,14 +87,29 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
 // memory and the result is normalised.
 constexpr int kMergeGroups = 8;
 
+// A sequence's length grows by one when the decode kernel appended the step's token itself (the token's
+// page must be mapped, exactly the condition the decode kernel used).
+struct BumpArgs {
+    int32_t* seq_lens;        // null: no fused append
+    const int32_t* page_table;
+    int max_pages, n_pages, Hq;
+};
+
 template <int D>
 __global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __restrict__ partials,
-                                                                 float* __restrict__ O, int n_splits, int n_rows) {
+                                                                 float* __restrict__ O, int n_splits, int n_rows,
+                                                                 BumpArgs bump) {
     __shared__ int m_s[D * kMergeGroups / 32];
     __shared__ float o_s[kMergeGroups][D + 1];
     pdl_wait();                                               // the partials come from the kernel before
     pdl_launch_dependents();
     const int row = blockIdx.x;                               // b * Hq + h
+    if (bump.seq_lens && threadIdx.x == 0 && row % bump.Hq == 0) {
+        // every block of the decode kernel has read the old length by now
+        const int b = row / bump.Hq, len = bump.seq_lens[b], lp = len / kPageTokens;
+        const int pidx = (len >= 0 && lp < bump.max_pages) ? bump.page_table[(size_t)b * bump.max_pages + lp] : -1;
+        if (pidx >= 0 && pidx < bump.n_pages) bump.seq_lens[b] = len + 1;
+    }
     const int dd = threadIdx.x % D, grp = threadIdx.x / D;
     const size_t stride = (size_t)n_rows * (D + 2);
     const float* base = partials + (size_t)row * (D + 2);
@@ -168,17 +186,20 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->stat_g = nullptr;
     a->n_bits = 0;
     a->k_max = 0;
+    a->Knew = nullptr;
+    a->Vnew = nullptr;
     *gt = GT;
     return SA_OK;
 }
 
 inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s) {
     const int rows = a.batch * a.Hq;
+    BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq};
     cudaError_t err;
     if (p.d == 64) err = launch_pdl(merge_kernel<64>, dim3(rows), dim3(64 * kMergeGroups), 0, s,
-                                    (const float*)a.partials, a.O, a.n_splits, rows);
+                                    (const float*)a.partials, a.O, a.n_splits, rows, bump);
     else err = launch_pdl(merge_kernel<128>, dim3(rows), dim3(128 * kMergeGroups), 0, s,
-                          (const float*)a.partials, a.O, a.n_splits, rows);
+                          (const float*)a.partials, a.O, a.n_splits, rows, bump);
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SA_OK : SA_ERR_CUDA;
 }
 

@@ -208,12 +208,7 @@ sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const
     if (cudaMemcpyAsync(dQ, Q_host, q, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
     if (cudaMemcpyAsync(dK, K_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
     if (cudaMemcpyAsync(dV, V_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
-    st = sa_append_kv(cfg, cache, dK, dV, 1, stream);
-    if (st != SA_OK) return st;
-    if (p.fp16)
-        st = sa_decode_attention_fp16(cfg, cache, dQ, dO, workspace, workspace_bytes, stream);
-    else
-        st = sa_decode_attention(cfg, cache, dQ, dO, workspace, workspace_bytes, nullptr, stream);
+    st = sa_decode_step(cfg, cache, dQ, dK, dV, dO, workspace, workspace_bytes, stream);
     if (st != SA_OK) return st;
     if (cudaMemcpyAsync(O_host, dO, o, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SA_ERR_CUDA;
     return SA_OK;

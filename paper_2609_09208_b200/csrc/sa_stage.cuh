@@ -21,6 +21,8 @@ SA_D void mbar_init(uint32_t mbar, uint32_t count) {
 }
 SA_D void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 SA_D void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// orders this thread's earlier plain global stores before bulk-async copies that read them
+SA_D void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 // one arrival that also announces `bytes` of pending copy traffic
 SA_D void mbar_arrive_expect_tx(uint32_t mbar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");

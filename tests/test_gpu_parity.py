@@ -499,3 +499,53 @@ def test_shiftav_long_sequence_and_host_checks(dev):
         assert err.value.status == bad["status"]
     torch.cuda.synchronize()
     assert bool((O == 7.0).all())
+
+
+# ------------------------------------------------------------------------------- fused decode step
+@pytest.mark.parametrize("d,Hq,Hkv,code,nibble,hadamard", [
+    (64, 32, 4, sa.SA_POTM4, False, False), (64, 32, 4, sa.SA_POT4, True, True), (64, 32, 4, sa.SA_POTM1, True, False),
+    (128, 32, 8, sa.SA_POTM2, False, True), (64, 8, 2, sa.SA_INT8, False, False), (64, 16, 1, sa.SA_POTM4, False, False),
+    (64, 32, 4, sa.SA_KV_FP16, False, False)])
+def test_decode_step_equals_append_then_decode(dev, d, Hq, Hkv, code, nibble, hadamard):
+    """sa_decode_step (the decode kernel writes the step's token itself) against sa_append_kv followed by
+    the decode call, over several consecutive steps: the same cache bytes, the same lengths, bit-identical
+    outputs.  Lengths chosen so that the new token opens a page, opens a 32-key tile, fills a tile, lands
+    in an empty sequence, and in one sequence has no mapped page (no append, length unchanged).
+    16 query heads on one KV head is the case the call serves with the two separate kernels."""
+    import torch
+    lens = np.array([64, 31, 95, 0, 4000, 128], dtype=np.int64)
+    n_steps = 3
+    k = 0 if code in (sa.SA_KV_FP16, sa.SA_INT8) else code
+    full = synth.make_case("step", lens + n_steps, Hq, Hkv, d, k, nibble=nibble, hadamard=hadamard, seed=3100 + d + code)
+    cfg = sa.make_config(d, Hq, Hkv, code, nibble=nibble, hadamard=hadamard)
+    B = len(lens)
+    caches = []
+    for _ in range(2):
+        n_pages = int(np.maximum((lens + n_steps + 63) // 64, 1).sum())
+        c = sa.PagedCache(cfg, lens, dev, extra_tokens=n_steps, permutation=synth.page_permutation(n_pages, 21))
+        pre = np.concatenate([np.arange(full.cu_lens[b], full.cu_lens[b] + lens[b]) for b in range(B)])
+        cu = np.concatenate([[0], np.cumsum(lens)])
+        c.fill(t16(full.K[pre], dev), t16(full.V[pre], dev), cu)
+        c.page_table[5, 2:] = -1                                # sequence 5 (128 tokens): no page for token 128
+        caches.append(c)
+    ref, fused = caches
+    rng = np.random.default_rng(8)
+    for step in range(n_steps):
+        new = np.array([full.cu_lens[b] + lens[b] + step for b in range(B)])
+        Kn, Vn = t16(full.K[new], dev), t16(full.V[new], dev)
+        Q = t16(synth.gaussian_fp16(rng, (B, Hq, d)), dev)
+        O1 = torch.full((B, Hq, d), float("nan"), dtype=torch.float32, device=dev)
+        O2 = torch.full_like(O1, float("nan"))
+        sa.append_kv(cfg, ref.handle, Kn, Vn, True)
+        if code == sa.SA_KV_FP16:
+            sa.decode_attention_fp16(cfg, ref.handle, Q, O1, ref.workspace)
+        else:
+            sa.decode_attention(cfg, ref.handle, Q, O1, ref.workspace)
+        sa.decode_step(cfg, fused.handle, Q, Kn, Vn, O2, fused.workspace)
+        torch.cuda.synchronize()
+        want_lens = lens + step + 1
+        want_lens[5] = 128
+        assert fused.seq_lens.cpu().numpy().tolist() == want_lens.tolist()
+        assert ref.seq_lens.cpu().numpy().tolist() == want_lens.tolist()
+        assert torch.equal(O1, O2), "step %d: outputs differ" % step
+    assert torch.equal(ref.pages, fused.pages)
