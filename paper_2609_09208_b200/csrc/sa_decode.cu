@@ -444,7 +444,10 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         // A bounded wait expired: make the failure visible in the output instead of returning a
         // plausible number (no copy of this warp can still be in flight into a buffer it re-uses).
 #pragma unroll
-        for (int g = 0; g < GT; ++g) l[g] = __int_as_float(0x7fc00000);
+        for (int g = 0; g < GT; ++g) {
+            l[g] = __int_as_float(0x7fc00000);
+            M[g] = max(M[g], 0);                               // a state that "saw no key" would be skipped by the merges
+        }
     }
 
     // ---- merge the warps of the block, write the block's partial ----

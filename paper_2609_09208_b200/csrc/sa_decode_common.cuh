@@ -140,7 +140,8 @@ __global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __
             o += o_s[g][dd];
             l += o_s[g][D];
         }
-        O[(size_t)row * D + dd] = (l > 0.0f) ? o / l : 0.0f;
+        // no key at all: zeros; a poisoned partial (a bounded wait gave up) stays visible as NaN
+        O[(size_t)row * D + dd] = (l == 0.0f) ? 0.0f : o / l;
     }
 }
 

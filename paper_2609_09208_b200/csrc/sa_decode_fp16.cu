@@ -208,7 +208,10 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
             issue(i + kStages);
         }
     }
-    if (failed) l = __int_as_float(0x7fc00000);    // a bounded wait expired: make it visible in the output
+    if (failed) {                                  // a bounded wait expired: make it visible in the output
+        l = __int_as_float(0x7fc00000);
+        M = max(M, 0);                             // a state that "saw no key" would be skipped by the merges
+    }
 
     // ---- per-warp state -> shared memory, merge the four warps, write the block's partial ----
     __syncthreads();                               // the merge scratch re-uses the stage buffers
