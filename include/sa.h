@@ -167,7 +167,11 @@ sa_status sa_fill_kv(const sa_config* cfg, const sa_cache* cache, const uint16_t
  * A sequence with seq_lens[b] == 0 yields zeros.
  * dbg_scores (nullable): int32 [batch, n_q_heads, max_pages_per_seq * 64]; receives A for every
  * cached key (test hook; slows the call down).
- * Results are deterministic run to run (fixed split assignment, no floating-point atomics). */
+ * Results are deterministic run to run (fixed split assignment, no floating-point atomics).
+ * The kernels are launched with programmatic stream serialisation; the decode kernel reads Q
+ * (and nothing else) before it waits for the preceding kernel in the stream, so Q must not be
+ * written by a kernel that signals programmatic launch completion before it has written Q
+ * (ordinary launches, copies and every kernel of this library satisfy that). */
 sa_status sa_decode_attention(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                               float* O, void* workspace, size_t workspace_bytes,
                               int32_t* dbg_scores, sa_stream stream);
