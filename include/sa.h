@@ -290,6 +290,11 @@ sa_status sa_debug_unpack(const sa_config* cfg, const sa_cache* cache, int b, in
  * to every sequence (incrementing seq_lens), runs the decode attention matching cfg->code
  * (quantised or SA_KV_FP16) and copies O [batch, n_q_heads, head_dim] float to O_host.
  * Everything is asynchronous on `stream`; synchronise it before reading O_host.
+ * If all four host buffers are pinned and device-addressable (cudaHostAlloc / cudaHostRegister
+ * memory under unified addressing), no copy engine is used: a small kernel fetches the inputs
+ * and the merge kernel stores O directly into host memory.  Otherwise the buffers are copied
+ * with cudaMemcpyAsync (a single copy for the inputs if Q_host, K_new_host and V_new_host follow
+ * one another in one host buffer and their sizes are multiples of 256 bytes).
  * `staging` is device scratch of at least sa_staging_bytes(); not shared between overlapping calls. */
 sa_status sa_staging_bytes(const sa_config* cfg, int batch, size_t* out);
 sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q_host,

@@ -124,6 +124,18 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
     *gt = GT;
 }
 
+// Inputs of one decode step from device-addressable pinned host memory into the staging buffer.
+__global__ void __launch_bounds__(256) stage_in_kernel(const uint4* __restrict__ q, const uint4* __restrict__ k,
+                                                       const uint4* __restrict__ v, uint4* __restrict__ dq,
+                                                       uint4* __restrict__ dk, uint4* __restrict__ dv, int nq, int nkv) {
+    pdl_wait();                                  // the staging buffer may still be read by the step before
+    pdl_launch_dependents();
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i < nq) dq[i] = q[i];
+    else if (i < nq + nkv) dk[i - nq] = k[i - nq];
+    else if (i < nq + 2 * nkv) dv[i - nq - nkv] = v[i - nq - nkv];
+}
+
 }  // namespace sa
 
 using namespace sa;
@@ -205,9 +217,34 @@ sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const
     uint16_t* dV = reinterpret_cast<uint16_t*>(base + up(q) + up(kv));
     float* dO = reinterpret_cast<float*>(base + up(q) + 2 * up(kv));
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(dQ, Q_host, q, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
-    if (cudaMemcpyAsync(dK, K_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
-    if (cudaMemcpyAsync(dV, V_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+    // Pinned host buffers that the device can address directly need no copy engine at all: a small kernel
+    // fetches the inputs (a few KB) and the merge kernel stores O straight into host memory.  A copy node
+    // costs several microseconds of stream time, which is most of such a step at batch 1.
+    void *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
+    const bool mapped = cudaHostGetDevicePointer(&mq, const_cast<uint16_t*>(Q_host), 0) == cudaSuccess &&
+                        cudaHostGetDevicePointer(&mk, const_cast<uint16_t*>(K_new_host), 0) == cudaSuccess &&
+                        cudaHostGetDevicePointer(&mv, const_cast<uint16_t*>(V_new_host), 0) == cudaSuccess &&
+                        cudaHostGetDevicePointer(&mo, O_host, 0) == cudaSuccess;
+    (void)cudaGetLastError();                                    // a pageable buffer is not an error here
+    auto al16 = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; };
+    if (mapped && al16(mq) && al16(mk) && al16(mv) && al16(mo) && q % 16 == 0 && kv % 16 == 0) {
+        const int nq = (int)(q / 16), nkv = (int)(kv / 16);
+        const unsigned blocks = (unsigned)((nq + 2 * nkv + 255) / 256);
+        if (launch_pdl(stage_in_kernel, dim3(blocks), dim3(256), 0, s, (const uint4*)mq, (const uint4*)mk, (const uint4*)mv,
+                       (uint4*)dQ, (uint4*)dK, (uint4*)dV, nq, nkv) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+            return SA_ERR_CUDA;
+        return sa_decode_step(cfg, cache, dQ, dK, dV, static_cast<float*>(mo), workspace, workspace_bytes, stream);
+    }
+    const char* hq = reinterpret_cast<const char*>(Q_host);
+    if (up(q) == q && up(kv) == kv && reinterpret_cast<const char*>(K_new_host) == hq + q &&
+        reinterpret_cast<const char*>(V_new_host) == hq + q + kv) {
+        // the three inputs follow one another on the host exactly as in the staging buffer: one copy
+        if (cudaMemcpyAsync(dQ, Q_host, q + 2 * kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+    } else {
+        if (cudaMemcpyAsync(dQ, Q_host, q, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+        if (cudaMemcpyAsync(dK, K_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+        if (cudaMemcpyAsync(dV, V_new_host, kv, cudaMemcpyHostToDevice, s) != cudaSuccess) return SA_ERR_CUDA;
+    }
     st = sa_decode_step(cfg, cache, dQ, dK, dV, dO, workspace, workspace_bytes, stream);
     if (st != SA_OK) return st;
     if (cudaMemcpyAsync(O_host, dO, o, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SA_ERR_CUDA;

@@ -357,8 +357,9 @@ def test_fp16_kernel_matches_textbook_attention(dev, d, Hq, Hkv, lens):
 
 
 # ------------------------------------------------------------------------------- host-buffer entry
+@pytest.mark.parametrize("pinned", [True, False])     # pinned: fetched / stored by kernels; pageable: copied
 @pytest.mark.parametrize("code", [sa.SA_POTM4, sa.SA_KV_FP16])
-def test_decode_step_from_host_buffers(dev, code):
+def test_decode_step_from_host_buffers(dev, code, pinned):
     import torch
     lens = np.array([100, 64, 0])
     full = synth.make_case("host", lens + 1, 8, 2, 64, 4, seed=2000)
@@ -367,9 +368,10 @@ def test_decode_step_from_host_buffers(dev, code):
     idx0 = np.concatenate([np.arange(full.cu_lens[b], full.cu_lens[b] + lens[b]) for b in range(3)]).astype(np.int64)
     cache.fill(t16(full.K[idx0], dev), t16(full.V[idx0], dev), np.concatenate([[0], np.cumsum(lens)]))
     last = np.array([full.cu_lens[b + 1] - 1 for b in range(3)])
-    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).pin_memory()
+    pin = lambda x: (lambda t: t.pin_memory() if pinned else t)(torch.from_numpy(np.ascontiguousarray(x).view(np.int16)))
     Qh, Kh, Vh = pin(full.Q), pin(full.K[last]), pin(full.V[last])
-    Oh = torch.zeros((3, 8, 64), dtype=torch.float32).pin_memory()
+    Oh = torch.zeros((3, 8, 64), dtype=torch.float32)
+    Oh = Oh.pin_memory() if pinned else Oh
     staging = torch.empty(sa.staging_bytes(cfg, 3), dtype=torch.uint8, device=dev)
     sa.decode_step_host(cfg, cache.handle, Qh, Kh, Vh, Oh, staging, cache.workspace)
     torch.cuda.synchronize()
