@@ -21,7 +21,7 @@
 namespace sa {
 
 // Shared-memory plan of one block (dynamic shared memory, 128-byte aligned):
-//   [NW warps x kStages stage buffers][mbarriers][packed queries or table][query scales]; the
+//   [NW warps x NS stage buffers][mbarriers][packed queries or table][query scales]; the
 //   block-merge scratch re-uses the stage buffers once every warp has left its tile loop.
 template <int D, int KB, bool NIB, int GT>
 struct DecodeSmem {
@@ -31,8 +31,12 @@ struct DecodeSmem {
     static constexpr int CH = NIB ? D / 32 : D / 16;
     static constexpr int PLANES = (NIB && kTable) ? KB : 0;           // dense planar container: mantissa bit planes
     using Stage = TileStage<CH, true, D, PLANES, D / 8>;
+    // Stage buffers per warp: two at d = 64 (the next tile is in flight while this one is computed); one at
+    // d = 128, where a tile is 8 KB and a second buffer would halve the resident warps (the other warps of the
+    // SM cover the copy instead).
+    static constexpr int NS = (D == 128) ? 1 : kStages;
     static constexpr int kStageOff = 0;
-    static constexpr int kMbarOff = NW * kStages * Stage::kBytes;
+    static constexpr int kMbarOff = NW * NS * Stage::kBytes;
     // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
     // the table of query multiples [D][NP][2^KB] x 8 bytes
     static constexpr int kQpOff = (kMbarOff + 128 + 255) & ~255;   // the table datapath wants 256-byte alignment
@@ -44,7 +48,7 @@ struct DecodeSmem {
     // codes in the stage buffer, which are dead by then.)
     static constexpr int kBytes = kQscaleOff + 128;
     static constexpr int kBlocksPerSM = decode_shape(D, KB).blocks_per_sm;
-    static_assert(NW * GT * (D + 2) * 4 <= NW * kStages * Stage::kBytes && NW * kStages * 8 <= 128, "merge scratch must fit in the stage buffers");
+    static_assert(NW * GT * (D + 2) * 4 <= NW * NS * Stage::kBytes && NW * NS * 8 <= 128, "merge scratch must fit in the stage buffers");
     static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
 };
 
@@ -57,6 +61,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     constexpr int EPL = D / 32;
     constexpr int NP = SM::NP;
     constexpr int NW = SM::NW, NT = 32 * NW;       // warps and threads per block
+    constexpr int NS = SM::NS;                     // stage buffers per warp
     constexpr int WORDS = NIB ? D / 8 : D / 4;     // 32-bit code words per key
     constexpr int MT = D / 16;                     // 16-dim row tiles of O^T in the A.V phase
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -71,13 +76,13 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;     // first query head of this block
     const int b = blockIdx.z;
     const int split = blockIdx.x;
-    const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
-    const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
-    const uint8_t* stage_ptr0 = smem + SM::kStageOff + warp * kStages * Stage::kBytes;
+    const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * NS * 8;
+    const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * NS * Stage::kBytes;
+    const uint8_t* stage_ptr0 = smem + SM::kStageOff + warp * NS * Stage::kBytes;
 
     if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < kStages; ++s) mbar_init(mbar0 + s * 8, 1u);
+        for (int s = 0; s < NS; ++s) mbar_init(mbar0 + s * 8, 1u);
         fence_mbar_init();
         fence_proxy_async();
     }
@@ -209,12 +214,12 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         fence_proxy_async_global();
         __syncwarp();
     }
-    // Lane 0: start the copies of my i-th tile into stage i % kStages.  A tile whose page is not
+    // Lane 0: start the copies of my i-th tile into stage i % NS.  A tile whose page is not
     // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
     auto issue = [&](int i) {
         const int tile = first + NW * i;
         const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
-        const int s = i % kStages;
+        const int s = i % NS;
         if (pidx < 0 || pidx >= a.n_pages) {
             mbar_arrive(mbar0 + s * 8);
         } else {
@@ -225,7 +230,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
     };
     if (lane == 0)
-        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
+        for (int i = 0; i < NS && i < n_my; ++i) issue(i);
 
     int M[GT];
     float l[GT];
@@ -247,14 +252,14 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 
     for (int i = 0; i < n_my; ++i) {
         const int tile = first + NW * i;
-        const int s = i % kStages;
-        const uint32_t parity = (uint32_t)(i / kStages) & 1u;
+        const int s = i % NS;
+        const uint32_t parity = (uint32_t)(i / NS) & 1u;
         // the decision is made warp-uniform: a lane must never leave the loop alone
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(mbar0 + s * 8, parity))) {
             failed = true;
             // give the other stage's copy (already issued) a bounded chance to land before this
             // warp's buffers are re-used by the block merge
-            if (i + 1 < n_my) (void)mbar_wait_bounded(mbar0 + ((i + 1) % kStages) * 8, (uint32_t)((i + 1) / kStages) & 1u);
+            if (NS > 1 && i + 1 < n_my) (void)mbar_wait_bounded(mbar0 + ((i + 1) % NS) * 8, (uint32_t)((i + 1) / NS) & 1u);
             break;
         }
         const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
@@ -355,9 +360,9 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 }
                 g_min = min(g_min, valid ? g_j : 0x7fffffff);
                 __syncwarp();
-                if (lane == 0 && i + kStages < n_my) {
+                if (lane == 0 && i + NS < n_my) {
                     fence_proxy_async();
-                    issue(i + kStages);
+                    issue(i + NS);
                 }
                 continue;
             }
@@ -435,9 +440,9 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             }
         }
         __syncwarp();                                         // every lane is done with this stage
-        if (lane == 0 && i + kStages < n_my) {
+        if (lane == 0 && i + NS < n_my) {
             fence_proxy_async();
-            issue(i + kStages);
+            issue(i + NS);
         }
     }
     if (failed) {
