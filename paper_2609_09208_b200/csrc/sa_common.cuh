@@ -35,12 +35,12 @@ sa_status make_plan(const sa_config* cfg, Plan* out);
 // Warps per block and resident blocks per SM of the decode kernel that serves a code
 // (kb: 0 PoT-4, 1 / 2 / 4 mantissa codes, 8 INT8; the kernels' launch bounds and shared-memory
 // plans are sized for exactly this, and the split plan counts on it).  The PoT-M4 table of query
-// multiples is 32 KB at d = 64: there eight warps share one table and two blocks are resident.
+// multiples is 32 KB at d = 64: there ten warps share one table and two blocks are resident.
 struct KernelShape {
     int warps, blocks_per_sm;
 };
 constexpr KernelShape decode_shape(int d, int kb) {
-    return (kb == 4 && d == 64) ? KernelShape{8, 2}
+    return (kb == 4 && d == 64) ? KernelShape{10, 2}
            : (kb == 4)          ? KernelShape{4, 3}
            : (kb == 1 || kb == 2) ? KernelShape{4, 4}
                                   : KernelShape{4, 5};

@@ -31,10 +31,10 @@ struct DecodeSmem {
     static constexpr int CH = NIB ? D / 32 : D / 16;
     static constexpr int PLANES = (NIB && kTable) ? KB : 0;           // dense planar container: mantissa bit planes
     using Stage = TileStage<CH, true, D, PLANES, D / 8>;
-    // Stage buffers per warp: two at d = 64 (the next tile is in flight while this one is computed); one at
-    // d = 128, where a tile is 8 KB and a second buffer would halve the resident warps (the other warps of the
-    // SM cover the copy instead).
-    static constexpr int NS = (D == 128) ? 1 : kStages;
+    // Stage buffers per warp: two (the next tile is in flight while this one is computed), except where a
+    // second buffer would cost resident warps — d = 128 (a tile is 8 KB) and PoT-M4 (32 KB table): there one,
+    // and the other warps of the SM cover the copy instead.
+    static constexpr int NS = (D == 128 || KB == 4) ? 1 : kStages;
     static constexpr int kStageOff = 0;
     static constexpr int kMbarOff = NW * NS * Stage::kBytes;
     // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
