@@ -35,13 +35,15 @@ sa_status make_plan(const sa_config* cfg, Plan* out);
 // Warps per block and resident blocks per SM of the decode kernel that serves a code
 // (kb: 0 PoT-4, 1 / 2 / 4 mantissa codes, 8 INT8; the kernels' launch bounds and shared-memory
 // plans are sized for exactly this, and the split plan counts on it).  The PoT-M4 table of query
-// multiples is 32 KB at d = 64: there ten warps share one table and two blocks are resident.
+// multiples is 32 KB at d = 64: there ten warps share one table and two blocks are resident (20
+// warps at 96 registers).  The smaller tables of PoT-M1 / M2 leave room for four 4-warp blocks, whose
+// finer granularity serves short and ragged sequences better.
 struct KernelShape {
     int warps, blocks_per_sm;
 };
 constexpr KernelShape decode_shape(int d, int kb) {
-    return (kb == 4 && d == 64) ? KernelShape{10, 2}
-           : (kb == 4)          ? KernelShape{4, 3}
+    return (kb == 4 && d == 64)   ? KernelShape{10, 2}
+           : (kb == 4)            ? KernelShape{4, 3}
            : (kb == 1 || kb == 2) ? KernelShape{4, 4}
                                   : KernelShape{4, 5};
 }
