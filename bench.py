@@ -332,6 +332,23 @@ def recorded_traffic(variant):
     return None
 
 
+def recorded_pipes(variant):
+    """Issue-slot and pipe utilisation of the main kernel from the committed ncu capture
+    (profiles/pipe_utilisation.txt: variant, batch, then per cent of peak while the SM is active)."""
+    path = os.path.join(ROOT, "profiles", "pipe_utilisation.txt")
+    rows = []
+    try:
+        for line in open(path):
+            parts = line.split("#")[0].split()
+            if len(parts) == 7 and parts[0] == variant:
+                rows.append({"batch": int(parts[1]), "issue_slots_pct": float(parts[2]), "alu_pipe_pct": float(parts[3]),
+                             "fma_pipe_pct": float(parts[4]), "lsu_pipe_pct": float(parts[5]),
+                             "shared_wavefronts_pct": float(parts[6])})
+    except Exception:
+        pass
+    return rows or None
+
+
 def time_steps(fn, n, dev):
     """n calls of fn between two CUDA events on the current stream; returns milliseconds."""
     import torch
@@ -469,12 +486,31 @@ def run_ours(args):
                   "replayed; stream synchronised once per step"}
     sampler.stop_flag = True
 
+    # ---- cold single call: one layer's step with L2 flushed (a 256 MB buffer written) before every call ----
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cold = []
+    for r in range(5):
+        flush.fill_(r)
+        c = wl.caches[r % wl.layers]
+        ev0.record()
+        sa.decode_step(wl.cfg, c.handle, wl.Q[0], wl.Kn[0], wl.Vn[0], wl.O[0], c.workspace)
+        ev1.record()
+        torch.cuda.synchronize()
+        cold.append(ev0.elapsed_time(ev1) * 1e3)
+    del flush
+    group = wl.Hq // wl.Hkv
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if wl.fp16 else "int32", "data": "synthetic", "config": workload_config(args),
         "clocks": clocks, "e2e": e2e, "gpu_launches": wl.launches_per_step * K,
         "hbm_gbs_step": value / args.gpus * wl.bpk / 1e9, "roofline": roofline,
+        "scores_per_s": value * group,                      # (query, key) scores: keys/s x query heads per KV head
+        "cold_call_us": {"median": sorted(cold)[len(cold) // 2], "best": min(cold),
+                         "what": "one sa_decode_step call (one layer), L2 flushed before each of 5 calls"},
+        "pipe_utilisation": recorded_pipes(args.variant),   # from the ncu captures under profiles/ (not measured live)
     }
     if rank == 0 and args.gpus == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.variant, args.seq_len, args.batch)
