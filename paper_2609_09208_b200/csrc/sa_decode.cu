@@ -178,6 +178,19 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     }
     __syncthreads();
 
+    // While the preceding kernel drains: a guess at this warp's first tile, from a length that kernel may be
+    // about to change, only to ask L2 for it (loads that bypass L1, so nothing stale can be read back later).
+    if (lane == 0) {
+        const int len_g = __ldcg(a.seq_lens + b) + (a.Knew ? 1 : 0);
+        const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
+        const int tile_g = (int)((long long)n_tiles_g * split / a.n_splits) + warp;
+        if (tile_g < (int)((long long)n_tiles_g * (split + 1) / a.n_splits)) {
+            const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
+            if (pidx_g >= 0 && pidx_g < a.n_pages)
+                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, a.kcode_off, a.meta_off, a.v_off,
+                                (tile_g & 1) * 32, a.zr == nullptr, a.plane_off);
+        }
+    }
     pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
 
     // ---- this warp's tiles; start the first copies ----

@@ -54,6 +54,12 @@ SA_D void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar)
                  : "memory");
 }
 
+// Ask for `bytes` (a multiple of 16) at src to be brought into L2; a hint that changes no state the
+// program can observe.
+SA_D void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+
 // Layout of one stage buffer: [code chunks: CHUNKS x 512 B][mantissa bit planes: PLANES x 32 rows of
 // PLANE_ROW bytes (dense planar container only)][metadata: 128 B or none][values: 32 rows].
 template <int CHUNKS, bool HAS_META, int VROW_BYTES, int PLANES = 0, int PLANE_ROW = 0>
@@ -85,6 +91,17 @@ struct TileStage {
         }
         if (HAS_META) bulk_g2s(dst + kMetaOff, block + meta_off + (size_t)tk0 * 4, 128u, mbar);
         if (with_values) bulk_g2s(dst + kVOff, block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes, mbar);
+    }
+    // The same ranges as issue(), as L2 prefetch hints.
+    SA_D static void prefetch(const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off, int tk0,
+                              bool with_values, size_t plane_off) {
+#pragma unroll
+        for (int c = 0; c < CHUNKS; ++c) bulk_prefetch_l2(block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
+#pragma unroll
+        for (int b = 0; b < PLANES; ++b)
+            bulk_prefetch_l2(block + plane_off + ((size_t)b * kPageTokens + tk0) * PLANE_ROW, (uint32_t)kPlaneBytes);
+        if (HAS_META) bulk_prefetch_l2(block + meta_off + (size_t)tk0 * 4, 128u);
+        if (with_values) bulk_prefetch_l2(block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes);
     }
 };
 
