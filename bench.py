@@ -96,7 +96,7 @@ class Workload:
             del K, V
         torch.cuda.synchronize()
         self.keys_per_step = layers * batch * T * Hkv
-        self.launches_per_step = layers * (3 if fp16 else 2)   # (append,) main kernel, merge
+        self.launches_per_step = layers * 2          # main kernel (appends the new token), merge
 
     def decode(self, l, stages=3):
         sa = self.sa
@@ -107,8 +107,8 @@ class Workload:
             sa.decode_attention(self.cfg, c.handle, self.Q[l], self.O[l], c.workspace, None, stages=stages)
 
     def step(self):
-        # one decode step per layer through the library's step entry: for the quantised caches the decode
-        # kernel writes the new token itself (2 kernels per layer), for FP16 append + decode (3 kernels)
+        # one decode step per layer through the library's step entry: the decode kernel writes the new token
+        # itself (2 kernels per layer: decode and split-K merge)
         for l in range(self.layers):
             c = self.caches[l]
             self.sa.decode_step(self.cfg, c.handle, self.Q[l], self.Kn[l], self.Vn[l], self.O[l], c.workspace)

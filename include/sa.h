@@ -191,8 +191,8 @@ sa_status sa_decode_attention_fp16(const sa_config* cfg, const sa_cache* cache, 
  * step; seq_lens[b] is incremented by the split-K merge kernel, after every block has read it.
  * As with sa_append_kv the token's page must already be mapped; if it is not, the token is not
  * written, the length stays, and the step attends over the old cache.
- * With a binary16 cache (SA_KV_FP16), or more than 8 query heads per KV head, the call runs the
- * two kernels separately.  Same buffers, alignment and workspace as sa_decode_attention;
+ * With more than 8 query heads per KV head the call runs the two kernels separately.  A binary16
+ * cache (SA_KV_FP16) is served the same way by the binary16 decode kernel.  Same buffers, alignment and workspace as sa_decode_attention;
  * K_new, V_new [batch, n_kv_heads, head_dim] binary16, 16-byte aligned. */
 sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                          const uint16_t* K_new, const uint16_t* V_new, float* O, void* workspace,

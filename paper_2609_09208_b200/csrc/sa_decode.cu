@@ -538,6 +538,7 @@ static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, c
 }
 
 namespace sa {
+void launch_decode_fp16_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s);   // sa_decode_fp16.cu
 // The decode kernel for these arguments (the score pass of the shift-A.V option when a.zr is set).
 void launch_decode_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s) {
     const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
@@ -583,8 +584,8 @@ extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache,
     int S, GT;
     if (cache && cache->batch > 0 && cache->max_pages_per_seq > 0) split_plan(p, cache->batch, cache->max_pages_per_seq, &S, &GT);
     else GT = 0;
-    if (p.fp16 || GT != p.G) {
-        // binary16 cache, or a query group wider than one block: the separate append kernel
+    if (GT != p.G) {
+        // a query group wider than one block: the separate append kernel
         st = sa_append_kv(cfg, cache, K_new, V_new, 1, stream);
         if (st != SA_OK) return st;
         return p.fp16 ? sa_decode_attention_fp16(cfg, cache, Q, O, workspace, workspace_bytes, stream)
@@ -597,8 +598,10 @@ extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache,
     a.Vnew = V_new;
     a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / (double)(1LL << p.F));
     if (p.int8) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / 127.0);
+    if (p.fp16) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d));
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    launch_decode_main(p, a, GT, s);
+    if (p.fp16) launch_decode_fp16_main(p, a, GT, s);
+    else launch_decode_main(p, a, GT, s);
     if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
     return launch_merge(p, a, s);
 }

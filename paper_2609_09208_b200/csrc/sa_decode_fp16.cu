@@ -12,6 +12,7 @@
 //                     A fragments of P; V fragments come from ldmatrix.trans on 8 x 8 blocks
 //                     (8 keys x one 16-byte chunk), which the chunk layout stores contiguously.
 #include "sa_common.cuh"
+#include "sa_cache_write.cuh"
 #include "sa_decode_common.cuh"
 #include "sa_mma.cuh"
 #include "sa_quant.cuh"
@@ -38,6 +39,13 @@ struct Fp16Stage {
 #pragma unroll
         for (int c = 0; c < kChunks; ++c)
             bulk_g2s(dst + kVOff + c * 512, block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+    }
+    // the same ranges as L2 prefetch hints
+    SA_D static void prefetch(const uint8_t* block, size_t k_off, size_t v_off, int tk0) {
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) bulk_prefetch_l2(block + k_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) bulk_prefetch_l2(block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
     }
 };
 
@@ -78,25 +86,7 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     }
     __syncwarp();
 
-    const int len = a.seq_lens[b];
-    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
-    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
-    const int first = tile0 + warp;
-    const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
-    auto issue = [&](int i) {
-        const int tile = first + 4 * i;
-        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
-        const int s = i % kStages;
-        if (pidx < 0 || pidx >= a.n_pages) {
-            mbar_arrive(mbar0 + s * 8);
-        } else {
-            const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
-            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.v_off, (tile & 1) * 32, mbar0 + s * 8);
-        }
-    };
-    if (lane == 0)
-        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
+    pdl_launch_dependents();    // the split-K merge may be scheduled as soon as blocks of this grid retire
 
     // Q fragments (A operand, rows = query heads; rows >= GT are zero): for 16-dim block kb the lane
     // holds dims 16kb + 2*quad + {0,1} and + 8 of query `row`.
@@ -110,6 +100,60 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
             qa[kb][1] = __ldg(q32 + kb * 8 + 4 + quad);
         }
     }
+
+    // While the preceding kernel drains: ask L2 for this warp's first tile, guessed from a length that kernel
+    // may be about to change (loads that bypass L1; a hint only).
+    if (lane == 0) {
+        const int len_g = __ldcg(a.seq_lens + b) + (a.Knew ? 1 : 0);
+        const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
+        const int tile_g = (int)((long long)n_tiles_g * split / a.n_splits) + warp;
+        if (tile_g < (int)((long long)n_tiles_g * (split + 1) / a.n_splits)) {
+            const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
+            if (pidx_g >= 0 && pidx_g < a.n_pages)
+                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, a.kcode_off, a.v_off, (tile_g & 1) * 32);
+        }
+    }
+    pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
+
+    int len = a.seq_lens[b];
+    int tile_new = -1, pidx_new = -1;
+    if (a.Knew) {
+        // fused append (see the quantised kernel): the step's new token goes to position len if its page is mapped
+        const int lp = len / kPageTokens;
+        pidx_new = (len >= 0 && lp < a.max_pages) ? a.page_table[(size_t)b * a.max_pages + lp] : -1;
+        if (pidx_new >= 0 && pidx_new < a.n_pages) {
+            tile_new = len >> 5;
+            len += 1;
+        }
+    }
+    const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
+    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
+    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int first = tile0 + warp;
+    const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
+    if (tile_new >= first && tile_new < tile1 && (tile_new - first) % 4 == 0) {      // this warp owns that tile
+        CacheArgs ca{};
+        ca.kcode_off = a.kcode_off;
+        ca.v_off = a.v_off;
+        uint8_t* block = const_cast<uint8_t*>(a.pages) + ((size_t)pidx_new * a.Hkv + kvh) * a.page_bytes;
+        const size_t rown = ((size_t)b * a.Hkv + kvh) * D;
+        write_token<D, 16>(block, ca, (len - 1) % kPageTokens, lane, a.Knew + rown, a.Vnew + rown);
+        fence_proxy_async_global();
+        __syncwarp();
+    }
+    auto issue = [&](int i) {
+        const int tile = first + 4 * i;
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int s = i % kStages;
+        if (pidx < 0 || pidx >= a.n_pages) {
+            mbar_arrive(mbar0 + s * 8);
+        } else {
+            const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
+            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.v_off, (tile & 1) * 32, mbar0 + s * 8);
+        }
+    };
+    if (lane == 0)
+        for (int i = 0; i < kStages && i < n_my; ++i) issue(i);
 
     int M = kMNone;                                // running maximum of this lane's query row
     float l = 0.0f;                                // this lane's share of the row's weight sum
@@ -245,7 +289,7 @@ static void launch_fp16_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         (void)once;
     }
-    decode_fp16_kernel<D, GT><<<grid, 128, bytes, s>>>(a);
+    (void)launch_pdl(decode_fp16_kernel<D, GT>, grid, dim3(128), (size_t)bytes, s, a);
 }
 
 template <int D>
@@ -257,6 +301,15 @@ static void launch_fp16(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) 
         default: launch_fp16_one<D, 1>(a, grid, s); break;
     }
 }
+
+namespace sa {
+// the binary16 decode kernel for these arguments (used by sa_decode_step as well)
+void launch_decode_fp16_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s) {
+    const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
+    if (p.d == 64) launch_fp16<64>(a, GT, grid, s);
+    else launch_fp16<128>(a, GT, grid, s);
+}
+}  // namespace sa
 
 extern "C" sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const sa_cache* cache,
                                                      const uint16_t* Q, float* O, void* workspace,
@@ -273,9 +326,7 @@ extern "C" sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const
     a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d));
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (stages & 1) {
-        const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
-        if (p.d == 64) launch_fp16<64>(a, GT, grid, s);
-        else launch_fp16<128>(a, GT, grid, s);
+        launch_decode_fp16_main(p, a, GT, s);
         if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
     }
     return (stages & 2) ? launch_merge(p, a, s) : SA_OK;
