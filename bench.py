@@ -349,6 +349,20 @@ def recorded_pipes(variant):
     return rows or None
 
 
+def recorded(fn, warm=2):
+    """Run fn a few times, then record it once in a CUDA graph and return the replay callable: small kernels
+    launched one by one from Python are bound by the host's launch rate (about 12 us per launch), not by the GPU."""
+    import torch
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    torch.cuda.synchronize()
+    return g.replay
+
+
 def time_steps(fn, n, dev):
     """n calls of fn between two CUDA events on the current stream; returns milliseconds."""
     import torch
@@ -425,9 +439,10 @@ def run_ours(args):
     def main_kernels():
         for l in range(wl.layers):
             wl.decode(l, stages=1)
+    replay_main = recorded(main_kernels)
     for _ in range(2):
-        main_kernels()
-    ms_main, _, _ = time_steps(main_kernels, K, dev)
+        replay_main()
+    ms_main, _, _ = time_steps(replay_main, K, dev)
     main_us = ms_main / (K * wl.layers) * 1e3
     alg_bytes = wl.algorithmic_bytes_per_main_launch()
     achieved = alg_bytes / (main_us * 1e-6) / 1e9
@@ -441,7 +456,7 @@ def run_ours(args):
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "kernel": "decode main kernel (scores + softmax + A.V)", "kernel_us": main_us,
                 "algorithmic_bytes_per_launch": alg_bytes,
-                "how": "CUDA events around %d back-to-back launches over %d distinct layer caches" % (K * wl.layers, wl.layers)}
+                "how": "CUDA events around %d back-to-back launches over %d distinct layer caches, replayed from a CUDA graph" % (K * wl.layers, wl.layers)}
 
     # ---- end to end through the host-buffer entry: pinned H2D of Q / new K,V and D2H of O per layer ----
     # one pinned input buffer per layer, Q | K_new | V_new after one another (the entry then needs one copy)
@@ -533,9 +548,10 @@ def context_rows(args, dev):
         def main_kernels():
             for l in range(wl.layers):
                 wl.decode(l, stages=1)
+        replay_main = recorded(main_kernels)
         for _ in range(2):
-            main_kernels()
-        ms, _, _ = time_steps(main_kernels, 10, dev)
+            replay_main()
+        ms, _, _ = time_steps(replay_main, 10, dev)
         us = ms / (10 * wl.layers) * 1e3
         keys = wl.batch * wl.T * wl.Hkv
         rows.append({"variant": variant, "batch": batch, "layers": layers, "main_kernel_us": us,

@@ -82,10 +82,17 @@ class Cell:
         for _ in range(3):
             self.run_once()
         torch.cuda.synchronize()
+        # one pass over the caches recorded in a CUDA graph: launched one by one from Python, short calls
+        # would be bound by the host's launch rate instead of the GPU
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run_once()
+        graph.replay()
+        torch.cuda.synchronize()
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record()
         for _ in range(reps):
-            self.run_once()
+            graph.replay()
         e.record()
         torch.cuda.synchronize()
         return s.elapsed_time(e) * 1e3 / (reps * len(self.caches))
