@@ -34,18 +34,20 @@ struct Plan {
 sa_status make_plan(const sa_config* cfg, Plan* out);
 // Warps per block and resident blocks per SM of the decode kernel that serves a code
 // (kb: 0 PoT-4, 1 / 2 / 4 mantissa codes, 8 INT8; the kernels' launch bounds and shared-memory
-// plans are sized for exactly this, and the split plan counts on it).  The PoT-M4 table of query
-// multiples is 32 KB at d = 64: there ten warps share one table and two blocks are resident (20
-// warps at 96 registers).  The smaller tables of PoT-M1 / M2 leave room for four 4-warp blocks, whose
-// finer granularity serves short and ragged sequences better.
+// plans are sized for exactly this, and the split plan counts on it).  At d = 64 two blocks of ten
+// warps (20 warps at 96 registers): for PoT-M4 the ten warps share one 32 KB table of query
+// multiples, and for every code fewer, larger blocks mean fewer prologues and partials, which is
+// most of the time of a batch-1 step.  PoT-M1 / M2 keep four blocks of four warps: their finer
+// granularity serves the short and ragged batches those codes are specified for (measured: 16 %
+// faster there, 6 % slower at T = 32768, batch 1).
 struct KernelShape {
     int warps, blocks_per_sm;
 };
 constexpr KernelShape decode_shape(int d, int kb) {
-    return (kb == 4 && d == 64)   ? KernelShape{10, 2}
-           : (kb == 4)            ? KernelShape{4, 3}
-           : (kb == 1 || kb == 2) ? KernelShape{4, 4}
-                                  : KernelShape{4, 5};
+    return (kb == 1 || kb == 2) ? KernelShape{4, 4}
+           : (d == 64)          ? KernelShape{10, 2}
+           : (kb == 4)          ? KernelShape{4, 3}
+                                : KernelShape{4, 5};
 }
 constexpr KernelShape kFp16Shape{4, 3};
 // number of splits of the key axis for a cache of this shape, and queries handled per block

@@ -39,7 +39,7 @@ struct DecodeSmem {
     static constexpr int kMbarOff = NW * NS * Stage::kBytes;
     // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
     // the table of query multiples [D][NP][2^KB] x 8 bytes
-    static constexpr int kQpOff = (kMbarOff + 128 + 255) & ~255;   // the table datapath wants 256-byte alignment
+    static constexpr int kQpOff = (kMbarOff + 256 + 255) & ~255;   // the table datapath wants 256-byte alignment
     // (the prologue's scratch for the unpacked queries, D x GT words, uses the same space first)
     static constexpr int kQpData = kTable ? D * NP * (8 << KB) : D * NP * 4;
     static constexpr int kQpBytes = kQpData > D * GT * 4 ? kQpData : D * GT * 4;
@@ -48,7 +48,7 @@ struct DecodeSmem {
     // codes in the stage buffer, which are dead by then.)
     static constexpr int kBytes = kQscaleOff + 128;
     static constexpr int kBlocksPerSM = decode_shape(D, KB).blocks_per_sm;
-    static_assert(NW * GT * (D + 2) * 4 <= NW * NS * Stage::kBytes && NW * NS * 8 <= 128, "merge scratch must fit in the stage buffers");
+    static_assert(NW * GT * (D + 2) * 4 <= NW * NS * Stage::kBytes && NW * NS * 8 <= 256, "merge scratch must fit in the stage buffers");
     static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
 };
 

@@ -97,7 +97,7 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
     const int bps = shape.blocks_per_sm, nw = shape.warps;
     const long long slots = (long long)kNumSMs * bps;
     const long long tiles = (long long)max_pages * (kPageTokens / 32);
-    long long cap = tiles / nw;                     // every warp should own at least one tile
+    long long cap = tiles / 2;                      // at least two tiles per block (short caches: spread them over the SMs)
     if (cap < 1) cap = 1;
     if (cap > 512) cap = 512;
     const double c_fix = 0.5;
