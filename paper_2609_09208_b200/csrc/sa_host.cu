@@ -128,8 +128,9 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
 __global__ void __launch_bounds__(256) stage_in_kernel(const uint4* __restrict__ q, const uint4* __restrict__ k,
                                                        const uint4* __restrict__ v, uint4* __restrict__ dq,
                                                        uint4* __restrict__ dk, uint4* __restrict__ dv, int nq, int nkv) {
-    pdl_wait();                                  // the staging buffer may still be read by the step before
-    pdl_launch_dependents();
+    // The staging buffer may still be read by the step before.  No early launch_dependents here: the decode
+    // kernel reads Q ahead of its own wait, so it must not start before this kernel has completed.
+    pdl_wait();
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i < nq) dq[i] = q[i];
     else if (i < nq + nkv) dk[i - nq] = k[i - nq];
