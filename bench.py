@@ -527,6 +527,15 @@ def run_ours(args):
                          "what": "one sa_decode_step call (one layer), L2 flushed before each of 5 calls"},
         "pipe_utilisation": recorded_pipes(args.variant),   # from the ncu captures under profiles/ (not measured live)
     }
+    pipes = line["pipe_utilisation"]
+    if pipes:
+        # The resource that actually binds the shift kernels is the integer ALU pipe (shift, logic, permute):
+        # 64 lanes per SM and clock.  Fraction from the recorded capture of the nearest batch size.
+        row = min(pipes, key=lambda r: abs(r["batch"] - wl.batch))
+        alu_peak = 148 * 64 * clocks.get("sm_mhz", 1965.0) * 1e6
+        line["roofline_alu"] = {"bound": "alu", "peak": alu_peak, "unit": "thread-instr/s", "frac": row["alu_pipe_pct"] / 100.0,
+                                "achieved": alu_peak * row["alu_pipe_pct"] / 100.0, "issue_slots_frac": row["issue_slots_pct"] / 100.0,
+                                "source": "ncu sm__inst_executed_pipe_alu of the capture at batch %d (profiles/)" % row["batch"]}
     if rank == 0 and args.gpus == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.variant, args.seq_len, args.batch)
     if rank == 0 and args.context:
