@@ -1,15 +1,16 @@
 // Decode attention over the power-of-two key cache: the hot path.
 //
-// Grid (split, KV head x query chunk, sequence), 128 threads.  A block quantises its GT query
-// heads into shared memory, then each of its four warps walks its own 32-key tiles of the
-// block's slice of the key axis with a private online-softmax state, so the main loop has no
-// block-wide barrier.  Per tile: lane = key for the integer scores (section II-B eq. (3) with
-// the mantissa code of eq. (5)), warp-wide maxima and an integer running maximum in the log2
-// domain (section II-E); then the floating-point A.V over the INT8 values as small tensor-core
-// products O^T[dims][queries] += V^T[dims][keys] P^T[keys][queries] (mma.m16n8k8, tf32 operands:
-// the INT8 values are exact, every weight is split into two tf32 terms, accumulation in FP32).
-// The four warps' states and then the blocks' partial results are merged with exact
-// power-of-two factors.
+// Grid (split, KV head x query chunk, sequence); 4 or 10 warps per block (decode_shape).  A block
+// quantises its GT query heads into shared memory (ahead of its wait on the preceding kernel),
+// then each of its warps walks its own 32-key tiles of the block's slice of the key axis with a
+// private online-softmax state, so the main loop has no block-wide barrier.  Per tile: lane = key
+// for the integer scores (section II-B eq. (3) with the mantissa code of eq. (5)), warp-wide maxima
+// and an integer running maximum in the log2 domain (section II-E); then the floating-point A.V
+// over the INT8 values as small tensor-core products
+// O^T[dims][queries] += V^T[dims][keys] P^T[keys][queries] (mma.m16n8k8, tf32 operands: the INT8
+// values are exact, every weight is split into two tf32 terms, accumulation in FP32).  The warps'
+// states and then the blocks' partial results are merged with exact power-of-two factors.
+// For sa_decode_step the warp that owns the new token's tile writes the token first (section II-F).
 #include "sa_common.cuh"
 #include "sa_cache_write.cuh"
 #include "sa_datapath.cuh"
@@ -20,7 +21,7 @@
 
 namespace sa {
 
-// Shared-memory plan of one block (dynamic shared memory, 128-byte aligned):
+// Shared-memory plan of one block (dynamic shared memory, 1024-byte aligned):
 //   [NW warps x NS stage buffers][mbarriers][packed queries or table][query scales]; the
 //   block-merge scratch re-uses the stage buffers once every warp has left its tile loop.
 template <int D, int KB, bool NIB, int GT>
