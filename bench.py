@@ -254,11 +254,11 @@ def cpu_baseline(variant, T, batch):
     sample = OracleSample(variant, T, batch, n_layers=2)
     threads = max(1, min(hw, 4 * batch))
     sample.run_layer(0, 1)                                   # warm the page cache
-    v1, t1 = sample.time_layers(12, 1)
-    vm, tm = sample.time_layers(24, threads)
+    v1, t1 = sample.time_layers(48, 1)                       # about 8 s on one core
+    vm, tm = sample.time_layers(120, threads)                # about 6 s on four
     return {"value": vm, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": "decode-time oracle stages (query quantise, integer scores, two-pass softmax + A.V; cache "
-                      "pre-encoded) on 24 layer passes of the workload (2 distinct layers, %d keys each), one host "
+                      "pre-encoded) on 120 layer passes of the workload (2 distinct layers, %d keys each), one host "
                       "thread per KV head; %.1f s" % (sample.keys_per_layer, tm),
             "value_1core": v1, "seconds_1core": t1, "host_threads_available": hw}
 
