@@ -113,23 +113,53 @@ __global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __
     const int dd = threadIdx.x % D, grp = threadIdx.x / D;
     const size_t stride = (size_t)n_rows * (D + 2);
     const float* base = partials + (size_t)row * (D + 2);
-    // global maximum of the integer running maxima
-    int Ms = kMNone;
-    for (int s = threadIdx.x; s < n_splits; s += D * kMergeGroups) Ms = max(Ms, __float_as_int(base[s * stride]));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) Ms = max(Ms, __shfl_xor_sync(0xffffffffu, Ms, o));
-    if ((threadIdx.x & 31) == 0) m_s[threadIdx.x >> 5] = Ms;
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < D * kMergeGroups / 32; ++w) Ms = max(Ms, m_s[w]);
     float l = 0.0f, o = 0.0f;
+    constexpr int kHeld = 16;                                 // splits per thread held in registers
+    if (n_splits <= kHeld * kMergeGroups) {
+        // Common case: every load of this thread is issued before anything waits on one of them (a single
+        // round trip to L2), then the maximum of the integer running maxima, then the exact rescale.
+        int Mv[kHeld];
+        float lv[kHeld], ov[kHeld];
+#pragma unroll
+        for (int k = 0; k < kHeld; ++k) {
+            const int s = grp + k * kMergeGroups;
+            const float* p = base + (size_t)(s < n_splits ? s : 0) * stride;
+            Mv[k] = (s < n_splits) ? __float_as_int(p[0]) : kMNone;
+            lv[k] = p[1];
+            ov[k] = p[2 + dd];
+        }
+        int Ms = kMNone;
+#pragma unroll
+        for (int k = 0; k < kHeld; ++k) Ms = max(Ms, Mv[k]);
+        // the thread's splits are those of its whole group: one value per group is enough
+        if (dd == 0) m_s[grp] = Ms;
+        __syncthreads();
+#pragma unroll
+        for (int g = 0; g < kMergeGroups; ++g) Ms = max(Ms, m_s[g]);
+#pragma unroll
+        for (int k = 0; k < kHeld; ++k) {
+            const float f = (Mv[k] == kMNone) ? 0.0f : pow2i_neg(Mv[k] - Ms);
+            l += lv[k] * f;
+            o += ov[k] * f;
+        }
+    } else {
+        // global maximum of the integer running maxima
+        int Ms = kMNone;
+        for (int s = threadIdx.x; s < n_splits; s += D * kMergeGroups) Ms = max(Ms, __float_as_int(base[s * stride]));
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) Ms = max(Ms, __shfl_xor_sync(0xffffffffu, Ms, o2));
+        if ((threadIdx.x & 31) == 0) m_s[threadIdx.x >> 5] = Ms;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < D * kMergeGroups / 32; ++w) Ms = max(Ms, m_s[w]);
 #pragma unroll 8
-    for (int s = grp; s < n_splits; s += kMergeGroups) {
-        const float* p = base + s * stride;
-        const int M = __float_as_int(p[0]);
-        const float f = (M == kMNone) ? 0.0f : pow2i_neg(M - Ms);
-        l += p[1] * f;
-        o += p[2 + dd] * f;
+        for (int s = grp; s < n_splits; s += kMergeGroups) {
+            const float* p = base + s * stride;
+            const int M = __float_as_int(p[0]);
+            const float f = (M == kMNone) ? 0.0f : pow2i_neg(M - Ms);
+            l += p[1] * f;
+            o += p[2 + dd] * f;
+        }
     }
     o_s[grp][dd] = o;
     if (dd == 0) o_s[grp][D] = l;
