@@ -37,7 +37,8 @@
  *                elements 32c .. 32c+31, byte i = element 32c+2i in the low nibble and 32c+2i+1
  *                in the high nibble, nibble = sign << 3 | g.
  *     meta_off : 64 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.
- *     v_off    : vhat, int8, row-major [64][head_dim].
+ *     v_off    : vhat, int8, in 16-byte chunks like the keys: chunk c (dims 16c .. 16c+15) of token t
+ *                at (c * 64 + t) * 16.
  *   For code = SA_KV_FP16 the block holds unquantised binary16 data: K and then V, each in
  *   16-byte chunks of 8 elements (chunk c of token t at (c * 64 + t) * 16), no metadata.
  */

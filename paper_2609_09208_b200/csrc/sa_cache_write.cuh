@@ -67,7 +67,10 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
             }
         }
     }
-    store_bytes<EPL>(block + a.v_off + (size_t)t * D + lane * EPL, vc);
+    {
+        const int mv = lane * EPL;                  // values: 16-dim chunks, chunk c of token t at (c * 64 + t) * 16
+        store_bytes<EPL>(block + a.v_off + ((size_t)(mv >> 4) * kPageTokens + t) * 16 + (mv & 15), vc);
+    }
     if (lane == 0)
         *reinterpret_cast<uint32_t*>(block + a.meta_off + (size_t)t * 4) = (smax & 0xffffu) | ((uint32_t)(uint8_t)(int8_t)gg << 16);
 }

@@ -437,11 +437,11 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                     bh[j][c] = __float_as_uint(hi);
                     bl[j][c] = __float_as_uint(pv - hi) & 0xffffe000u;
                 }
-            const uint32_t vaddr = stage0 + s * Stage::kBytes + Stage::kVOff + lane * D;
+            const uint32_t vaddr = stage0 + s * Stage::kBytes + Stage::kVOff + lane * 16;   // chunk mt of key row `lane`
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 uint32_t x[4];
-                ldmatrix_x4_trans(x, vaddr + mt * 16);
+                ldmatrix_x4_trans(x, vaddr + mt * 512);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t a0 = __float_as_uint((float)(int8_t)(x[j]));

@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
         store_bytes<EPL>(codes + (size_t)v * D + m, c);
     }
     if (vhat) {
-        const uint8_t* src = block + a.v_off + (size_t)t * D + m;
+        const uint8_t* src = block + a.v_off + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15);
         uint8_t c[EPL];
 #pragma unroll
         for (int i = 0; i < EPL; ++i) c[i] = src[i];

@@ -159,16 +159,17 @@ __global__ void __launch_bounds__(128) shiftav_kernel(DecodeArgs a) {
             for (int g = 0; g < GT; ++g)
 #pragma unroll
                 for (int c = 0; c < DPL; ++c) acc[g][c] = 0u;
-            const uint8_t* vbase = st + Stage::kVOff + lane * DPL;
+            // values are staged in 16-dim chunks of 512 bytes: this lane's dims sit in chunk (lane * DPL) / 16
+            const uint8_t* vbase = st + Stage::kVOff + ((lane * DPL) >> 4) * 512 + ((lane * DPL) & 15);
 #pragma unroll 4
             for (int t = 0; t < 32; ++t) {
                 uint32_t v[DPL];
                 if constexpr (DPL == 2) {
-                    const uint32_t vv = *reinterpret_cast<const uint16_t*>(vbase + t * D);
+                    const uint32_t vv = *reinterpret_cast<const uint16_t*>(vbase + t * 16);
                     v[0] = (uint32_t)(int32_t)(int8_t)(vv);
                     v[1] = (uint32_t)(int32_t)(int8_t)(vv >> 8);
                 } else {
-                    const uint32_t vv = *reinterpret_cast<const uint32_t*>(vbase + t * D);
+                    const uint32_t vv = *reinterpret_cast<const uint32_t*>(vbase + t * 16);
 #pragma unroll
                     for (int c = 0; c < DPL; ++c) v[c] = (uint32_t)(int32_t)(int8_t)(vv >> (8 * c));
                 }

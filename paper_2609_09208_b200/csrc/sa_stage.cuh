@@ -61,7 +61,8 @@ SA_D void bulk_prefetch_l2(const void* src, uint32_t bytes) {
 }
 
 // Layout of one stage buffer: [code chunks: CHUNKS x 512 B][mantissa bit planes: PLANES x 32 rows of
-// PLANE_ROW bytes (dense planar container only)][metadata: 128 B or none][values: 32 rows].
+// PLANE_ROW bytes (dense planar container only)][metadata: 128 B or none][value chunks: VROW_BYTES / 16 x 512 B,
+// chunk c = 16 dims of the 32 tokens after one another, as in the page].
 template <int CHUNKS, bool HAS_META, int VROW_BYTES, int PLANES = 0, int PLANE_ROW = 0>
 struct TileStage {
     static constexpr int kCodeBytes = CHUNKS * 512;
@@ -90,7 +91,11 @@ struct TileStage {
                          (uint32_t)kPlaneBytes, mbar);
         }
         if (HAS_META) bulk_g2s(dst + kMetaOff, block + meta_off + (size_t)tk0 * 4, 128u, mbar);
-        if (with_values) bulk_g2s(dst + kVOff, block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes, mbar);
+        if (with_values) {
+#pragma unroll
+            for (int c = 0; c < VROW_BYTES / 16; ++c)
+                bulk_g2s(dst + kVOff + c * 512, block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+        }
     }
     // The same ranges as issue(), as L2 prefetch hints.
     SA_D static void prefetch(const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off, int tk0,
@@ -101,7 +106,10 @@ struct TileStage {
         for (int b = 0; b < PLANES; ++b)
             bulk_prefetch_l2(block + plane_off + ((size_t)b * kPageTokens + tk0) * PLANE_ROW, (uint32_t)kPlaneBytes);
         if (HAS_META) bulk_prefetch_l2(block + meta_off + (size_t)tk0 * 4, 128u);
-        if (with_values) bulk_prefetch_l2(block + v_off + (size_t)tk0 * VROW_BYTES, (uint32_t)kVBytes);
+        if (with_values) {
+#pragma unroll
+            for (int c = 0; c < VROW_BYTES / 16; ++c) bulk_prefetch_l2(block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
+        }
     }
 };
 
