@@ -31,9 +31,9 @@
  *   ((size_t)p * n_kv_heads + h) * page_bytes and holds page_tokens = 64 tokens of KV head h:
  *     kcode_off: key codes in 16-byte chunks, chunk c of token t at (c * 64 + t) * 16.
  *                Byte container (any k): chunk c holds elements 16c .. 16c+15, one byte each:
- *                the canonical byte with its exponent field replaced by g = 7 - e (g = 0 for the
- *                zero code), i.e. canonical ^ 0x70, so that g - 1 is the shift amount and zeroed
- *                memory reads as zero codes.  Nibble container (PoT-4 only): chunk c holds
+ *                sign << 7 | mantissa field << 3 | g, with the canonical byte's 4-bit mantissa
+ *                field and g = 7 - e (g = 0 for the zero code), so that g - 1 is the shift amount,
+ *                the mantissa field times 8 a table offset, and zeroed memory reads as zero codes.  Nibble container (PoT-4 only): chunk c holds
  *                elements 32c .. 32c+31, byte i = element 32c+2i in the low nibble and 32c+2i+1
  *                in the high nibble, nibble = sign << 3 | g.
  *     meta_off : 64 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.

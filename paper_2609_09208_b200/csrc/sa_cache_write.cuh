@@ -31,9 +31,10 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
         smax = encode_key_int8_vec<EPL>(kb, lane, a.hadamard != 0, kc);      // uniform INT8: stored as is
     } else {
         smax = encode_key_vec<EPL, K>(kb, lane, a.hadamard != 0, kc);
-        // physical exponent field g = 7 - e (0 for the zero code): canonical byte ^ 0x70
+        // byte container: the physical byte (phys_byte); the sub-byte containers below work on the canonical
+        // byte with its exponent field replaced by g = 7 - e (0 for the zero code), i.e. canonical ^ 0x70
 #pragma unroll
-        for (int i = 0; i < EPL; ++i) kc[i] ^= 0x70;
+        for (int i = 0; i < EPL; ++i) kc[i] = NIB ? (uint8_t)(kc[i] ^ 0x70) : phys_byte(kc[i]);
     }
     const int gg = quantise_value_vec<EPL>(vb, vc);
     uint8_t* kdst = block + a.kcode_off;

@@ -57,6 +57,17 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
 // Exact helpers (usable on host for unit tests of the arithmetic, and on device).
 // ---------------------------------------------------------------------------------------------
 
+// Byte container: physical byte of a canonical code byte (sign << 7 | e << 4 | mantissa << (4 - k)):
+//   sign << 7 | mantissa field << 3 | g,   g = 7 - e for a non-zero element, 0 for the zero code.
+// The exponent field sits in the low bits (g - 1 is the shift amount), the mantissa field at bits
+// 3 .. 6 (times 8 it is the byte offset of a table entry), and zeroed memory reads as zero codes.
+SA_HD uint8_t phys_byte(uint8_t canon) {
+    return (uint8_t)((canon & 0x80u) | ((canon & 0x0fu) << 3) | (((canon >> 4) & 7u) ^ 7u));
+}
+SA_HD uint8_t canon_byte(uint8_t phys) {
+    return (uint8_t)((phys & 0x80u) | (((phys & 7u) ^ 7u) << 4) | ((phys >> 3) & 0x0fu));
+}
+
 // Normalise a non-zero binary16 magnitude (15 bits) to M * 2^X with M in [1024, 2047].
 SA_HD void half_normalise(uint32_t mag_bits, int* M, int* X) {
     const int ex = (int)(mag_bits >> 10);

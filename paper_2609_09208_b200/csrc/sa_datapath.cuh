@@ -18,10 +18,9 @@
 //   32-bit totals.
 // Mantissa codes (KB = 1, 2, 4): table datapath, see TableScore below.
 //
-// Physical code format inside a page (differs from the canonical byte only in the exponent field):
-// byte = sign << 7 | g << 4 | mantissa, g = 7 - e for a non-zero element and 0 for the zero code,
-// i.e. physical = canonical ^ 0x70 (and nibble = canonical nibble ^ 0x7).  The shift amount is
-// g - 1, which is 0xffffffff for the zero code, and a shift by 32 or more returns 0.
+// Physical code format inside a page: byte container  sign << 7 | mantissa field << 3 | g  (phys_byte in
+// sa_common.cuh), nibble  sign << 3 | g,  with g = 7 - e for a non-zero element and 0 for the zero code.
+// The shift amount is g - 1, which is 0xffffffff for the zero code, and a shift by 32 or more returns 0.
 #pragma once
 #include "sa_common.cuh"
 
@@ -153,7 +152,7 @@ struct PackedShift {
 template <int NP>
 SA_HD void accumulate_word_bytes(PackedShift<NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
     // shift amounts g - 1 per byte: 0..6, and 0xff for the zero code (g = 0)
-    const uint32_t gw = (w >> 4) & 0x07070707u;
+    const uint32_t gw = w & 0x07070707u;
     const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -266,10 +265,10 @@ struct TableScore {
     // whose table starts at grp (256-byte aligned).
     template <int W4, typename Base>
     SA_HD void accumulate_word(uint32_t w, Base grp) {
-        const uint32_t gw = (w >> 4) & 0x07070707u;
+        const uint32_t gw = w & 0x07070707u;
         const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;       // shift amounts g - 1; 0xff for the zero code
-        // byte offsets mu * 8 of the mantissas' entries (mu = the byte's low nibble >> (4 - KB))
-        const uint32_t offs = KB == 4 ? (w << 3) & 0x78787878u : KB == 2 ? (w << 1) & 0x18181818u : w & 0x08080808u;
+        // byte offsets mu * 8 of the mantissas' entries: the mantissa field (bits 3 .. 6) holds mu << (4 - KB)
+        const uint32_t offs = KB == 4 ? w & 0x78787878u : KB == 2 ? (w >> 2) & 0x18181818u : (w >> 3) & 0x08080808u;
         elements<W4, 0>(w, rw, offs, grp);
     }
     // Dense planar container (PoT-M1 / PoT-M2 only): one 32-bit word of sign/exponent nibbles = 8

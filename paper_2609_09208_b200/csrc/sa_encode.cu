@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
         if (!NIB) {
             const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15);
 #pragma unroll
-            for (int i = 0; i < EPL; ++i) c[i] = src[i] ^ xor_mask;      // 0x70 for the power-of-two codes, 0 for INT8
+            for (int i = 0; i < EPL; ++i) c[i] = xor_mask ? canon_byte(src[i]) : src[i];   // power-of-two codes / INT8 stored as is
         } else {
             const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 5) * kPageTokens + t) * 16 + ((m & 31) >> 1);
 #pragma unroll

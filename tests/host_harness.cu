@@ -6,7 +6,7 @@
 using namespace sa;
 
 // Scores of one PoT-4 key (canonical code bytes) against 8 queries, through the same packed
-// datapath and word decoders the decode kernel uses (physical codes = canonical ^ 0x70).
+// datapath and word decoders the decode kernel uses (byte container: phys_byte; nibbles: canonical nibble ^ 7).
 static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
     alignas(16) static uint32_t qp[128][4];
     for (int m = 0; m < d; ++m)
@@ -16,7 +16,7 @@ static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool ni
     if (!nibble_path) {
         for (int m0 = 0; m0 < d; m0 += 4) {
             uint32_t w = 0;
-            for (int i = 0; i < 4; ++i) w |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * i);
+            for (int i = 0; i < 4; ++i) w |= (uint32_t)phys_byte(canon[m0 + i]) << (8 * i);
             accumulate_word_bytes<4>(pl, w, &qp[m0][0], 4);
         }
     } else {
@@ -42,7 +42,7 @@ static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t*
     ts.begin(1u);
     for (int m0 = 0; m0 < d; m0 += 16) {
         uint32_t w[4] = {0, 0, 0, 0};
-        for (int i = 0; i < 16; ++i) w[i / 4] |= (uint32_t)(canon[m0 + i] ^ 0x70) << (8 * (i % 4));
+        for (int i = 0; i < 16; ++i) w[i / 4] |= (uint32_t)phys_byte(canon[m0 + i]) << (8 * (i % 4));
         const uint8_t* grp = tab + m0 * TS::kElemBytes;
         ts.template accumulate_word<0>(w[0], grp);
         ts.template accumulate_word<1>(w[1], grp);
