@@ -8,7 +8,8 @@
  * General rules for every function
  *   - `extern "C"`, returns an sa_status, never throws, never aborts.
  *   - Pointers are DEVICE pointers unless the parameter name ends in `_host`.  All memory is
- *     owned by the caller; the library allocates no device memory and keeps no state.
+ *     owned by the caller; the library allocates no device memory and keeps no state between
+ *     calls (the one exception, a fixed scratch array, is sa_decode_attention_static).
  *   - Work is enqueued on the caller's stream (`sa_stream` is a `cudaStream_t`); no function
  *     synchronises.  Arguments are validated on the host before anything is launched; a call
  *     that returns an error has launched nothing.
@@ -193,8 +194,9 @@ sa_status sa_decode_attention_fp16(const sa_config* cfg, const sa_cache* cache, 
  * As with sa_append_kv the token's page must already be mapped; if it is not, the token is not
  * written, the length stays, and the step attends over the old cache.
  * With more than 8 query heads per KV head the call runs the two kernels separately.  A binary16
- * cache (SA_KV_FP16) is served the same way by the binary16 decode kernel.  Same buffers, alignment and workspace as sa_decode_attention;
- * K_new, V_new [batch, n_kv_heads, head_dim] binary16, 16-byte aligned. */
+ * cache (SA_KV_FP16) is served the same way by the binary16 decode kernel.  Same buffers,
+ * alignment and workspace as sa_decode_attention; K_new, V_new [batch, n_kv_heads, head_dim]
+ * binary16, 16-byte aligned. */
 sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                          const uint16_t* K_new, const uint16_t* V_new, float* O, void* workspace,
                          size_t workspace_bytes, sa_stream stream);
