@@ -392,8 +392,9 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 if (a.dbg_scores && valid)
                     a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
                 const float z = valid ? (float)A[g] * qscale_s[g] * s_j : -INFINITY;
-                // ceil of the tile's largest logit: ceil is monotone, so take the integer maximum
-                const int Mt = warp_max_s32(__float2int_ru(fminf(fmaxf(z, -1.0e8f), 1.0e8f)));
+                // ceil of the tile's largest logit: ceil is monotone, so take the integer maximum (the
+                // conversion saturates; a lane without a key gives the smallest integer)
+                const int Mt = max(warp_max_s32(__float2int_ru(z)), -(1 << 28));
                 const int Mn = max(M[g], Mt);
                 resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);          // exact power of two
                 changed |= (Mn != M[g]);
