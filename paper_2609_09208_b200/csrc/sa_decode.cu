@@ -386,12 +386,14 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             float (*p_t)[8] = reinterpret_cast<float (*)[8]>(const_cast<uint8_t*>(st));
             bool changed = false;
             float resc[GT];
+            const float s_v = valid ? s_j : 0.0f, z_bias = valid ? 0.0f : -INFINITY;
             float pv[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};        // unused query columns stay zero
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 if (a.dbg_scores && valid)
                     a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
-                const float z = valid ? (float)A[g] * qscale_s[g] * s_j : -INFINITY;
+                // a lane without a key gets z = -inf through the addend (the product is rounded once either way)
+                const float z = fmaf((float)A[g] * qscale_s[g], s_v, z_bias);
                 // ceil of the tile's largest logit: ceil is monotone, so take the integer maximum (the
                 // conversion saturates; a lane without a key gives the smallest integer)
                 const int Mt = max(warp_max_s32(__float2int_ru(z)), -(1 << 28));
@@ -399,7 +401,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);          // exact power of two
                 changed |= (Mn != M[g]);
                 M[g] = Mn;
-                const float p = valid ? ex2_approx(z - (float)Mn) : 0.0f;
+                const float p = ex2_approx(z - (float)Mn);     // 2^-inf = 0 for a lane without a key
                 l[g] = l[g] * resc[g] + p;
                 pv[g] = p * vscale;                                                 // weight times 2^-g_j
             }
