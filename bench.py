@@ -256,7 +256,18 @@ def cpu_baseline(variant, T, batch):
     sample.run_layer(0, 1)                                   # warm the page cache
     v1, t1 = sample.time_layers(48, 1)                       # about 8 s on one core
     vm, tm = sample.time_layers(120, threads)                # about 6 s on four
-    return {"value": vm, "unit": UNIT, "cores": threads, "kind": "oracle",
+    stages = None
+    code_k, nibble, hadamard, fp16 = VARIANTS[variant]
+    if not fp16:
+        # one layer through the oracle's whole chain on one core, with its per-stage clocks (the cache build —
+        # key encode and value quantise — is not part of a decode step; it is shown for proportion)
+        case = synth.make_case("cpu_stages", [T] * batch, 32, 4, 64, code_k if code_k != 8 else 0, seed=4242)
+        res = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, code_k, 6 + (code_k if code_k != 8 else 0),
+                                   hadamard=hadamard, n_threads=1)
+        st = [float(x) for x in res["stage_seconds"]]
+        stages = {"rotate_and_quantise_query": st[0], "encode_keys_and_quantise_values": st[1], "integer_scores": st[2],
+                  "softmax_and_av": st[3], "what": "one layer (%d keys), one core, seconds" % (batch * T * 4)}
+    return {"value": vm, "unit": UNIT, "cores": threads, "kind": "oracle", "stage_seconds": stages,
             "sample": "decode-time oracle stages (query quantise, integer scores, two-pass softmax + A.V; cache "
                       "pre-encoded) on 120 layer passes of the workload (2 distinct layers, %d keys each), one host "
                       "thread per KV head; %.1f s" % (sample.keys_per_layer, tm),
