@@ -591,3 +591,37 @@ def test_random_shapes_against_oracle(dev, seed):
     torch.cuda.synchronize()
     assert torch.equal(O, O2)
     check_against_oracle(full, O.cpu().numpy(), dbg.cpu().numpy(), F=F)
+
+
+def test_config3_T32k_through_decode_step_in_a_cuda_graph(dev):
+    """The benchmark's launch configuration at full size: PoT-M4, batch 1, 32/4 heads, d = 64, a cache of
+    32 767 tokens plus the step's new one, sa_decode_step recorded in a CUDA graph and replayed — outputs
+    against the oracle over all 32 768 keys, and the appended token's codes bit-exact."""
+    import torch
+    case = synth.config3(4)
+    T = int(case.lens[0])
+    cfg = cfg_of(case)
+    cache = sa.PagedCache(cfg, np.array([T - 1]), dev, extra_tokens=4, permutation=synth.page_permutation((T + 3 + 63) // 64, 5))
+    cache.fill(t16(case.K[:T - 1], dev), t16(case.V[:T - 1], dev), np.array([0, T - 1]))
+    Q, Kn, Vn = t16(case.Q, dev), t16(case.K[T - 1:T], dev), t16(case.V[T - 1:T], dev)
+    O = torch.full((1, 32, 64), float("nan"), dtype=torch.float32, device=dev)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):                      # warm-up outside the capture, on a side stream
+        sa.decode_step(cfg, cache.handle, Q, Kn, Vn, O, cache.workspace)
+    torch.cuda.synchronize()
+    cache.seq_lens.fill_(T - 1)                          # take the warm-up's append back
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        sa.decode_step(cfg, cache.handle, Q, Kn, Vn, O, cache.workspace)
+    O.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(cache.seq_lens[0]) == T
+    check_against_oracle(case, O.cpu().numpy(), None)
+    codes = torch.zeros((T, 4, 64), dtype=torch.uint8, device=dev)
+    scales = torch.zeros((T, 4), dtype=torch.int16, device=dev)
+    sa.debug_unpack(cfg, cache.handle, 0, T, codes, scales)
+    torch.cuda.synchronize()
+    want_c, want_s = ora.encode_keys(case.K[T - 1:T], 4)
+    assert np.array_equal(codes[T - 1:].cpu().numpy(), want_c)
+    assert np.array_equal(scales[T - 1:].cpu().numpy().view(np.uint16), want_s.view(np.uint16))
