@@ -55,6 +55,10 @@ VARIANTS = {
     "fp16": (0, False, False, True),
     "int8mac": (8, False, False, False),      # uniform INT8 keys, dp4a scores: the paper's multiply-native comparison
 }
+# the same codes with the shifts executed by the integer multiplier (SA_FLAG_SHIFT_BY_MULTIPLY; not the default)
+MULSHIFT = {"potm4_mulshift": "potm4", "potm1_mulshift": "potm1", "pot4_nibble_mulshift": "pot4_nibble"}
+for _name, _base in MULSHIFT.items():
+    VARIANTS[_name] = VARIANTS[_base]
 
 
 def bytes_per_key(d, code_k, nibble, fp16):
@@ -76,7 +80,8 @@ class Workload:
         self.d, self.Hq, self.Hkv = d, Hq, Hkv
         self.fp16 = fp16
         self.bpk = bytes_per_key(d, code_k, nibble, fp16)
-        self.cfg = sa.make_config(d, Hq, Hkv, sa.SA_KV_FP16 if fp16 else code_k, nibble=nibble, hadamard=hadamard)
+        self.cfg = sa.make_config(d, Hq, Hkv, sa.SA_KV_FP16 if fp16 else code_k, nibble=nibble, hadamard=hadamard,
+                                  shift_by_multiply=variant in MULSHIFT)
         self.caches, self.Q, self.Kn, self.Vn, self.O = [], [], [], [], []
         cu = np.arange(batch + 1, dtype=np.int64) * T
         pages_per_seq = (T + room_tokens + 63) // 64

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libsa.so")
 SA_POT4, SA_POTM1, SA_POTM2, SA_POTM4, SA_INT8, SA_KV_FP16 = 0, 1, 2, 4, 8, 16
 SA_KLAYOUT_BYTE, SA_KLAYOUT_NIBBLE, SA_KLAYOUT_PLANAR = 0, 1, 2
 SA_FLAG_HADAMARD = 1
+SA_FLAG_SHIFT_BY_MULTIPLY = 2
 PAGE_TOKENS = 64
 
 EXPORTS = [
@@ -76,14 +77,15 @@ def _check(st: int, where: str):
 
 
 def make_config(head_dim: int, n_q_heads: int, n_kv_heads: int, code: int, *, nibble: bool = False,
-                headroom_F: int = 0, hadamard: bool = False) -> SaConfig:
+                headroom_F: int = 0, hadamard: bool = False, shift_by_multiply: bool = False) -> SaConfig:
     """nibble=True selects the dense sub-byte container of the code: two 4-bit codes per byte for PoT-4,
-    nibbles plus mantissa bit planes (5 / 6 bits per element) for PoT-M1 / PoT-M2."""
+    nibbles plus mantissa bit planes (5 / 6 bits per element) for PoT-M1 / PoT-M2.  shift_by_multiply=True
+    selects the non-default decode kernels whose shifts run on the integer multiplier (same scores)."""
     klayout = SA_KLAYOUT_BYTE
     if nibble:
         klayout = SA_KLAYOUT_NIBBLE if code == SA_POT4 else SA_KLAYOUT_PLANAR
     return SaConfig(head_dim, n_q_heads, n_kv_heads, code, klayout, headroom_F, PAGE_TOKENS,
-                    SA_FLAG_HADAMARD if hadamard else 0)
+                    (SA_FLAG_HADAMARD if hadamard else 0) | (SA_FLAG_SHIFT_BY_MULTIPLY if shift_by_multiply else 0))
 
 
 def get_layout(cfg: SaConfig) -> SaLayout:

@@ -23,6 +23,7 @@ constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no k
 // ---------------------------------------------------------------------------------------------
 struct Plan {
     int d, Hq, Hkv, G, k;     // k = mantissa bits (0 for SA_KV_FP16)
+    bool mulshift;            // SA_FLAG_SHIFT_BY_MULTIPLY: the scores' shifts run on the integer multiplier
     bool fp16, nibble, hadamard, int8;   // nibble: 4-bit sign/exponent codes (PoT-4 nibble container, or with k = 1, 2
                                          // the dense planar container); int8: the uniform INT8 comparison code
     int F;                    // head-room actually used

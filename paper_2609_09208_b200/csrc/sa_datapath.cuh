@@ -110,7 +110,9 @@ SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (
 // and at the end  lower-query sum = tot - (hit << 16) - bias  (exact: the true value is far below
 // 2^32) and  upper-query sum = hit.  That is one ALU instruction and two FMA-pipe adds per window
 // register.
-template <int NP>
+// MUL (the non-default SA_FLAG_SHIFT_BY_MULTIPLY): the element's sigma * 2^r is formed once and every
+// packed pair is multiplied by it — modulo 2^32 the same value as shifting first and multiplying by sigma.
+template <int NP, bool MUL = false>
 struct PackedShift {
     uint32_t win[NP];           // window sums, lower half biased by 0x8000
     uint32_t tot[NP], hit[NP];  // running totals, see above
@@ -125,12 +127,14 @@ struct PackedShift {
     }
     // r: shift amount (>= 32 for the zero code); sg: +1 or -1
     SA_HD void element_first(uint32_t r, uint32_t sg, const uint32_t* qp) {
+        const uint32_t m = MUL ? shl_clamp_hd(sg, r) : sg;     // sigma * 2^r (0 for the zero code)
 #pragma unroll
-        for (int p = 0; p < NP; ++p) win[p] = mad_fma(shl_clamp_hd(qp[p], r), sg, 0x8000u);
+        for (int p = 0; p < NP; ++p) win[p] = MUL ? mad_fma(qp[p], m, 0x8000u) : mad_fma(shl_clamp_hd(qp[p], r), sg, 0x8000u);
     }
     SA_HD void element_next(uint32_t r, uint32_t sg, const uint32_t* qp) {
+        const uint32_t m = MUL ? shl_clamp_hd(sg, r) : sg;
 #pragma unroll
-        for (int p = 0; p < NP; ++p) win[p] = mad_fma(shl_clamp_hd(qp[p], r), sg, win[p]);
+        for (int p = 0; p < NP; ++p) win[p] = MUL ? mad_fma(qp[p], m, win[p]) : mad_fma(shl_clamp_hd(qp[p], r), sg, win[p]);
     }
     SA_HD void window_end() {
         ++n_windows;
@@ -149,8 +153,8 @@ struct PackedShift {
 
 // One 32-bit word of the byte container = 4 elements.  qp points at the packed queries of the
 // word's first element; consecutive elements are `stride` words apart.
-template <int NP>
-SA_HD void accumulate_word_bytes(PackedShift<NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
+template <int NP, bool MUL>
+SA_HD void accumulate_word_bytes(PackedShift<NP, MUL>& pl, uint32_t w, const uint32_t* qp, int stride) {
     // shift amounts g - 1 per byte: 0..6, and 0xff for the zero code (g = 0)
     const uint32_t gw = w & 0x07070707u;
     const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;
@@ -167,8 +171,8 @@ SA_HD void accumulate_word_bytes(PackedShift<NP>& pl, uint32_t w, const uint32_t
 }
 
 // One 32-bit word of the nibble container = 8 elements, two windows.
-template <int NP>
-SA_HD void accumulate_word_nibbles(PackedShift<NP>& pl, uint32_t w, const uint32_t* qp, int stride) {
+template <int NP, bool MUL>
+SA_HD void accumulate_word_nibbles(PackedShift<NP, MUL>& pl, uint32_t w, const uint32_t* qp, int stride) {
     const uint32_t ge = w & 0x07070707u, go = (w >> 4) & 0x07070707u;   // g of even / odd elements
     const uint32_t re = (ge + 0x7f7f7f7fu) ^ 0x80808080u, ro = (go + 0x7f7f7f7fu) ^ 0x80808080u;
     const uint32_t we = w << 4;                                         // even elements' sign at the byte's top bit
@@ -228,7 +232,9 @@ SA_HD void table_gather(const uint8_t* base, uint32_t offs, int i, uint32_t& x, 
     y = e[1];
 }
 
-template <int KB, int NGP>
+// MUL (SA_FLAG_SHIFT_BY_MULTIPLY, not the default): sigma * 2^r is formed once per key element and the
+// update is one multiply-add of the table entry by it.
+template <int KB, int NGP, bool MUL = false>
 struct TableScore {
     static constexpr int kRowBytes = 8 << KB;              // one (element, query pair) row
     static constexpr int kElemBytes = NGP * kRowBytes;     // all query pairs of one element
@@ -241,14 +247,15 @@ struct TableScore {
 #pragma unroll
         for (int g = 0; g < 2 * NGP; ++g) acc[g] = 0;
     }
-    // query pairs GP .. NGP - 1 of one element; IMM = byte offset of the element's rows within the group
+    // query pairs GP .. NGP - 1 of one element; IMM = byte offset of the element's rows within the group;
+    // sg = sigma (with MUL: sigma * 2^r, and r is not used)
     template <int IMM, int GP, typename Base>
     SA_HD void element_pairs(Base grp, uint32_t offs, int i, uint32_t r, uint32_t sg) {
         if constexpr (GP < NGP) {
             uint32_t x, y;
             table_gather<IMM + GP * kRowBytes>(grp, offs, i, x, y);
-            acc[2 * GP] = mad_fma(shl_clamp_hd(x, r), sg, acc[2 * GP]);
-            acc[2 * GP + 1] = mad_fma(shl_clamp_hd(y, r), sg, acc[2 * GP + 1]);
+            acc[2 * GP] = MUL ? mad_fma(x, sg, acc[2 * GP]) : mad_fma(shl_clamp_hd(x, r), sg, acc[2 * GP]);
+            acc[2 * GP + 1] = MUL ? mad_fma(y, sg, acc[2 * GP + 1]) : mad_fma(shl_clamp_hd(y, r), sg, acc[2 * GP + 1]);
             element_pairs<IMM, GP + 1>(grp, offs, i, r, sg);
         }
     }
@@ -257,7 +264,7 @@ struct TableScore {
         if constexpr (I < 4) {
             const uint32_t r = prmt_hd(rw, 0u, 0x4440u | I);
             const uint32_t sg = mad_fma(prmt_hd(w, 0u, 0x8888u | (0x1111u * I)), two, one);   // sigma: 0 / -1 -> +1 / -1
-            element_pairs<(W4 * 4 + I) * kElemBytes, 0>(grp, offs, I, r, sg);
+            element_pairs<(W4 * 4 + I) * kElemBytes, 0>(grp, offs, I, r, MUL ? shl_clamp_hd(sg, r) : sg);
             elements<W4, I + 1>(w, rw, offs, grp);
         }
     }
@@ -281,7 +288,7 @@ struct TableScore {
             constexpr int byte = NI >> 1;
             const uint32_t r = prmt_hd((NI & 1) ? ro : re, 0u, 0x4440u | byte);
             const uint32_t sg = mad_fma(prmt_hd((NI & 1) ? w : we, 0u, 0x8888u | (0x1111u * byte)), two, one);
-            element_pairs<(W8 * 8 + NI) * kElemBytes, 0>(grp, (NI & 1) ? offs_o : offs_e, byte, r, sg);
+            element_pairs<(W8 * 8 + NI) * kElemBytes, 0>(grp, (NI & 1) ? offs_o : offs_e, byte, r, MUL ? shl_clamp_hd(sg, r) : sg);
             nibble_elements<W8, NI + 1>(w, we, re, ro, offs_e, offs_o, grp);
         }
     }

@@ -53,10 +53,11 @@ struct DecodeSmem {
     static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
 };
 
-template <int D, int KB, bool NIB, int GT>
+template <int D, int KB, bool NIB, int GT, bool MUL = false>
 __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM)) decode_kernel(DecodeArgs a) {
     // KB = 0: PoT-4 (packed shift datapath); KB = 1, 2, 4: mantissa codes (table datapath);
-    // KB = 8: uniform INT8 comparison code (dp4a)
+    // KB = 8: uniform INT8 comparison code (dp4a).  MUL: the shifts run on the integer multiplier
+    // (SA_FLAG_SHIFT_BY_MULTIPLY; same scores, reported separately from the shift kernels).
     using SM = DecodeSmem<D, KB, NIB, GT>;
     using Stage = typename SM::Stage;
     constexpr int EPL = D / 32;
@@ -287,7 +288,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             int32_t A[GT];
             const uint32_t* cw = reinterpret_cast<const uint32_t*>(st) + lane * 4;
             if constexpr (SM::kTable) {
-                using TS = TableScore<KB, NP>;
+                using TS = TableScore<KB, NP, MUL>;
                 uint32_t grp = smem_addr(smem + SM::kQpOff);    // table of the next 16 elements (256-byte aligned)
                 TS ts;
                 ts.begin(a.one);
@@ -330,13 +331,13 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)ts.score(g) << a.f_extra);   // exact: the true sum fits INT32
             } else if constexpr (KB != 8) {
-                PackedShift<NP> pl;
+                PackedShift<NP, MUL> pl;
                 pl.begin(a.one);
 #pragma unroll 1
                 for (int wq = 0; wq < WORDS; ++wq) {
                     const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
-                    if constexpr (!NIB) accumulate_word_bytes<NP>(pl, w, &qp_s[wq * 4][0], NP);
-                    else accumulate_word_nibbles<NP>(pl, w, &qp_s[wq * 8][0], NP);
+                    if constexpr (!NIB) accumulate_word_bytes(pl, w, &qp_s[wq * 4][0], NP);
+                    else accumulate_word_nibbles(pl, w, &qp_s[wq * 8][0], NP);
                 }
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
@@ -502,43 +503,49 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 
 using namespace sa;
 
-template <int D, int KB, bool NIB, int GT>
+template <int D, int KB, bool NIB, int GT, bool MUL>
 static void launch_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
     constexpr int bytes = DecodeSmem<D, KB, NIB, GT>::kBytes;
     if (bytes > 48 * 1024) {
         // opt in to more than 48 KB of dynamic shared memory (an attribute of the function; no allocation)
-        static const cudaError_t once = cudaFuncSetAttribute(decode_kernel<D, KB, NIB, GT>,
+        static const cudaError_t once = cudaFuncSetAttribute(decode_kernel<D, KB, NIB, GT, MUL>,
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         (void)once;
     }
-    (void)launch_pdl(decode_kernel<D, KB, NIB, GT>, grid, dim3(32 * DecodeSmem<D, KB, NIB, GT>::NW), (size_t)bytes, s, a);
+    (void)launch_pdl(decode_kernel<D, KB, NIB, GT, MUL>, grid, dim3(32 * DecodeSmem<D, KB, NIB, GT>::NW), (size_t)bytes, s, a);
 }
 
-template <int D, int KB, bool NIB>
+template <int D, int KB, bool NIB, bool MUL>
 static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     switch (GT) {
-        case 8: launch_one<D, KB, NIB, 8>(a, grid, s); break;
-        case 4: launch_one<D, KB, NIB, 4>(a, grid, s); break;
-        case 2: launch_one<D, KB, NIB, 2>(a, grid, s); break;
-        default: launch_one<D, KB, NIB, 1>(a, grid, s); break;
+        case 8: launch_one<D, KB, NIB, 8, MUL>(a, grid, s); break;
+        case 4: launch_one<D, KB, NIB, 4, MUL>(a, grid, s); break;
+        case 2: launch_one<D, KB, NIB, 2, MUL>(a, grid, s); break;
+        default: launch_one<D, KB, NIB, 1, MUL>(a, grid, s); break;
+    }
+}
+
+template <int D, bool MUL>
+static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
+    if (p.nibble) {
+        if (p.k == 0) launch_gt<D, 0, true, MUL>(a, GT, grid, s);
+        else if (p.k == 1) launch_gt<D, 1, true, MUL>(a, GT, grid, s);       // dense planar container
+        else launch_gt<D, 2, true, MUL>(a, GT, grid, s);
+        return;
+    }
+    switch (p.k) {
+        case 0: launch_gt<D, 0, false, MUL>(a, GT, grid, s); break;
+        case 1: launch_gt<D, 1, false, MUL>(a, GT, grid, s); break;
+        case 2: launch_gt<D, 2, false, MUL>(a, GT, grid, s); break;
+        default: launch_gt<D, 4, false, MUL>(a, GT, grid, s); break;
     }
 }
 
 template <int D>
-static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
-    if (p.nibble) {
-        if (p.k == 0) launch_gt<D, 0, true>(a, GT, grid, s);
-        else if (p.k == 1) launch_gt<D, 1, true>(a, GT, grid, s);       // dense planar container
-        else launch_gt<D, 2, true>(a, GT, grid, s);
-        return;
-    }
-    if (p.int8) { launch_gt<D, 8, false>(a, GT, grid, s); return; }
-    switch (p.k) {
-        case 0: launch_gt<D, 0, false>(a, GT, grid, s); break;
-        case 1: launch_gt<D, 1, false>(a, GT, grid, s); break;
-        case 2: launch_gt<D, 2, false>(a, GT, grid, s); break;
-        default: launch_gt<D, 4, false>(a, GT, grid, s); break;
-    }
+static void launch_dim(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
+    if (p.int8) launch_gt<D, 8, false, false>(a, GT, grid, s);
+    else if (p.mulshift) launch_code<D, true>(p, a, GT, grid, s);
+    else launch_code<D, false>(p, a, GT, grid, s);
 }
 
 namespace sa {
@@ -546,8 +553,8 @@ void launch_decode_fp16_main(const Plan& p, const DecodeArgs& a, int GT, cudaStr
 // The decode kernel for these arguments (the score pass of the shift-A.V option when a.zr is set).
 void launch_decode_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s) {
     const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
-    if (p.d == 64) launch_code<64>(p, a, GT, grid, s);
-    else launch_code<128>(p, a, GT, grid, s);
+    if (p.d == 64) launch_dim<64>(p, a, GT, grid, s);
+    else launch_dim<128>(p, a, GT, grid, s);
 }
 }  // namespace sa
 

@@ -12,7 +12,9 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
         return SA_ERR_INVALID_ARG;
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return SA_ERR_UNSUPPORTED;
     if (cfg->page_tokens != kPageTokens) return SA_ERR_UNSUPPORTED;
-    if (cfg->flags & ~SA_FLAG_HADAMARD) return SA_ERR_INVALID_ARG;
+    if (cfg->flags & ~(SA_FLAG_HADAMARD | SA_FLAG_SHIFT_BY_MULTIPLY)) return SA_ERR_INVALID_ARG;
+    p.mulshift = (cfg->flags & SA_FLAG_SHIFT_BY_MULTIPLY) != 0;
+    if (p.mulshift && (cfg->code == SA_KV_FP16 || cfg->code == SA_INT8)) return SA_ERR_UNSUPPORTED;   // no shift to move
     p.d = cfg->head_dim;
     p.Hq = cfg->n_q_heads;
     p.Hkv = cfg->n_kv_heads;

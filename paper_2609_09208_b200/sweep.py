@@ -27,12 +27,13 @@ def bytes_per_key(d, code, nibble):
 
 class Cell:
     def __init__(self, dev, lens, Hq, Hkv, d, code, nibble=False, hadamard=False, outliers=True, seed=1, min_bytes=400e6,
-                 shiftav=False):
+                 shiftav=False, shift_by_multiply=False):
         import torch
         from . import binding as sa
         from . import synth
         self.sa, self.torch = sa, torch
-        self.cfg = sa.make_config(d, Hq, Hkv, code, nibble=nibble, hadamard=hadamard and code != 16)
+        self.cfg = sa.make_config(d, Hq, Hkv, code, nibble=nibble, hadamard=hadamard and code != 16,
+                                  shift_by_multiply=shift_by_multiply)      # non-default: shifts on the integer multiplier
         self.fp16 = code == 16
         self.shiftav = shiftav                                # eq. (6), (7) option: N = k_max = 15
         lens = np.asarray(lens, dtype=np.int64)
@@ -129,6 +130,9 @@ def main():
         for code, nib in ([] if quick else [(0, True), (4, False)]):
             cell("cfg3 T=32768 B=%d %s%s shift-based A.V (N = k_max = 15)" % (B, names[code], "_nibble" if nib else ""),
                  [32768] * B, 32, 4, 64, code, nibble=nib, outliers=False, shiftav=True)
+        for code, nib in ([] if quick else [(0, True), (1, False), (4, False)]):
+            cell("cfg3 T=32768 B=%d %s%s shifts on the integer multiplier" % (B, names[code], "_nibble" if nib else ""),
+                 [32768] * B, 32, 4, 64, code, nibble=nib, outliers=False, shift_by_multiply=True)
     lens4 = np.random.Generator(np.random.PCG64(4001)).integers(2048, 16385, size=16)
     cell("cfg4 ragged B=16 [2048,16384] potm2", lens4, 32, 4, 64, 2)
     cell("cfg4 ragged B=16 [2048,16384] fp16", lens4, 32, 4, 64, 16)

@@ -7,23 +7,24 @@ using namespace sa;
 
 // Scores of one PoT-4 key (canonical code bytes) against 8 queries, through the same packed
 // datapath and word decoders the decode kernel uses (byte container: phys_byte; nibbles: canonical nibble ^ 7).
+template <bool MUL>
 static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
     alignas(16) static uint32_t qp[128][4];
     for (int m = 0; m < d; ++m)
         for (int p = 0; p < 4; ++p) qp[m][p] = pack_pair(q8[(2 * p) * d + m], q8[(2 * p + 1) * d + m]);
-    PackedShift<4> pl;
+    PackedShift<4, MUL> pl;
     pl.begin(1u);
     if (!nibble_path) {
         for (int m0 = 0; m0 < d; m0 += 4) {
             uint32_t w = 0;
             for (int i = 0; i < 4; ++i) w |= (uint32_t)phys_byte(canon[m0 + i]) << (8 * i);
-            accumulate_word_bytes<4>(pl, w, &qp[m0][0], 4);
+            accumulate_word_bytes(pl, w, &qp[m0][0], 4);
         }
     } else {
         for (int m0 = 0; m0 < d; m0 += 8) {
             uint32_t w = 0;
             for (int i = 0; i < 8; ++i) w |= (uint32_t)((canon[m0 + i] ^ 0x70) >> 4) << (4 * i);
-            accumulate_word_nibbles<4>(pl, w, &qp[m0][0], 4);
+            accumulate_word_nibbles(pl, w, &qp[m0][0], 4);
         }
     }
     for (int g = 0; g < 8; ++g) out[g] = pl.score(g);
@@ -31,9 +32,9 @@ static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool ni
 
 // The scores of a mantissa code (k = 1, 2, 4) through the table datapath.
 // The same scores through the table datapath of the mantissa codes.
-template <int K>
+template <int K, bool MUL>
 static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
-    using TS = TableScore<K, 4>;
+    using TS = TableScore<K, 4, MUL>;
     alignas(256) static uint8_t tab[128 * TS::kElemBytes];
     for (int m = 0; m < d; ++m)
         for (int gp = 0; gp < 4; ++gp)
@@ -54,9 +55,9 @@ static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t*
 
 // The same through the dense planar container (k = 1, 2): sign/exponent nibbles, two per byte, and the
 // mantissa bits in k separate bit planes.
-template <int K>
+template <int K, bool MUL>
 static void score8_planar(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
-    using TS = TableScore<K, 4>;
+    using TS = TableScore<K, 4, MUL>;
     alignas(256) static uint8_t tab[128 * TS::kElemBytes];
     for (int m = 0; m < d; ++m)
         for (int gp = 0; gp < 4; ++gp)
@@ -80,18 +81,23 @@ static void score8_planar(const uint8_t* canon, const int8_t* q8, int d, int32_t
     for (int g = 0; g < 8; ++g) out[g] = ts.score(g);
 }
 
+template <bool MUL>
+static void score8_any(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) {
+    // path 0: byte container (packed datapath for k = 0, table datapath otherwise); 1: nibble container
+    // (k = 0) or dense planar container (k = 1, 2)
+    if (k == 0) score8_packed<MUL>(canon, q8, d, path != 0, out);
+    else if (path != 0 && k == 1) score8_planar<1, MUL>(canon, q8, d, out);
+    else if (path != 0 && k == 2) score8_planar<2, MUL>(canon, q8, d, out);
+    else if (k == 1) score8_table<1, MUL>(canon, q8, d, out);
+    else if (k == 2) score8_table<2, MUL>(canon, q8, d, out);
+    else score8_table<4, MUL>(canon, q8, d, out);
+}
+
 extern "C" {
-void hh_score8_planar(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
-    if (k == 1) score8_planar<1>(canon, q8, d, out);
-    else score8_planar<2>(canon, q8, d, out);
-}
-void hh_score8_table(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
-    switch (k) {
-        case 1: score8_table<1>(canon, q8, d, out); break;
-        case 2: score8_table<2>(canon, q8, d, out); break;
-        default: score8_table<4>(canon, q8, d, out); break;
-    }
-}
+void hh_score8_planar(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) { score8_any<false>(k, canon, q8, d, 1, out); }
+void hh_score8_table(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) { score8_any<false>(k, canon, q8, d, 0, out); }
+// the same datapaths with the shifts executed as multiplications by 2^r
+void hh_score8_mul(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) { score8_any<true>(k, canon, q8, d, path, out); }
 int hh_encode_element(int k, unsigned a_bits, unsigned s_bits) {
     switch (k) {
         case 0: return encode_element<0>(a_bits, s_bits);
@@ -105,7 +111,6 @@ void hh_encode_many(int k, const uint16_t* a_bits, int64_t n, unsigned s_bits, u
 }
 int hh_value_exponent(unsigned amax_bits) { return value_exponent(amax_bits); }
 void hh_score8(int k, const uint8_t* canon, const int8_t* q8, int d, int nibble_path, int32_t* out) {
-    if (k == 0) score8_packed(canon, q8, d, nibble_path != 0, out);
-    else hh_score8_table(k, canon, q8, d, out);
+    score8_any<false>(k, canon, q8, d, k == 0 ? nibble_path : 0, out);
 }
 }

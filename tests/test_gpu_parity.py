@@ -28,10 +28,10 @@ def t16(x, dev):
     return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev)
 
 
-def cfg_of(case, *, code=None, F=0):
+def cfg_of(case, *, code=None, F=0, shift_by_multiply=False):
     code = case.code_k if code is None else code
     return sa.make_config(case.head_dim, case.n_q_heads, case.n_kv_heads, code, nibble=case.nibble,
-                          headroom_F=F, hadamard=case.hadamard)
+                          headroom_F=F, hadamard=case.hadamard, shift_by_multiply=shift_by_multiply)
 
 
 def build_cache(case, dev, *, cfg=None, permute_seed=None, extra_tokens=0):
@@ -43,9 +43,9 @@ def build_cache(case, dev, *, cfg=None, permute_seed=None, extra_tokens=0):
     return cfg, cache
 
 
-def run_decode(case, dev, *, F=0, want_scores=True, permute_seed=None):
+def run_decode(case, dev, *, F=0, want_scores=True, permute_seed=None, shift_by_multiply=False):
     import torch
-    cfg = cfg_of(case, F=F)
+    cfg = cfg_of(case, F=F, shift_by_multiply=shift_by_multiply)
     cfg, cache = build_cache(case, dev, cfg=cfg, permute_seed=permute_seed)
     O = torch.full((case.batch, case.n_q_heads, case.head_dim), float("nan"), dtype=torch.float32, device=dev)
     dbg = None
@@ -625,3 +625,36 @@ def test_config3_T32k_through_decode_step_in_a_cuda_graph(dev):
     want_c, want_s = ora.encode_keys(case.K[T - 1:T], 4)
     assert np.array_equal(codes[T - 1:].cpu().numpy(), want_c)
     assert np.array_equal(scales[T - 1:].cpu().numpy().view(np.uint16), want_s.view(np.uint16))
+
+
+# ------------------------------------------------------ shifts on the integer multiplier (non-default option)
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 32, 4), (128, 8, 2), (64, 6, 2)])
+@pytest.mark.parametrize("k,nibble", [(0, False), (0, True), (1, False), (1, True), (2, False), (2, True), (4, False)])
+def test_shift_by_multiply_gives_the_same_scores(dev, d, Hq, Hkv, k, nibble):
+    """SA_FLAG_SHIFT_BY_MULTIPLY: INT32 scores bit-exact against the oracle (hence equal to the shift kernels'),
+    outputs within the tolerance; ragged batch with an empty sequence, several tiles, head-room above the default."""
+    F = 6 + k + (2 if d == 64 else 0)
+    case = synth.make_case("mulshift", [700, 0, 33, 129], Hq, Hkv, d, k, outliers=True, seed=4700 + 10 * k + d, nibble=nibble)
+    O, dbg, _ = run_decode(case, dev, F=F, permute_seed=7, shift_by_multiply=True)
+    check_against_oracle(case, O, dbg, F=F)
+
+
+def test_shift_by_multiply_step_matches_the_shift_kernel_bitwise(dev):
+    """The fused step with the option on and off: the same appended token, and outputs equal bit for bit
+    (the scores are the same integers and everything after them is the same code)."""
+    import torch
+    case = synth.config3(4, T=4096 + 1)
+    T = int(case.lens[0])
+    outs = []
+    for flag in (False, True):
+        cfg = cfg_of(case, shift_by_multiply=flag)
+        cache = sa.PagedCache(cfg, np.array([T - 1]), dev, extra_tokens=1)
+        cache.fill(t16(case.K[:T - 1], dev), t16(case.V[:T - 1], dev), np.array([0, T - 1]))
+        O = torch.full((1, 32, 64), float("nan"), dtype=torch.float32, device=dev)
+        sa.decode_step(cfg, cache.handle, t16(case.Q, dev), t16(case.K[T - 1:], dev), t16(case.V[T - 1:], dev), O, cache.workspace)
+        torch.cuda.synchronize()
+        assert int(cache.seq_lens[0]) == T
+        outs.append((O.cpu().numpy(), cache.pages.cpu().numpy()))
+    assert np.array_equal(outs[0][0].view(np.uint32), outs[1][0].view(np.uint32))
+    assert np.array_equal(outs[0][1], outs[1][1])
+    check_against_oracle(case, outs[1][0], None)
