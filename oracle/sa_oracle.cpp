@@ -342,7 +342,7 @@ void ora_attention_twopass(const int64_t* A, const float* delta, const uint16_t*
 
 // ---------------------------------------------------------------------------------
 // Uniform INT8 key code: the comparison datapath of section III and section VI (an INT8
-// multiply-accumulate kernel "built on the same tiling"; Table II lists the uniform INT8
+// multiply-accumulate kernel with the tiling of the shift kernel; Table II lists the uniform INT8
 // quantiser as an accuracy baseline).  Per key vector: scale = largest magnitude (binary16),
 // khat = clamp(round-half-even(K * 127 / amax), -127, 127), decided in binary32 exactly like
 // the query quantiser; K ~ (scale / 127) * khat.  Scores are plain integer dot products
@@ -460,7 +460,7 @@ void ora_attention_online(const int64_t* A, const float* delta, const uint16_t* 
 
 // ---------------------------------------------------------------------------------
 // Log2-quantised attention weights and the shift-based A.V: section II-E, eq. (6) and
-// eq. (7) — the paper's non-default option ("both products multiplier-free").
+// eq. (7) — the paper's non-default option, in which the second product needs no multiplier either.
 //
 //   M      = ceil(max_j z_j)                      (integer, log2 domain, z = logit * log2 e)
 //   k_j    = round(M - z_j) >= 0,  weight 2^-k_j                                   eq. (6)
