@@ -14,7 +14,7 @@
 //           smallest value exponent;
 //   pass 2  shiftav_kernel below: reduces those statistics to M and g_ref, then per 32-key tile
 //           forms the shift indices (lane = key), accumulates vhat << index in INT32 (lane =
-//           output dims; "a per-tile INT32 accumulator suffices") and adds the tile's sum to FP32
+//           output dims; the paper notes that an INT32 accumulator per tile is enough) and adds the tile's sum to FP32
 //           running sums; a key with k_j > k_max is dropped everywhere, one with a negative shift
 //           index from the numerator only;
 //   merge   the ordinary split-K merge (all partials share the reference M, so its factors are 1).
