@@ -56,7 +56,7 @@ VARIANTS = {
     "int8mac": (8, False, False, False),      # uniform INT8 keys, dp4a scores: the paper's multiply-native comparison
 }
 # the same codes with the shifts executed by the integer multiplier (SA_FLAG_SHIFT_BY_MULTIPLY; not the default)
-MULSHIFT = {"potm4_mulshift": "potm4", "potm1_mulshift": "potm1", "pot4_nibble_mulshift": "pot4_nibble"}
+MULSHIFT = {"potm4_mulshift": "potm4", "potm1_mulshift": "potm1", "potm2_mulshift": "potm2"}
 for _name, _base in MULSHIFT.items():
     VARIANTS[_name] = VARIANTS[_base]
 

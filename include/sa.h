@@ -82,13 +82,13 @@ enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_INT8 = 8, SA_KV
 enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1, SA_KLAYOUT_PLANAR = 2 };
 /* flags */
 #define SA_FLAG_HADAMARD 1u /* rotate Q and K by the normalised Walsh-Hadamard matrix before quantising */
-/* Decode kernels only, power-of-two codes only, off by default: execute the left shift of eq. (3), (4) on the
- * integer multiplier.  Each key element is decoded once, for the whole query group, to sigma * 2^(F - k - e)
- * (0 for the zero code) and every (query, element) update is one integer multiply-add by that power of two
- * instead of a shift followed by the sign multiply-add.  The INT32 scores are the same bit for bit.  This
- * uses the multiplier array as a barrel shifter, so it is not the paper's multiplier-free datapath; it is
- * the mid-point between the shift kernels and the INT8 multiply-accumulate comparison (section III), and is
- * reported as such. */
+/* Decode kernels only, mantissa codes (PoT-M1 / M2 / M4) only, off by default: execute the left shift of
+ * eq. (3), (4) on the integer multiplier.  Each key element is decoded once, for the whole query group, to
+ * sigma * 2^(F - k - e) (0 for the zero code) and every (query, element) update is one integer multiply-add
+ * by that power of two instead of a shift followed by the sign multiply-add.  The INT32 scores are the same
+ * bit for bit.  This uses the multiplier array as a barrel shifter, so it is not the paper's multiplier-free
+ * datapath; it is the mid-point between the shift kernels and the INT8 multiply-accumulate comparison
+ * (section III), and is reported as such.  (PoT-4 has no shift left in its key loop: SA_ERR_UNSUPPORTED.) */
 #define SA_FLAG_SHIFT_BY_MULTIPLY 2u
 
 typedef struct {

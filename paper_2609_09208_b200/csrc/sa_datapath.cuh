@@ -9,9 +9,11 @@
 //   q_lo borrows from the upper half; all arithmetic below is plain integer arithmetic on P, so
 //   the two halves stay exact as long as the lower half's running sum fits in 16 bits).  One
 //   shift and one add then serve two (query, element) pairs.
+// * The shift P << r depends on the key only through its exponent, so the block shifts every packed
+//   pair by every r once (ShiftTable) and the key loop looks the shifted pair up.
 // * The sign flip and the add are one multiply-add by sigma = +1 or -1 (the multiplier only ever
 //   sees +1 or -1: magnitudes are shifted, never multiplied).  It issues on the FMA pipe while the
-//   shifts and byte permutes issue on the ALU pipe: on sm_100a the two pipes run side by side
+//   byte permutes issue on the ALU pipe: on sm_100a the two pipes run side by side
 //   (64 + 64 thread-instructions per clock per SM).
 // * A window of 4 elements (4 * 127 * 2^6 < 2^15) is accumulated in the packed register, whose
 //   lower half is biased by 0x8000 so that it never borrows; then both halves are added into
@@ -110,9 +112,7 @@ SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (
 // and at the end  lower-query sum = tot - (hit << 16) - bias  (exact: the true value is far below
 // 2^32) and  upper-query sum = hit.  That is one ALU instruction and two FMA-pipe adds per window
 // register.
-// MUL (the non-default SA_FLAG_SHIFT_BY_MULTIPLY): the element's sigma * 2^r is formed once and every
-// packed pair is multiplied by it — modulo 2^32 the same value as shifting first and multiplying by sigma.
-template <int NP, bool MUL = false>
+template <int NP>
 struct PackedShift {
     uint32_t win[NP];           // window sums, lower half biased by 0x8000
     uint32_t tot[NP], hit[NP];  // running totals, see above
@@ -125,16 +125,14 @@ struct PackedShift {
 #pragma unroll
         for (int p = 0; p < NP; ++p) tot[p] = hit[p] = 0;
     }
-    // r: shift amount (>= 32 for the zero code); sg: +1 or -1
-    SA_HD void element_first(uint32_t r, uint32_t sg, const uint32_t* qp) {
-        const uint32_t m = MUL ? shl_clamp_hd(sg, r) : sg;     // sigma * 2^r (0 for the zero code)
+    // sg: +1 or -1; x: the element's packed pairs, already shifted (an entry of ShiftTable)
+    SA_HD void entry_first(uint32_t sg, const uint32_t (&x)[NP]) {
 #pragma unroll
-        for (int p = 0; p < NP; ++p) win[p] = MUL ? mad_fma(qp[p], m, 0x8000u) : mad_fma(shl_clamp_hd(qp[p], r), sg, 0x8000u);
+        for (int p = 0; p < NP; ++p) win[p] = mad_fma(x[p], sg, 0x8000u);
     }
-    SA_HD void element_next(uint32_t r, uint32_t sg, const uint32_t* qp) {
-        const uint32_t m = MUL ? shl_clamp_hd(sg, r) : sg;
+    SA_HD void entry_next(uint32_t sg, const uint32_t (&x)[NP]) {
 #pragma unroll
-        for (int p = 0; p < NP; ++p) win[p] = MUL ? mad_fma(qp[p], m, win[p]) : mad_fma(shl_clamp_hd(qp[p], r), sg, win[p]);
+        for (int p = 0; p < NP; ++p) win[p] = mad_fma(x[p], sg, win[p]);
     }
     SA_HD void window_end() {
         ++n_windows;
@@ -151,46 +149,94 @@ struct PackedShift {
     }
 };
 
-// One 32-bit word of the byte container = 4 elements.  qp points at the packed queries of the
-// word's first element; consecutive elements are `stride` words apart.
-template <int NP, bool MUL>
-SA_HD void accumulate_word_bytes(PackedShift<NP, MUL>& pl, uint32_t w, const uint32_t* qp, int stride) {
-    // shift amounts g - 1 per byte: 0..6, and 0xff for the zero code (g = 0)
-    const uint32_t gw = w & 0x07070707u;
-    const uint32_t rw = (gw + 0x7f7f7f7fu) ^ 0x80808080u;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t r = prmt_hd(rw, 0u, 0x4440u | i);                          // byte i, zero-extended
-        const uint32_t sg = prmt_hd(w, 0u, 0x8888u | (0x1111u * i)) | 1u;         // top bit of byte i replicated, | 1
-        uint32_t q[NP];
-        load_np<NP>(qp + i * stride, q);
-        if (i == 0) pl.element_first(r, sg, q);
-        else pl.element_next(r, sg, q);
+// ---------------------------------------------------------------------------------------------
+// PoT-4 with the shifts hoisted out of the key loop.
+//
+// The shifted query q << r does not depend on the key, only on its exponent field: the block prepares
+// S[m][g][pair] = packed pair of element m shifted left by g - 1 (g = 1 .. 7; the entry of g = 0, the
+// zero code, is 0) once, in shared memory, and the key loop fetches the entry of ITS key's g — all
+// query pairs of the element with one vector load — and adds it with the sign (one multiply-add by
+// sigma on the FMA pipe per packed pair).  Per key element the ALU pipe then only sees two byte
+// permutes.  The row of one element holds 8 entries of 4 NP bytes: lanes with different g read
+// different banks, lanes with the same g the same address.  The windows, the bias and the totals are
+// those of PackedShift; the values added are bit for bit the ones it would have shifted itself.
+// ---------------------------------------------------------------------------------------------
+template <int NP>
+struct ShiftTable {
+    static constexpr int kEntryBytes = 4 * NP;             // the NP packed pairs of one (element, g)
+    static constexpr int kRowBytes = 8 * kEntryBytes;      // g = 0 .. 7: one element
+    static constexpr int kShift = NP == 4 ? 4 : NP == 2 ? 3 : 2;      // log2(kEntryBytes)
+    static_assert(NP == 1 || NP == 2 || NP == 4, "one, two or four packed query pairs");
+    // entry g of a packed pair
+    static SA_HD uint32_t entry(uint32_t packed, int g) { return g == 0 ? 0u : packed << (g - 1); }
+    // low address byte of element e (counted from a 256-byte aligned group start) before its g is added,
+    // and the rest of its offset
+    static SA_HD constexpr uint32_t low(int e) { return (uint32_t)(e * kRowBytes) & 0xffu; }
+    static SA_HD constexpr int high(int e) { return (e * kRowBytes) & ~0xff; }
+};
+
+// The NP words at (base with its low byte replaced by byte i of offs) + IMM.
+template <int NP, int IMM>
+SA_HD void shift_gather(uint32_t base, uint32_t offs, int i, uint32_t (&x)[NP]) {
+#ifdef __CUDA_ARCH__
+    const uint32_t addr = prmt_hd(offs, base, 0x7650u | (uint32_t)i);
+    if constexpr (NP == 4) asm("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4+%5];" : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]) : "r"(addr), "n"(IMM));
+    else if constexpr (NP == 2) asm("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(x[0]), "=r"(x[1]) : "r"(addr), "n"(IMM));
+    else asm("ld.shared.u32 %0, [%1+%2];" : "=r"(x[0]) : "r"(addr), "n"(IMM));
+#else
+    (void)base; (void)offs; (void)i;
+    for (int p = 0; p < NP; ++p) x[p] = 0u;      // shared-space addresses exist on the device only
+#endif
+}
+template <int NP, int IMM>
+SA_HD void shift_gather(const uint8_t* base, uint32_t offs, int i, uint32_t (&x)[NP]) {
+    const uintptr_t addr = (reinterpret_cast<uintptr_t>(base) & ~(uintptr_t)0xff) | ((offs >> (8 * i)) & 0xffu);
+    const uint32_t* e = reinterpret_cast<const uint32_t*>(addr + IMM);
+    for (int p = 0; p < NP; ++p) x[p] = e[p];
+}
+
+// Elements I .. 3 of one window: element E0 + STEP * I of the group, byte I of offs and of sw (sign at the
+// byte's top bit).
+template <int NP, int E0, int STEP, int I, typename Base>
+SA_HD void shift_window(PackedShift<NP>& pl, uint32_t sw, uint32_t offs, Base grp) {
+    if constexpr (I < 4) {
+        using ST = ShiftTable<NP>;
+        constexpr int e = E0 + STEP * I;
+        uint32_t x[NP];
+        shift_gather<NP, ST::high(e)>(grp, offs, I, x);
+        const uint32_t sg = mad_fma(prmt_hd(sw, 0u, 0x8888u | (0x1111u * I)), pl.one + pl.one, pl.one);   // +1 / -1
+        if (I == 0) pl.entry_first(sg, x);
+        else pl.entry_next(sg, x);
+        shift_window<NP, E0, STEP, I + 1>(pl, sw, offs, grp);
     }
+}
+
+// One 32-bit word of the byte container = 4 elements: word W4 (0 .. 3) of a group of 16 elements whose
+// table rows start at grp (256-byte aligned).
+template <int NP, int W4, typename Base>
+SA_HD void accumulate_word_bytes_tab(PackedShift<NP>& pl, uint32_t w, Base grp) {
+    using ST = ShiftTable<NP>;
+    constexpr uint32_t pattern = ST::low(W4 * 4) | (ST::low(W4 * 4 + 1) << 8) | (ST::low(W4 * 4 + 2) << 16) | (ST::low(W4 * 4 + 3) << 24);
+    const uint32_t offs = ((w << ST::kShift) & (0x07070707u << ST::kShift)) | pattern;      // g * entry bytes + row
+    shift_window<NP, W4 * 4, 1, 0>(pl, w, offs, grp);
     pl.window_end();
 }
 
-// One 32-bit word of the nibble container = 8 elements, two windows.
-template <int NP, bool MUL>
-SA_HD void accumulate_word_nibbles(PackedShift<NP, MUL>& pl, uint32_t w, const uint32_t* qp, int stride) {
-    const uint32_t ge = w & 0x07070707u, go = (w >> 4) & 0x07070707u;   // g of even / odd elements
-    const uint32_t re = (ge + 0x7f7f7f7fu) ^ 0x80808080u, ro = (go + 0x7f7f7f7fu) ^ 0x80808080u;
-    const uint32_t we = w << 4;                                         // even elements' sign at the byte's top bit
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int ni = half * 4 + i;                                // element within the word
-            const int byte = ni >> 1;
-            const uint32_t r = prmt_hd((ni & 1) ? ro : re, 0u, 0x4440u | byte);
-            const uint32_t sg = prmt_hd((ni & 1) ? w : we, 0u, 0x8888u | (0x1111u * byte)) | 1u;
-            uint32_t q[NP];
-            load_np<NP>(qp + ni * stride, q);
-            if (i == 0) pl.element_first(r, sg, q);
-            else pl.element_next(r, sg, q);
-        }
-        pl.window_end();
-    }
+// One 32-bit word of the nibble container = 8 elements (low nibble = even element), two windows: the even
+// and the odd elements (the order of the terms within the exact sum is free).  grp: the rows of the word's
+// first element (256-byte aligned).
+template <int NP, typename Base>
+SA_HD void accumulate_word_nibbles_tab(PackedShift<NP>& pl, uint32_t w, Base grp) {
+    using ST = ShiftTable<NP>;
+    constexpr uint32_t pat_e = ST::low(0) | (ST::low(2) << 8) | (ST::low(4) << 16) | (ST::low(6) << 24);
+    constexpr uint32_t pat_o = ST::low(1) | (ST::low(3) << 8) | (ST::low(5) << 16) | (ST::low(7) << 24);
+    const uint32_t we = w << 4;                                          // even elements' sign at the byte's top bit
+    const uint32_t offs_e = ((w << ST::kShift) & (0x07070707u << ST::kShift)) | pat_e;
+    const uint32_t offs_o = ((w >> (4 - ST::kShift)) & (0x07070707u << ST::kShift)) | pat_o;
+    shift_window<NP, 0, 2, 0>(pl, we, offs_e, grp);
+    pl.window_end();
+    shift_window<NP, 1, 2, 0>(pl, w, offs_o, grp);
+    pl.window_end();
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -38,11 +38,11 @@ struct DecodeSmem {
     static constexpr int NS = (D == 128 || KB == 4) ? 1 : kStages;
     static constexpr int kStageOff = 0;
     static constexpr int kMbarOff = NW * NS * Stage::kBytes;
-    // PoT-4: packed query pairs [D][NP]; INT8: D/4 x GT words of four queries; mantissa codes:
-    // the table of query multiples [D][NP][2^KB] x 8 bytes
-    static constexpr int kQpOff = (kMbarOff + 256 + 255) & ~255;   // the table datapath wants 256-byte alignment
+    // PoT-4: the shifted packed query pairs [D][8][NP]; INT8: D/4 x GT words of four queries; mantissa
+    // codes: the table of query multiples [D][NP][2^KB] x 8 bytes
+    static constexpr int kQpOff = (kMbarOff + 256 + 255) & ~255;   // the table datapaths want 256-byte alignment
     // (the prologue's scratch for the unpacked queries, D x GT words, uses the same space first)
-    static constexpr int kQpData = kTable ? D * NP * (8 << KB) : D * NP * 4;
+    static constexpr int kQpData = kTable ? D * NP * (8 << KB) : KB == 0 ? D * 8 * NP * 4 : D * NP * 4;
     static constexpr int kQpBytes = kQpData > D * GT * 4 ? kQpData : D * GT * 4;
     static constexpr int kQscaleOff = kQpOff + kQpBytes;
     // (The softmax weights of a tile need no space of their own: they overwrite the tile's key
@@ -67,7 +67,6 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     constexpr int WORDS = NIB ? D / 8 : D / 4;     // 32-bit code words per key
     constexpr int MT = D / 16;                     // 16-dim row tiles of O^T in the A.V phase
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint32_t (*qp_s)[NP] = reinterpret_cast<uint32_t (*)[NP]>(smem + SM::kQpOff);
     float* qscale_s = reinterpret_cast<float*>(smem + SM::kQscaleOff);
     int32_t (*q_s)[GT] = reinterpret_cast<int32_t (*)[GT]>(smem + SM::kQpOff);     // prologue only
     float (*red_s)[GT][D + 2] = reinterpret_cast<float (*)[GT][D + 2]>(smem + SM::kStageOff);
@@ -153,10 +152,20 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
         }
         __syncthreads();                                       // q_s is about to be overwritten
+        // S[m][g][pair] = the packed pair shifted by g - 1 (0 for g = 0); the entries of one pair are written
+        // starting at a g that depends on the element, so that the lanes of a warp use different banks
+        uint32_t* tab = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
 #pragma unroll
         for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
             const int idx = threadIdx.x + k * NT;
-            if (idx < D * NP) qp_s[idx / NP][idx % NP] = qp_reg[k];
+            const int m = idx / NP, p = idx % NP;
+            if (idx < D * NP) {
+#pragma unroll
+                for (int st = 0; st < 8; ++st) {
+                    const int g = (st + m) & 7;
+                    tab[(m * 8 + g) * NP + p] = ShiftTable<NP>::entry(qp_reg[k], g);
+                }
+            }
         }
     } else {
         // four consecutive elements of one query per word, in the byte order of the key words
@@ -331,13 +340,29 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)ts.score(g) << a.f_extra);   // exact: the true sum fits INT32
             } else if constexpr (KB != 8) {
-                PackedShift<NP, MUL> pl;
+                // PoT-4: the packed pairs, shifted ahead of the loop, are looked up by the key's exponent field
+                using ST = ShiftTable<NP>;
+                PackedShift<NP> pl;
                 pl.begin(a.one);
+                uint32_t grp = smem_addr(smem + SM::kQpOff);     // rows of the next group of elements (256-byte aligned)
+                if constexpr (!NIB) {
 #pragma unroll 1
-                for (int wq = 0; wq < WORDS; ++wq) {
-                    const uint32_t w = cw[(wq >> 2) * 128 + (wq & 3)];
-                    if constexpr (!NIB) accumulate_word_bytes(pl, w, &qp_s[wq * 4][0], NP);
-                    else accumulate_word_nibbles(pl, w, &qp_s[wq * 8][0], NP);
+                    for (int c = 0; c < D / 16; ++c, grp += 16 * ST::kRowBytes) {
+                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        accumulate_word_bytes_tab<NP, 0>(pl, w4.x, grp);
+                        accumulate_word_bytes_tab<NP, 1>(pl, w4.y, grp);
+                        accumulate_word_bytes_tab<NP, 2>(pl, w4.z, grp);
+                        accumulate_word_bytes_tab<NP, 3>(pl, w4.w, grp);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c, grp += 32 * ST::kRowBytes) {
+                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        accumulate_word_nibbles_tab<NP>(pl, w4.x, grp);
+                        accumulate_word_nibbles_tab<NP>(pl, w4.y, grp + 8 * ST::kRowBytes);
+                        accumulate_word_nibbles_tab<NP>(pl, w4.z, grp + 16 * ST::kRowBytes);
+                        accumulate_word_nibbles_tab<NP>(pl, w4.w, grp + 24 * ST::kRowBytes);
+                    }
                 }
 #pragma unroll
                 for (int g = 0; g < GT; ++g) A[g] = (int32_t)((uint32_t)pl.score(g) << a.f_extra);   // exact: the true sum fits INT32
@@ -528,13 +553,13 @@ static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
 template <int D, bool MUL>
 static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     if (p.nibble) {
-        if (p.k == 0) launch_gt<D, 0, true, MUL>(a, GT, grid, s);
+        if (p.k == 0) launch_gt<D, 0, true, false>(a, GT, grid, s);     // (PoT-4 has no MUL variant: the plan refuses it)
         else if (p.k == 1) launch_gt<D, 1, true, MUL>(a, GT, grid, s);       // dense planar container
         else launch_gt<D, 2, true, MUL>(a, GT, grid, s);
         return;
     }
     switch (p.k) {
-        case 0: launch_gt<D, 0, false, MUL>(a, GT, grid, s); break;
+        case 0: launch_gt<D, 0, false, false>(a, GT, grid, s); break;
         case 1: launch_gt<D, 1, false, MUL>(a, GT, grid, s); break;
         case 2: launch_gt<D, 2, false, MUL>(a, GT, grid, s); break;
         default: launch_gt<D, 4, false, MUL>(a, GT, grid, s); break;

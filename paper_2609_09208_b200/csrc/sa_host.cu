@@ -14,7 +14,8 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
     if (cfg->page_tokens != kPageTokens) return SA_ERR_UNSUPPORTED;
     if (cfg->flags & ~(SA_FLAG_HADAMARD | SA_FLAG_SHIFT_BY_MULTIPLY)) return SA_ERR_INVALID_ARG;
     p.mulshift = (cfg->flags & SA_FLAG_SHIFT_BY_MULTIPLY) != 0;
-    if (p.mulshift && (cfg->code == SA_KV_FP16 || cfg->code == SA_INT8)) return SA_ERR_UNSUPPORTED;   // no shift to move
+    // no shift in the key loop to move: FP16 and INT8 have none, PoT-4 looks its shifted queries up
+    if (p.mulshift && (cfg->code == SA_KV_FP16 || cfg->code == SA_INT8 || cfg->code == SA_POT4)) return SA_ERR_UNSUPPORTED;
     p.d = cfg->head_dim;
     p.Hq = cfg->n_q_heads;
     p.Hkv = cfg->n_kv_heads;

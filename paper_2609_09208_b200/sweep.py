@@ -130,7 +130,7 @@ def main():
         for code, nib in ([] if quick else [(0, True), (4, False)]):
             cell("cfg3 T=32768 B=%d %s%s shift-based A.V (N = k_max = 15)" % (B, names[code], "_nibble" if nib else ""),
                  [32768] * B, 32, 4, 64, code, nibble=nib, outliers=False, shiftav=True)
-        for code, nib in ([] if quick else [(0, True), (1, False), (4, False)]):
+        for code, nib in ([] if quick else [(1, False), (4, False)]):
             cell("cfg3 T=32768 B=%d %s%s shifts on the integer multiplier" % (B, names[code], "_nibble" if nib else ""),
                  [32768] * B, 32, 4, 64, code, nibble=nib, outliers=False, shift_by_multiply=True)
     lens4 = np.random.Generator(np.random.PCG64(4001)).integers(2048, 16385, size=16)

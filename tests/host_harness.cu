@@ -7,24 +7,31 @@ using namespace sa;
 
 // Scores of one PoT-4 key (canonical code bytes) against 8 queries, through the same packed
 // datapath and word decoders the decode kernel uses (byte container: phys_byte; nibbles: canonical nibble ^ 7).
-template <bool MUL>
 static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
-    alignas(16) static uint32_t qp[128][4];
+    using ST = ShiftTable<4>;
+    alignas(256) static uint8_t tab[128 * ST::kRowBytes];          // S[m][g][pair]: the shifted packed pairs
     for (int m = 0; m < d; ++m)
-        for (int p = 0; p < 4; ++p) qp[m][p] = pack_pair(q8[(2 * p) * d + m], q8[(2 * p + 1) * d + m]);
-    PackedShift<4, MUL> pl;
+        for (int g = 0; g < 8; ++g)
+            for (int p = 0; p < 4; ++p)
+                reinterpret_cast<uint32_t*>(tab)[(m * 8 + g) * 4 + p] =
+                    ST::entry(pack_pair(q8[(2 * p) * d + m], q8[(2 * p + 1) * d + m]), g);
+    PackedShift<4> pl;
     pl.begin(1u);
     if (!nibble_path) {
-        for (int m0 = 0; m0 < d; m0 += 4) {
-            uint32_t w = 0;
-            for (int i = 0; i < 4; ++i) w |= (uint32_t)phys_byte(canon[m0 + i]) << (8 * i);
-            accumulate_word_bytes(pl, w, &qp[m0][0], 4);
+        for (int m0 = 0; m0 < d; m0 += 16) {
+            uint32_t w[4] = {0, 0, 0, 0};
+            for (int i = 0; i < 16; ++i) w[i / 4] |= (uint32_t)phys_byte(canon[m0 + i]) << (8 * (i % 4));
+            const uint8_t* grp = tab + m0 * ST::kRowBytes;
+            accumulate_word_bytes_tab<4, 0>(pl, w[0], grp);
+            accumulate_word_bytes_tab<4, 1>(pl, w[1], grp);
+            accumulate_word_bytes_tab<4, 2>(pl, w[2], grp);
+            accumulate_word_bytes_tab<4, 3>(pl, w[3], grp);
         }
     } else {
         for (int m0 = 0; m0 < d; m0 += 8) {
             uint32_t w = 0;
             for (int i = 0; i < 8; ++i) w |= (uint32_t)((canon[m0 + i] ^ 0x70) >> 4) << (4 * i);
-            accumulate_word_nibbles(pl, w, &qp[m0][0], 4);
+            accumulate_word_nibbles_tab<4>(pl, w, (const uint8_t*)(tab + m0 * ST::kRowBytes));
         }
     }
     for (int g = 0; g < 8; ++g) out[g] = pl.score(g);
@@ -85,7 +92,7 @@ template <bool MUL>
 static void score8_any(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) {
     // path 0: byte container (packed datapath for k = 0, table datapath otherwise); 1: nibble container
     // (k = 0) or dense planar container (k = 1, 2)
-    if (k == 0) score8_packed<MUL>(canon, q8, d, path != 0, out);
+    if (k == 0) score8_packed(canon, q8, d, path != 0, out);            // PoT-4 has one datapath
     else if (path != 0 && k == 1) score8_planar<1, MUL>(canon, q8, d, out);
     else if (path != 0 && k == 2) score8_planar<2, MUL>(canon, q8, d, out);
     else if (k == 1) score8_table<1, MUL>(canon, q8, d, out);

@@ -84,9 +84,10 @@ def test_config_validation():
     bad = sa.make_config(64, 32, 4, sa.SA_POTM4)
     bad.flags = 8
     assert _status(sa.get_layout, bad) == 1
-    # the shift-by-multiply option exists for the power-of-two codes only
-    for code, nib in [(sa.SA_POT4, False), (sa.SA_POT4, True), (sa.SA_POTM1, True), (sa.SA_POTM2, False), (sa.SA_POTM4, False)]:
+    # the shift-by-multiply option exists for the mantissa codes only
+    for code, nib in [(sa.SA_POTM1, False), (sa.SA_POTM1, True), (sa.SA_POTM2, False), (sa.SA_POTM4, False)]:
         assert _status(sa.get_layout, sa.make_config(64, 32, 4, code, nibble=nib, shift_by_multiply=True)) == 0
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POT4, nibble=True, shift_by_multiply=True)) == 2
     assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_KV_FP16, shift_by_multiply=True)) == 2
     assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_INT8, shift_by_multiply=True)) == 2
     # head-room: F >= 6 + k (left shifts only), and the INT32 bound d*127*(2^(k+1)-1)*2^(F-k) < 2^31

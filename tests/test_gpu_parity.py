@@ -629,7 +629,7 @@ def test_config3_T32k_through_decode_step_in_a_cuda_graph(dev):
 
 # ------------------------------------------------------ shifts on the integer multiplier (non-default option)
 @pytest.mark.parametrize("d,Hq,Hkv", [(64, 32, 4), (128, 8, 2), (64, 6, 2)])
-@pytest.mark.parametrize("k,nibble", [(0, False), (0, True), (1, False), (1, True), (2, False), (2, True), (4, False)])
+@pytest.mark.parametrize("k,nibble", [(1, False), (1, True), (2, False), (2, True), (4, False)])
 def test_shift_by_multiply_gives_the_same_scores(dev, d, Hq, Hkv, k, nibble):
     """SA_FLAG_SHIFT_BY_MULTIPLY: INT32 scores bit-exact against the oracle (hence equal to the shift kernels'),
     outputs within the tolerance; ragged batch with an empty sequence, several tiles, head-room above the default."""

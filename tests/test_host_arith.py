@@ -111,7 +111,7 @@ def test_score_datapaths_equal_oracle_scores(hh, k, d):
                                     out.ctypes.data_as(C.c_void_p))
                 assert np.array_equal(out.astype(np.int64), want[:, 0]), ("planar", trial, out, want[:, 0])
         # the non-default kernels that run the shifts on the integer multiplier: the same integers again
-        for path in ((0, 1) if k in (0, 1, 2) else (0,)):
+        for path in (() if k == 0 else (0, 1) if k in (1, 2) else (0,)):
             hh.hh_score8_mul(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
                              C.c_int(path), out.ctypes.data_as(C.c_void_p))
             assert np.array_equal(out.astype(np.int64), want[:, 0]), ("shift by multiply", path, trial, out, want[:, 0])
