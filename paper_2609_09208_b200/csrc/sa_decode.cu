@@ -414,10 +414,13 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             float resc[GT];
             const float s_v = valid ? s_j : 0.0f, z_bias = valid ? 0.0f : -INFINITY;
             float pv[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};        // unused query columns stay zero
+            if (a.dbg_scores && valid) {                      // parity tests only: one branch around all the stores
+#pragma unroll
+                for (int g = 0; g < GT; ++g)
+                    a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
+            }
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
-                if (a.dbg_scores && valid)
-                    a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
                 // a lane without a key gets z = -inf through the addend (the product is rounded once either way)
                 const float z = fmaf((float)A[g] * qscale_s[g], s_v, z_bias);
                 // ceil of the tile's largest logit: ceil is monotone, so take the integer maximum (the
