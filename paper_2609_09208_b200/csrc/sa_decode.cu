@@ -427,7 +427,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 // conversion saturates; a lane without a key gives the smallest integer)
                 const int Mt = max(warp_max_s32(__float2int_ru(z)), -(1 << 28));
                 const int Mn = max(M[g], Mt);
-                resc[g] = (M[g] == kMNone) ? 0.0f : pow2i_neg(M[g] - Mn);          // exact power of two
+                resc[g] = pow2i_neg(M[g] - Mn);               // exact power of two; 0 while M is still "no key seen" (-2^29)
                 changed |= (Mn != M[g]);
                 M[g] = Mn;
                 const float p = ex2_approx(z - (float)Mn);     // 2^-inf = 0 for a lane without a key
