@@ -53,8 +53,11 @@ struct DecodeSmem {
     static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
 };
 
-template <int D, int KB, bool NIB, int GT, bool MUL = false>
+template <int D, int KB, bool NIB, int GT, int MODE = 0>
 __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM)) decode_kernel(DecodeArgs a) {
+    // MODE 0: the decode kernel; 1: the same with SA_FLAG_SHIFT_BY_MULTIPLY; 2: the score pass of the shift-based
+    // A.V option (a.zr set: rounded logits and statistics instead of softmax and A.V), kept out of the other two
+    constexpr bool MUL = (MODE == 1), SP = (MODE == 2);
     // KB = 0: PoT-4 (packed shift datapath); KB = 1, 2, 4: mantissa codes (table datapath);
     // KB = 8: uniform INT8 comparison code (dp4a).  MUL: the shifts run on the integer multiplier
     // (SA_FLAG_SHIFT_BY_MULTIPLY; same scores, reported separately from the shift kernels).
@@ -225,7 +228,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     const int n_my = first < tile1 ? (tile1 - first + NW - 1) / NW : 0;
     if (tile_new >= first && tile_new < tile1 && (tile_new - first) % NW == 0) {      // warp-uniform: this warp owns that tile
         // encode / quantise the token and write it into its page before the tile is copied to shared memory
-        constexpr int MODE = (KB == 8) ? 32 : (NIB ? 8 + KB : KB);
+        constexpr int WMODE = (KB == 8) ? 32 : (NIB ? 8 + KB : KB);
         CacheArgs ca{};
         ca.kcode_off = a.kcode_off;
         ca.meta_off = a.meta_off;
@@ -234,7 +237,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         ca.hadamard = a.hadamard;
         uint8_t* block = const_cast<uint8_t*>(a.pages) + ((size_t)pidx_new * a.Hkv + kvh) * a.page_bytes;
         const size_t row = ((size_t)b * a.Hkv + kvh) * D;
-        write_token<D, MODE>(block, ca, (len - 1) % kPageTokens, lane, a.Knew + row, a.Vnew + row);
+        write_token<D, WMODE>(block, ca, (len - 1) % kPageTokens, lane, a.Knew + row, a.Vnew + row);
         fence_proxy_async_global();
         __syncwarp();
     }
@@ -387,7 +390,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             const float s_j = half_bits_to_float(meta & 0xffffu);
             const int g_j = (int)(int8_t)((meta >> 16) & 0xffu);
             const float vscale = valid ? pow2i(-g_j) : 0.0f;  // 2^-g_j; g_j in [-10, 30] for written tokens
-            if (a.zr) {
+            if constexpr (SP) {
                 // Score pass of the shift-based A.V option (eq. (6)): store the rounded logits and keep
                 // the ceiling of the largest one and the smallest value exponent; no softmax, no A.V here.
 #pragma unroll
@@ -503,7 +506,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 
     // ---- merge the warps of the block, write the block's partial ----
     __syncthreads();                                           // the merge scratch re-uses the stage buffers
-    if (a.zr) {
+    if constexpr (SP) {
         // score pass of the shift-A.V option: the block's statistics instead of a partial
         int* stat_s = reinterpret_cast<int*>(smem + SM::kStageOff);           // [NW][GT + 1]
         g_min = warp_min_s32(g_min);
@@ -531,49 +534,51 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 
 using namespace sa;
 
-template <int D, int KB, bool NIB, int GT, bool MUL>
+template <int D, int KB, bool NIB, int GT, int MODE>
 static void launch_one(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
     constexpr int bytes = DecodeSmem<D, KB, NIB, GT>::kBytes;
     if (bytes > 48 * 1024) {
         // opt in to more than 48 KB of dynamic shared memory (an attribute of the function; no allocation)
-        static const cudaError_t once = cudaFuncSetAttribute(decode_kernel<D, KB, NIB, GT, MUL>,
+        static const cudaError_t once = cudaFuncSetAttribute(decode_kernel<D, KB, NIB, GT, MODE>,
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
         (void)once;
     }
-    (void)launch_pdl(decode_kernel<D, KB, NIB, GT, MUL>, grid, dim3(32 * DecodeSmem<D, KB, NIB, GT>::NW), (size_t)bytes, s, a);
+    (void)launch_pdl(decode_kernel<D, KB, NIB, GT, MODE>, grid, dim3(32 * DecodeSmem<D, KB, NIB, GT>::NW), (size_t)bytes, s, a);
 }
 
-template <int D, int KB, bool NIB, bool MUL>
+template <int D, int KB, bool NIB, int MODE>
 static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     switch (GT) {
-        case 8: launch_one<D, KB, NIB, 8, MUL>(a, grid, s); break;
-        case 4: launch_one<D, KB, NIB, 4, MUL>(a, grid, s); break;
-        case 2: launch_one<D, KB, NIB, 2, MUL>(a, grid, s); break;
-        default: launch_one<D, KB, NIB, 1, MUL>(a, grid, s); break;
+        case 8: launch_one<D, KB, NIB, 8, MODE>(a, grid, s); break;
+        case 4: launch_one<D, KB, NIB, 4, MODE>(a, grid, s); break;
+        case 2: launch_one<D, KB, NIB, 2, MODE>(a, grid, s); break;
+        default: launch_one<D, KB, NIB, 1, MODE>(a, grid, s); break;
     }
 }
 
-template <int D, bool MUL>
+template <int D, int MODE>
 static void launch_code(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
+    constexpr int kPot4Mode = (MODE == 1) ? 0 : MODE;      // PoT-4 has no multiply variant (the plan refuses it)
     if (p.nibble) {
-        if (p.k == 0) launch_gt<D, 0, true, false>(a, GT, grid, s);     // (PoT-4 has no MUL variant: the plan refuses it)
-        else if (p.k == 1) launch_gt<D, 1, true, MUL>(a, GT, grid, s);       // dense planar container
-        else launch_gt<D, 2, true, MUL>(a, GT, grid, s);
+        if (p.k == 0) launch_gt<D, 0, true, kPot4Mode>(a, GT, grid, s);
+        else if (p.k == 1) launch_gt<D, 1, true, MODE>(a, GT, grid, s);      // dense planar container
+        else launch_gt<D, 2, true, MODE>(a, GT, grid, s);
         return;
     }
     switch (p.k) {
-        case 0: launch_gt<D, 0, false, false>(a, GT, grid, s); break;
-        case 1: launch_gt<D, 1, false, MUL>(a, GT, grid, s); break;
-        case 2: launch_gt<D, 2, false, MUL>(a, GT, grid, s); break;
-        default: launch_gt<D, 4, false, MUL>(a, GT, grid, s); break;
+        case 0: launch_gt<D, 0, false, kPot4Mode>(a, GT, grid, s); break;
+        case 1: launch_gt<D, 1, false, MODE>(a, GT, grid, s); break;
+        case 2: launch_gt<D, 2, false, MODE>(a, GT, grid, s); break;
+        default: launch_gt<D, 4, false, MODE>(a, GT, grid, s); break;
     }
 }
 
 template <int D>
 static void launch_dim(const Plan& p, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
-    if (p.int8) launch_gt<D, 8, false, false>(a, GT, grid, s);
-    else if (p.mulshift) launch_code<D, true>(p, a, GT, grid, s);
-    else launch_code<D, false>(p, a, GT, grid, s);
+    if (p.int8) launch_gt<D, 8, false, 0>(a, GT, grid, s);
+    else if (a.zr) launch_code<D, 2>(p, a, GT, grid, s);         // score pass of the shift-based A.V option
+    else if (p.mulshift) launch_code<D, 1>(p, a, GT, grid, s);
+    else launch_code<D, 0>(p, a, GT, grid, s);
 }
 
 namespace sa {
