@@ -295,6 +295,18 @@ def test_query_group_sizes(dev, Hq, Hkv):
     check_against_oracle(case, O, dbg)
 
 
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("nibble", [False, True])
+@pytest.mark.parametrize("Hq,Hkv", [(1, 1), (2, 1), (3, 1), (8, 2), (12, 1), (16, 2)])
+def test_pot4_query_group_sizes(dev, Hq, Hkv, nibble, d):
+    """PoT-4 looks its shifted packed query pairs up in a table whose rows hold 1, 2 or 4 pairs (groups of 1-2, 3-4,
+    5-8 query heads per block) with a different address pattern each: every row width, both containers, both head
+    dimensions, an odd group (a pair with one query) and a group wider than one block."""
+    case = synth.make_case("gqa4", [300, 77, 1], Hq, Hkv, d, 0, outliers=True, nibble=nibble, seed=1650 + Hq + d)
+    O, dbg, _ = run_decode(case, dev, permute_seed=3)
+    check_against_oracle(case, O, dbg)
+
+
 @pytest.mark.parametrize("k,F", [(0, 7), (0, 18), (1, 9), (4, 12), (4, 16)])
 def test_headroom_F(dev, k, F):
     # F = 7 with PoT-4 is the paper's worked bound (d * 127 * 2^7); larger F only shifts the exact integer
