@@ -37,17 +37,19 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
         for (int i = 0; i < EPL; ++i) kc[i] = NIB ? (uint8_t)(kc[i] ^ 0x70) : phys_byte(kc[i]);
     }
     const int gg = quantise_value_vec<EPL>(vb, vc);
+    block += (size_t)(t >> 5) * (a.page_bytes >> 1);          // the token's half of the page; offsets are within a half
+    t &= 31;
     uint8_t* kdst = block + a.kcode_off;
     if (!NIB) {
         const int m = lane * EPL;                   // first element of this lane
-        store_bytes<EPL>(kdst + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15), kc);
+        store_bytes<EPL>(kdst + ((size_t)(m >> 4) * kTileTokens + t) * 16 + (m & 15), kc);
     } else {
         // two elements per byte: low nibble = even element, high nibble = odd element
         uint8_t nb[EPL / 2];
 #pragma unroll
         for (int i = 0; i < EPL / 2; ++i) nb[i] = (uint8_t)((kc[2 * i] >> 4) | (kc[2 * i + 1] & 0xf0));
         const int m = lane * EPL;
-        store_bytes<EPL / 2>(kdst + ((size_t)(m >> 5) * kPageTokens + t) * 16 + ((m & 31) >> 1), nb);
+        store_bytes<EPL / 2>(kdst + ((size_t)(m >> 5) * kTileTokens + t) * 16 + ((m & 31) >> 1), nb);
         if constexpr (K > 0 && K < 8) {
             // dense planar container: mantissa bit b of element m goes to bit m % 8 of byte m / 8 of plane b.
             // A lane holds EPL consecutive elements, so 8 / EPL lanes share a byte; lane B assembles byte B.
@@ -63,14 +65,14 @@ SA_D void write_token_quant(uint8_t* block, const CacheArgs& a, int t, int lane,
                     for (int l = 0; l < LPB; ++l)
 #pragma unroll
                         for (int i = 0; i < EPL; ++i) byte |= ((mask[i] >> (LPB * lane + l)) & 1u) << (EPL * l + i);
-                    block[a.plane_off + ((size_t)bit * kPageTokens + t) * (D / 8) + lane] = (uint8_t)byte;
+                    block[a.plane_off + ((size_t)bit * kTileTokens + t) * (D / 8) + lane] = (uint8_t)byte;
                 }
             }
         }
     }
     {
-        const int mv = lane * EPL;                  // values: 16-dim chunks, chunk c of token t at (c * 64 + t) * 16
-        store_bytes<EPL>(block + a.v_off + ((size_t)(mv >> 4) * kPageTokens + t) * 16 + (mv & 15), vc);
+        const int mv = lane * EPL;                  // values: 16-dim chunks, chunk c of token t at (c * 32 + t) * 16 within the half
+        store_bytes<EPL>(block + a.v_off + ((size_t)(mv >> 4) * kTileTokens + t) * 16 + (mv & 15), vc);
     }
     if (lane == 0)
         *reinterpret_cast<uint32_t*>(block + a.meta_off + (size_t)t * 4) = (smax & 0xffffu) | ((uint32_t)(uint8_t)(int8_t)gg << 16);
@@ -84,7 +86,9 @@ SA_D void write_token_fp16(uint8_t* block, const CacheArgs& a, int t, int lane, 
     load_vec_bits<EPL>(krow, lane, kb);
     load_vec_bits<EPL>(vrow, lane, vb);
     const int m = lane * EPL;                        // K and V both in 16-byte chunks of 8 elements
-    const size_t off = ((size_t)(m >> 3) * kPageTokens + t) * 16 + (size_t)(m & 7) * 2;
+    block += (size_t)(t >> 5) * (a.page_bytes >> 1);          // the token's half of the page
+    t &= 31;
+    const size_t off = ((size_t)(m >> 3) * kTileTokens + t) * 16 + (size_t)(m & 7) * 2;
     uint16_t* kdst = reinterpret_cast<uint16_t*>(block + a.kcode_off + off);
     uint16_t* vdst = reinterpret_cast<uint16_t*>(block + a.v_off + off);
 #pragma unroll

@@ -14,6 +14,14 @@
 namespace sa {
 
 constexpr int kPageTokens = 64;
+constexpr int kTileTokens = 32;           // a page block is two halves of 32 tokens, each laid out like one staged tile
+// Bytes of one half of a (page, KV head) block: code chunks, mantissa bit planes (dense planar container),
+// metadata, value chunks.  kb: mantissa bits (8 for the INT8 comparison code); nib: sub-byte container.
+// The page plan (make_plan) and the kernels' stage plans are both checked against it.
+constexpr int half_block_bytes(int d, int kb, bool nib) {
+    return kTileTokens * (nib ? d / 2 : d) + ((nib && kb > 0) ? kb * kTileTokens * (d / 8) : 0) + kTileTokens * 4 + kTileTokens * d;
+}
+constexpr int half_block_bytes_fp16(int d) { return 2 * kTileTokens * d * 2; }
 constexpr int kNumSMs = 148;              // B200
 constexpr int kEmax = 6;                  // largest exponent of the 3-bit field
 constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no key seen yet"

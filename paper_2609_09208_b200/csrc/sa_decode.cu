@@ -51,6 +51,7 @@ struct DecodeSmem {
     static constexpr int kBlocksPerSM = decode_shape(D, KB).blocks_per_sm;
     static_assert(NW * GT * (D + 2) * 4 <= NW * NS * Stage::kBytes && NW * NS * 8 <= 256, "merge scratch must fit in the stage buffers");
     static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
+    static_assert(Stage::kBytes == half_block_bytes(D, KB, NIB), "a stage buffer is a verbatim copy of half a page block");
 };
 
 template <int D, int KB, bool NIB, int GT, int MODE = 0>
@@ -201,8 +202,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         if (tile_g < (int)((long long)n_tiles_g * (split + 1) / a.n_splits)) {
             const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
             if (pidx_g >= 0 && pidx_g < a.n_pages)
-                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, a.kcode_off, a.meta_off, a.v_off,
-                                (tile_g & 1) * 32, a.zr == nullptr, a.plane_off);
+                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, (tile_g & 1) * 32, !SP);
         }
     }
     pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
@@ -230,6 +230,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         // encode / quantise the token and write it into its page before the tile is copied to shared memory
         constexpr int WMODE = (KB == 8) ? 32 : (NIB ? 8 + KB : KB);
         CacheArgs ca{};
+        ca.page_bytes = a.page_bytes;
         ca.kcode_off = a.kcode_off;
         ca.meta_off = a.meta_off;
         ca.v_off = a.v_off;
@@ -251,9 +252,8 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             mbar_arrive(mbar0 + s * 8);
         } else {
             const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
-            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
-                         mbar0 + s * 8, true, a.zr == nullptr,    // the score pass of the shift-A.V option needs no values
-                         a.plane_off);
+            Stage::issue(stage0 + s * Stage::kBytes, block, (tile & 1) * 32, mbar0 + s * 8, true,
+                         !SP);                                    // the score pass of the shift-A.V option needs no values
         }
     };
     if (lane == 0)

@@ -25,27 +25,22 @@ SA_D uint32_t pack_half2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Stage buffer of one 32-key tile: K chunks [D/8][32 keys][16 B], then V chunks [D/8][32 keys][16 B].
+// Stage buffer of one 32-key tile = one half of a page block: K chunks [D/8][32 keys][16 B], then V chunks
+// [D/8][32 keys][16 B].
 template <int D>
 struct Fp16Stage {
     static constexpr int kChunks = D / 8;
     static constexpr int kVOff = kChunks * 512;
     static constexpr int kBytes = 2 * kChunks * 512;
-    SA_D static void issue(uint32_t dst, const uint8_t* block, size_t k_off, size_t v_off, int tk0, uint32_t mbar) {
+    static_assert(kBytes == half_block_bytes_fp16(D), "a stage buffer is a verbatim copy of half a page block");
+    // tk0 = 0 or 32: the tile is that half of the (page, KV head) block, laid out like the stage buffer: one copy
+    SA_D static void issue(uint32_t dst, const uint8_t* block, int tk0, uint32_t mbar) {
         mbar_arrive_expect_tx(mbar, (uint32_t)kBytes);
-#pragma unroll
-        for (int c = 0; c < kChunks; ++c)
-            bulk_g2s(dst + c * 512, block + k_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
-#pragma unroll
-        for (int c = 0; c < kChunks; ++c)
-            bulk_g2s(dst + kVOff + c * 512, block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
+        bulk_g2s(dst, block + (size_t)(tk0 >> 5) * kBytes, (uint32_t)kBytes, mbar);
     }
-    // the same ranges as L2 prefetch hints
-    SA_D static void prefetch(const uint8_t* block, size_t k_off, size_t v_off, int tk0) {
-#pragma unroll
-        for (int c = 0; c < kChunks; ++c) bulk_prefetch_l2(block + k_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
-#pragma unroll
-        for (int c = 0; c < kChunks; ++c) bulk_prefetch_l2(block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
+    // the same range as an L2 prefetch hint
+    SA_D static void prefetch(const uint8_t* block, int tk0) {
+        bulk_prefetch_l2(block + (size_t)(tk0 >> 5) * kBytes, (uint32_t)kBytes);
     }
 };
 
@@ -110,7 +105,7 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         if (tile_g < (int)((long long)n_tiles_g * (split + 1) / a.n_splits)) {
             const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
             if (pidx_g >= 0 && pidx_g < a.n_pages)
-                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, a.kcode_off, a.v_off, (tile_g & 1) * 32);
+                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, (tile_g & 1) * 32);
         }
     }
     pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
@@ -133,6 +128,7 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
     if (tile_new >= first && tile_new < tile1 && (tile_new - first) % 4 == 0) {      // this warp owns that tile
         CacheArgs ca{};
+        ca.page_bytes = a.page_bytes;
         ca.kcode_off = a.kcode_off;
         ca.v_off = a.v_off;
         uint8_t* block = const_cast<uint8_t*>(a.pages) + ((size_t)pidx_new * a.Hkv + kvh) * a.page_bytes;
@@ -149,7 +145,7 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
             mbar_arrive(mbar0 + s * 8);
         } else {
             const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
-            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.v_off, (tile & 1) * 32, mbar0 + s * 8);
+            Stage::issue(stage0 + s * Stage::kBytes, block, (tile & 1) * 32, mbar0 + s * 8);
         }
     };
     if (lane == 0)

@@ -117,16 +117,17 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
     const int tt = (int)(v / a.Hkv), h = (int)(v % a.Hkv);
     const uint8_t* block = page_block(a, b, tt / kPageTokens, h);
     if (!block) return;
-    const int t = tt % kPageTokens;
+    block += (size_t)((tt % kPageTokens) >> 5) * (a.page_bytes >> 1);      // the token's half of the page
+    const int t = tt & 31;
     const int m = lane * EPL;
     if (codes) {
         uint8_t c[EPL];
         if (!NIB) {
-            const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15);
+            const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 4) * kTileTokens + t) * 16 + (m & 15);
 #pragma unroll
             for (int i = 0; i < EPL; ++i) c[i] = xor_mask ? canon_byte(src[i]) : src[i];   // power-of-two codes / INT8 stored as is
         } else {
-            const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 5) * kPageTokens + t) * 16 + ((m & 31) >> 1);
+            const uint8_t* src = block + a.kcode_off + ((size_t)(m >> 5) * kTileTokens + t) * 16 + ((m & 31) >> 1);
 #pragma unroll
             for (int i = 0; i < EPL / 2; ++i) {
                 c[2 * i] = (uint8_t)((src[i] << 4) ^ 0x70);
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
             }
             // dense planar container: the canonical mantissa is left-aligned in the low nibble
             for (int bit = 0; bit < planes; ++bit) {
-                const uint8_t* pl = block + a.plane_off + ((size_t)bit * kPageTokens + t) * (D / 8);
+                const uint8_t* pl = block + a.plane_off + ((size_t)bit * kTileTokens + t) * (D / 8);
 #pragma unroll
                 for (int i = 0; i < EPL; ++i) c[i] |= (uint8_t)(((pl[(m + i) >> 3] >> ((m + i) & 7)) & 1u) << (4 - planes + bit));
             }
@@ -142,7 +143,7 @@ __global__ void __launch_bounds__(128) unpack_kernel(CacheArgs a, int b, int T, 
         store_bytes<EPL>(codes + (size_t)v * D + m, c);
     }
     if (vhat) {
-        const uint8_t* src = block + a.v_off + ((size_t)(m >> 4) * kPageTokens + t) * 16 + (m & 15);
+        const uint8_t* src = block + a.v_off + ((size_t)(m >> 4) * kTileTokens + t) * 16 + (m & 15);
         uint8_t c[EPL];
 #pragma unroll
         for (int i = 0; i < EPL; ++i) c[i] = src[i];

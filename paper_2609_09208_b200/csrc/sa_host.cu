@@ -30,9 +30,10 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
         p.F = 0;
         p.f_extra = 0;
         p.lay.kcode_off = 0;
-        p.lay.meta_off = (size_t)kPageTokens * p.d * 2;   // empty metadata block
+        p.lay.meta_off = (size_t)kTileTokens * p.d * 2;   // empty metadata block
         p.lay.v_off = p.lay.meta_off;
-        p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d * 2;
+        p.lay.page_bytes = 2 * (p.lay.v_off + (size_t)kTileTokens * p.d * 2);
+        if (p.lay.page_bytes != 2 * (size_t)half_block_bytes_fp16(p.d)) return SA_ERR_UNSUPPORTED;
         p.lay.align = 256;
         *out = p;
         return SA_OK;
@@ -44,9 +45,10 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
         p.F = 0;
         p.f_extra = 0;
         p.lay.kcode_off = 0;
-        p.lay.meta_off = (size_t)kPageTokens * p.d;
-        p.lay.v_off = p.lay.meta_off + (size_t)kPageTokens * 4;
-        p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d;
+        p.lay.meta_off = (size_t)kTileTokens * p.d;
+        p.lay.v_off = p.lay.meta_off + (size_t)kTileTokens * 4;
+        p.lay.page_bytes = 2 * (p.lay.v_off + (size_t)kTileTokens * p.d);
+        if (p.lay.page_bytes != 2 * (size_t)half_block_bytes(p.d, 8, false)) return SA_ERR_UNSUPPORTED;
         p.lay.align = 256;
         *out = p;
         return SA_OK;
@@ -71,11 +73,13 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
     if (bound >= (1LL << 31)) return SA_ERR_UNSUPPORTED;
     p.f_extra = p.F - p.k - kEmax;
     const size_t kbytes = p.nibble ? (size_t)p.d / 2 : (size_t)p.d;
+    // offsets within one 32-token half of the block; the second half follows the first
     p.lay.kcode_off = 0;
-    p.plane_off = (size_t)kPageTokens * kbytes;                 // k bit planes of d / 8 bytes per token (planar only)
-    p.lay.meta_off = p.plane_off + (p.nibble ? (size_t)p.k * kPageTokens * (p.d / 8) : 0);
-    p.lay.v_off = p.lay.meta_off + (size_t)kPageTokens * 4;
-    p.lay.page_bytes = p.lay.v_off + (size_t)kPageTokens * p.d;
+    p.plane_off = (size_t)kTileTokens * kbytes;                 // k bit planes of d / 8 bytes per token (planar only)
+    p.lay.meta_off = p.plane_off + (p.nibble ? (size_t)p.k * kTileTokens * (p.d / 8) : 0);
+    p.lay.v_off = p.lay.meta_off + (size_t)kTileTokens * 4;
+    p.lay.page_bytes = 2 * (p.lay.v_off + (size_t)kTileTokens * p.d);
+    if (p.lay.page_bytes != 2 * (size_t)half_block_bytes(p.d, p.k, p.nibble)) return SA_ERR_UNSUPPORTED;   // the kernels' stage plans
     p.lay.align = 256;
     *out = p;
     return SA_OK;

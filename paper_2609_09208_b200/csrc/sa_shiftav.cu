@@ -82,8 +82,7 @@ __global__ void __launch_bounds__(128) shiftav_kernel(DecodeArgs a) {
             mbar_arrive(mbar0 + s * 8);
         } else {
             const uint8_t* block = a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes;
-            Stage::issue(stage0 + s * Stage::kBytes, block, a.kcode_off, a.meta_off, a.v_off, (tile & 1) * 32,
-                         mbar0 + s * 8, false, true);
+            Stage::issue_values(stage0 + s * Stage::kBytes, block, a.page_bytes, a.meta_off, (tile & 1) * 32, mbar0 + s * 8);
         }
     };
     if (lane == 0)

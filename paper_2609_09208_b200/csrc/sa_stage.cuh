@@ -1,8 +1,8 @@
 // Shared-memory staging of 32-token tiles with bulk-async (TMA, 1-D) copies and mbarriers.
 //
-// Each warp owns a small ring of stage buffers.  Lane 0 issues, for one tile, one bulk copy per
-// 16-byte code chunk (the page layout keeps chunk c of 32 consecutive tokens in 512 contiguous
-// bytes), one for the metadata and one for the value rows; all of them complete on the stage's
+// Each warp owns a small ring of stage buffers.  Lane 0 issues, for one tile, one bulk copy: a page
+// block is two 32-token halves, each holding its code chunks, mantissa planes, metadata and value
+// chunks one after another exactly as the stage buffer does.  It completes on the stage's
 // mbarrier, which the whole warp then polls.  Every wait is bounded: after kWaitLimit unsuccessful
 // polls the caller poisons its result with NaN and leaves its loop instead of spinning on.
 // Copies are plain (no cluster qualifier): every block stages its own tiles.
@@ -74,42 +74,29 @@ struct TileStage {
     static constexpr int kVBytes = 32 * VROW_BYTES;
     static constexpr int kBytes = kVOff + kVBytes;            // a multiple of 128
 
-    // Issued by one lane.  `block` is the (page, KV head) block, tk0 the tile's first token (0 or 32).
-    // with_codes / with_values: which parts of the tile the caller needs (at least one of them).
-    SA_D static void issue(uint32_t dst, const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off,
-                           int tk0, uint32_t mbar, bool with_codes = true, bool with_values = true,
-                           size_t plane_off = 0) {
-        mbar_arrive_expect_tx(mbar, (uint32_t)((with_codes ? kCodeBytes + PLANES * kPlaneBytes : 0) + kMetaBytes +
-                                               (with_values ? kVBytes : 0)));
-        if (with_codes) {
-#pragma unroll
-            for (int c = 0; c < CHUNKS; ++c)
-                bulk_g2s(dst + c * 512, block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
-#pragma unroll
-            for (int b = 0; b < PLANES; ++b)
-                bulk_g2s(dst + kPlaneOff + b * kPlaneBytes, block + plane_off + ((size_t)b * kPageTokens + tk0) * PLANE_ROW,
-                         (uint32_t)kPlaneBytes, mbar);
-        }
-        if (HAS_META) bulk_g2s(dst + kMetaOff, block + meta_off + (size_t)tk0 * 4, 128u, mbar);
-        if (with_values) {
-#pragma unroll
-            for (int c = 0; c < VROW_BYTES / 16; ++c)
-                bulk_g2s(dst + kVOff + c * 512, block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u, mbar);
-        }
+    // Issued by one lane.  `block` is the (page, KV head) block, tk0 the tile's first token (0 or 32): the
+    // tile is that half of the block, which is laid out exactly like the stage buffer, so it is one copy.
+    // with_codes / with_values: which parts of the tile the caller needs (at least one of them); the
+    // metadata sits between the two and comes with either.
+    SA_D static void issue(uint32_t dst, const uint8_t* block, int tk0, uint32_t mbar, bool with_codes = true,
+                           bool with_values = true) {
+        const uint8_t* half = block + (size_t)(tk0 >> 5) * kBytes;
+        const uint32_t lo = with_codes ? 0u : (uint32_t)kMetaOff;
+        const uint32_t hi = with_values ? (uint32_t)kBytes : (uint32_t)kVOff;
+        mbar_arrive_expect_tx(mbar, hi - lo);
+        bulk_g2s(dst + lo, half + lo, hi - lo, mbar);
     }
-    // The same ranges as issue(), as L2 prefetch hints.
-    SA_D static void prefetch(const uint8_t* block, size_t kcode_off, size_t meta_off, size_t v_off, int tk0,
-                              bool with_values, size_t plane_off) {
-#pragma unroll
-        for (int c = 0; c < CHUNKS; ++c) bulk_prefetch_l2(block + kcode_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
-#pragma unroll
-        for (int b = 0; b < PLANES; ++b)
-            bulk_prefetch_l2(block + plane_off + ((size_t)b * kPageTokens + tk0) * PLANE_ROW, (uint32_t)kPlaneBytes);
-        if (HAS_META) bulk_prefetch_l2(block + meta_off + (size_t)tk0 * 4, 128u);
-        if (with_values) {
-#pragma unroll
-            for (int c = 0; c < VROW_BYTES / 16; ++c) bulk_prefetch_l2(block + v_off + ((size_t)c * kPageTokens + tk0) * 16, 512u);
-        }
+    // Metadata and values only, for a stage plan without code chunks (CHUNKS = 0, PLANES = 0) reading a block
+    // whose halves do hold codes: the two parts follow one another from meta_off to the end of the half.
+    SA_D static void issue_values(uint32_t dst, const uint8_t* block, size_t page_bytes, size_t meta_off, int tk0,
+                                  uint32_t mbar) {
+        static_assert(CHUNKS == 0 && PLANES == 0, "the stage holds metadata and values only");
+        mbar_arrive_expect_tx(mbar, (uint32_t)kBytes);
+        bulk_g2s(dst, block + (size_t)(tk0 >> 5) * (page_bytes >> 1) + meta_off, (uint32_t)kBytes, mbar);
+    }
+    // The same range as issue(), as an L2 prefetch hint.
+    SA_D static void prefetch(const uint8_t* block, int tk0, bool with_values) {
+        bulk_prefetch_l2(block + (size_t)(tk0 >> 5) * kBytes, with_values ? (uint32_t)kBytes : (uint32_t)kVOff);
     }
 };
 
