@@ -29,19 +29,21 @@
  *
  * Cache layout (this library's own; section II-F only fixes what is stored)
  *   The page pool is n_pages * n_kv_heads blocks of `page_bytes`; block (p, h) starts at
- *   ((size_t)p * n_kv_heads + h) * page_bytes and holds page_tokens = 64 tokens of KV head h:
- *     kcode_off: key codes in 16-byte chunks, chunk c of token t at (c * 64 + t) * 16.
+ *   ((size_t)p * n_kv_heads + h) * page_bytes and holds page_tokens = 64 tokens of KV head h as two
+ *   halves of page_bytes / 2 bytes, tokens 0..31 and 32..63.  A half is what a decode kernel stages for
+ *   one 32-key tile, with a single bulk copy; the offsets below are relative to the half, t = token % 32:
+ *     kcode_off: key codes in 16-byte chunks, chunk c of token t at (c * 32 + t) * 16.
  *                Byte container (any k): chunk c holds elements 16c .. 16c+15, one byte each:
  *                sign << 7 | mantissa field << 3 | g, with the canonical byte's 4-bit mantissa
  *                field and g = 7 - e (g = 0 for the zero code), so that g - 1 is the shift amount,
  *                the mantissa field times 8 a table offset, and zeroed memory reads as zero codes.  Nibble container (PoT-4 only): chunk c holds
  *                elements 32c .. 32c+31, byte i = element 32c+2i in the low nibble and 32c+2i+1
  *                in the high nibble, nibble = sign << 3 | g.
- *     meta_off : 64 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.
+ *     meta_off : 32 records of 4 bytes: binary16 s_j, int8 g_j, one zero byte.
  *     v_off    : vhat, int8, in 16-byte chunks like the keys: chunk c (dims 16c .. 16c+15) of token t
- *                at (c * 64 + t) * 16.
- *   For code = SA_KV_FP16 the block holds unquantised binary16 data: K and then V, each in
- *   16-byte chunks of 8 elements (chunk c of token t at (c * 64 + t) * 16), no metadata.
+ *                at (c * 32 + t) * 16.
+ *   For code = SA_KV_FP16 each half holds unquantised binary16 data: K and then V, each in
+ *   16-byte chunks of 8 elements (chunk c of token t at (c * 32 + t) * 16), no metadata.
  */
 #ifndef SA_H_
 #define SA_H_
@@ -76,9 +78,9 @@ enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_INT8 = 8, SA_KV
  * SA_KLAYOUT_NIBBLE: SA_POT4 only, two 4-bit codes (sign, exponent) per byte.
  * SA_KLAYOUT_PLANAR: SA_POTM1 / SA_POTM2 only, the dense 5- and 6-bit form of section II-F (the
  *   paper's 109-byte PoT-M1 record): the sign/exponent nibbles as in SA_KLAYOUT_NIBBLE, followed at
- *   kcode_off + 64 * head_dim / 2 by k bit planes of the mantissa, plane b holding head_dim / 8
- *   bytes per token (bit m % 8 of byte m / 8 = bit b of element m's mantissa), 64 tokens after one
- *   another.  108 / 116 bytes per key at head_dim = 64 against 132 in the byte container. */
+ *   kcode_off + 32 * head_dim / 2 (within each half of the block) by k bit planes of the mantissa, plane b
+ *   holding head_dim / 8 bytes per token (bit m % 8 of byte m / 8 = bit b of element m's mantissa), the
+ *   half's 32 tokens after one another.  108 / 116 bytes per key at head_dim = 64 against 132 in the byte container. */
 enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1, SA_KLAYOUT_PLANAR = 2 };
 /* flags */
 #define SA_FLAG_HADAMARD 1u /* rotate Q and K by the normalised Walsh-Hadamard matrix before quantising */
@@ -106,7 +108,7 @@ typedef struct {
 
 typedef struct {
     size_t page_bytes; /* bytes of one (page, KV head) block */
-    size_t kcode_off;  /* offsets inside a block */
+    size_t kcode_off;  /* offsets inside each 32-token half of a block (the second half starts at page_bytes / 2) */
     size_t meta_off;
     size_t v_off;
     size_t align;      /* required alignment of the pool base pointer */
