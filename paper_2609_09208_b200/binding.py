@@ -199,7 +199,11 @@ def decode_attention_shiftav(cfg, cache: SaCache, Q, O, workspace, n_bits: int =
 
 
 PIPE_KINDS = ["shl", "lop3", "iadd3", "imad_by_one", "prmt", "shl+imad1", "lop3+imad1", "ffma", "ffma2",
-              "imad", "dp4a", "popc+add", "i2f+fadd", "shl+lop3+imad1"]
+              "imad", "dp4a", "popc+add", "i2f+fadd", "shl+lop3+imad1", "vshl.wrap.add", "vshl.clamp.add", "shl+add",
+              "lds128_broadcast", "lds64_gather", "cvt.f32.s32", "cvt.rpi.s32.f32", "ex2", "cvt.f32.s8", "prmt+fadd",
+              "mul.hi", "lds64_scattered"]
+# instructions per step of a kind's chain ("a+b": a pair; the mixes alternate single instructions)
+PIPE_KIND_INSTR = {"popc+add": 2, "i2f+fadd": 2, "shl+add": 2, "prmt+fadd": 2}
 
 
 def pipe_microbench(kind: int, iters: int, blocks: int, sink):

@@ -51,9 +51,14 @@ def _compile_one(src, obj, defines, verbose):
 
 def build(force: bool = False, verbose: bool = False, defines=(), out: str = LIB) -> str:
     """Compile what is stale and link ``out``.  ``defines``: extra ``-D...`` flags (a distinct object cache per set)."""
-    os.makedirs(OBJ_DIR, exist_ok=True)
     tag = _tag(defines)
+    stamp = os.path.join(OBJ_DIR, os.path.basename(out) + ".tag")      # which object set the library was linked from
+    linked = open(stamp).read() if os.path.exists(stamp) else None
     hdr_time = max(os.path.getmtime(h) for h in _headers())
+    src_time = max(hdr_time, max(os.path.getmtime(s) for s in sources()))
+    if not force and os.path.exists(out) and os.path.getmtime(out) >= src_time and linked in (tag, None if not defines else tag):
+        return out                                  # up to date (a library shipped without its objects is trusted by its date)
+    os.makedirs(OBJ_DIR, exist_ok=True)
     jobs, objs = [], []
     for src in sources():
         obj = os.path.join(OBJ_DIR, "%s.%s.o" % (os.path.splitext(os.path.basename(src))[0], tag))
@@ -64,8 +69,6 @@ def build(force: bool = False, verbose: bool = False, defines=(), out: str = LIB
         with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as ex:
             for f in [ex.submit(_compile_one, s, o, defines, verbose) for s, o in jobs]:
                 f.result()
-    stamp = os.path.join(OBJ_DIR, os.path.basename(out) + ".tag")      # which object set the library was linked from
-    linked = open(stamp).read() if os.path.exists(stamp) else ""
     if jobs or linked != tag or not os.path.exists(out) or any(os.path.getmtime(o) > os.path.getmtime(out) for o in objs):
         tmp = out + ".%d.tmp" % os.getpid()
         subprocess.check_call([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs)

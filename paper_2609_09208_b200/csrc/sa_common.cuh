@@ -220,6 +220,12 @@ SA_D void hadamard_warp(float (&x)[EPL], uint32_t (&bits)[EPL], int lane) {
     for (int i = 0; i < EPL; ++i) bits[i] = __half_as_ushort(__float2half_rn(__fmul_rn(x[i], scale)));
 }
 
+// First tile of split s when n_tiles tiles are cut into n_splits slices: floor(n_tiles * s / n_splits) in 32-bit
+// unsigned arithmetic (a 64-bit division is a long software routine on the GPU, and this sits on the critical
+// path of every block); the host refuses caches with max tiles * splits >= 2^31.
+SA_D int split_begin(int n_tiles, int s, int n_splits) {
+    return (int)((uint32_t)n_tiles * (uint32_t)s / (uint32_t)n_splits);
+}
 // 2^e as a float, built from the exponent field; e must lie in [-126, 127].
 SA_D float pow2i(int e) { return __int_as_float((e + 127) << 23); }
 // 2^e for e <= 0, flushing to 0 below the normal range (used for softmax rescales, which are

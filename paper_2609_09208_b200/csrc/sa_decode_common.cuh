@@ -1,9 +1,10 @@
 // Pieces shared by the quantised and the FP16 decode kernels: kernel arguments, the merge of
-// the four warps of a block, and the split-K merge (section II-F: the grid has a split
+// the warps of a block, and the split-K merge (section II-F: the grid has a split
 // dimension; the merge rule follows from the integer running maximum of section II-E:
 // M* = max_s M_s, every partial is rescaled by the exact factor 2^(M_s - M*)).
 #pragma once
 #include "sa_common.cuh"
+#include "sa_mma.cuh"
 
 namespace sa {
 
@@ -30,7 +31,8 @@ struct DecodeArgs {
     const uint16_t* Vnew;
 };
 
-// red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace.
+// red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace
+// (used by the kernels whose warps write their states to shared memory themselves).
 template <int D, int GT, int NW = 4>
 SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], int b, int h0, int split) {
     for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 32 * NW) {
@@ -50,42 +52,87 @@ SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2]
     }
 }
 
-// Per-warp states (M, l, O) -> one partial per block.  acc[mt] is the 16 x 8 tile (dims x queries)
-// of O^T in the accumulator layout of mma.m16n8k8: lane (gq, t4) holds dims 16 mt + 2 gq (c0, c1)
-// and 16 mt + 2 gq + 1 (c2, c3) of queries 2 t4 (c0, c2) and 2 t4 + 1 (c1, c3).
+// Per-warp states (M, l, O) -> one partial per block, in three steps separated by two block barriers:
+// the integer maxima of all warps go to shared memory and one thread per query takes their maximum Mb;
+// every warp scales its own state by the exact factor 2^(M - Mb) in registers and writes it out; the
+// threads of the block add the warps' rows in a fixed order (deterministic) and store the partial.
+// red_s[w][g] = {unused, l, O[D]} of warp w; the maxima live in the first words of the rows:
+// red_s[w][g][0] = M of warp w before the first barrier, red_s[0][g][0] = Mb after the second.
+// acc[mt] is the 16 x 8 tile (dims x queries) of O^T in the accumulator layout of mma.m16n8k8: lane
+// (gq, t4) holds dims 16 mt + 2 gq (c0, c1) and 16 mt + 2 gq + 1 (c2, c3) of queries 2 t4 (c0, c2) and
+// 2 t4 + 1 (c1, c3).
 template <int D, int GT, int NW>
 SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], const int (&M)[GT],
                                 float (&l)[GT], float (&acc)[D / 16][4], int lane, int warp, int b, int h0,
                                 int split) {
     const int gq = lane >> 2, t4 = lane & 3;
+    float lsum[GT];
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
-        const float lsum = warp_sum_f32(l[g]);
-        if (lane == 0) {
-            red_s[warp][g][0] = __int_as_float(M[g]);
-            red_s[warp][g][1] = lsum;
+        lsum[g] = warp_sum_f32(l[g]);
+        if (lane == 0) red_s[warp][g][0] = __int_as_float(M[g]);
+    }
+    __syncthreads();
+    if (threadIdx.x < GT) {
+        int Mb = kMNone;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) Mb = max(Mb, __float_as_int(red_s[w][threadIdx.x][0]));
+        red_s[0][threadIdx.x][0] = __int_as_float(Mb);       // (only this thread reads that column before the barrier)
+    }
+    __syncthreads();
+    // a warp that saw no key (M = "none") has l = 0 and O = 0; its factor is 0 or, if no warp saw one, 1
+    float f[GT];
+#pragma unroll
+    for (int g = 0; g < GT; ++g) f[g] = pow2i_neg(M[g] - __float_as_int(red_s[0][g][0]));
+    float f0 = 0.0f, f1 = 0.0f;                              // factors of this lane's queries 2 t4, 2 t4 + 1
+#pragma unroll
+    for (int g = 0; g < GT; ++g)
+        if (t4 == g / 2) {
+            if (g & 1) f1 = f[g];
+            else f0 = f[g];
         }
+    if (lane == 0) {
+#pragma unroll
+        for (int g = 0; g < GT; ++g) red_s[warp][g][1] = lsum[g] * f[g];
     }
 #pragma unroll
     for (int mt = 0; mt < D / 16; ++mt) {
         const int dim = 16 * mt + 2 * gq;
         if (2 * t4 < GT) {
-            red_s[warp][2 * t4][2 + dim] = acc[mt][0];
-            red_s[warp][2 * t4][2 + dim + 1] = acc[mt][2];
+            red_s[warp][2 * t4][2 + dim] = acc[mt][0] * f0;
+            red_s[warp][2 * t4][2 + dim + 1] = acc[mt][2] * f0;
         }
         if (2 * t4 + 1 < GT) {
-            red_s[warp][2 * t4 + 1][2 + dim] = acc[mt][1];
-            red_s[warp][2 * t4 + 1][2 + dim + 1] = acc[mt][3];
+            red_s[warp][2 * t4 + 1][2 + dim] = acc[mt][1] * f1;
+            red_s[warp][2 * t4 + 1][2 + dim + 1] = acc[mt][3] * f1;
         }
     }
     __syncthreads();
-    block_combine_and_store<D, GT, NW>(a, red_s, b, h0, split);
+    for (int idx = threadIdx.x; idx < GT * (D + 2); idx += 32 * NW) {
+        const int g = idx / (D + 2), c = idx % (D + 2);       // c = 0: M, 1: l, c >= 2: O[c - 2]
+        float v = red_s[0][g][c];
+        if (c != 0) {
+#pragma unroll
+            for (int w = 1; w < NW; ++w) v += red_s[w][g][c];
+        }
+        a.partials[(((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2) + c] = v;
+    }
 }
 
-// One block per (sequence, query head): kMergeGroups groups of D threads each take every
-// kMergeGroups-th split (independent, unrolled loads), then the groups are combined in shared
-// memory and the result is normalised.
-constexpr int kMergeGroups = 8;
+// Split-K merge.  One block of 128 threads per (sequence, query head, 16 output dims): 4 lanes of four
+// dims times 32 groups of splits; a thread's loads (three splits at a time) are all in flight
+// together, so up to 96 splits cost one round trip to L2.  Each thread merges its splits with a local
+// maximum, the block takes the maximum M* of those, every thread rescales its sum by the exact
+// 2^(M_local - M*), and the groups are added in a fixed order (deterministic).  The block is kept this
+// small — 128 threads, at most 32 registers, 2.7 KB of shared memory — so that it fits on an SM beside
+// two resident blocks of the decode kernel: the next decode kernel is launched while this one runs
+// (programmatic dependent launch), and a merge block that took the place of one of its blocks would make
+// that block, and with it the whole grid, finish late.
+constexpr int kMergeThreads = 128;
+constexpr int kMergeDims = 16;                                // output dims per block
+constexpr int kMergeLanes = kMergeDims / 4;                   // float4 lanes
+constexpr int kMergeGroups = kMergeThreads / kMergeLanes;     // groups of splits
+constexpr int kMergeChunk = 3;                                // splits per thread whose loads are in flight together
 
 // A sequence's length grows by one when the decode kernel appended the step's token itself (the token's
 // page must be mapped, exactly the condition the decode kernel used).
@@ -96,82 +143,88 @@ struct BumpArgs {
 };
 
 template <int D>
-__global__ void __launch_bounds__(D * kMergeGroups) merge_kernel(const float* __restrict__ partials,
-                                                                 float* __restrict__ O, int n_splits, int n_rows,
-                                                                 BumpArgs bump) {
-    __shared__ int m_s[D * kMergeGroups / 32];
-    __shared__ float o_s[kMergeGroups][D + 1];
+__global__ void __launch_bounds__(kMergeThreads, 16) merge_kernel(const float* __restrict__ partials,
+                                                                  float* __restrict__ O, int n_splits, int n_rows,
+                                                                  BumpArgs bump) {
+    __shared__ int mw_s[kMergeThreads / 32];
+    __shared__ float4 o_s[kMergeGroups][kMergeLanes];
+    __shared__ float l_s[kMergeGroups];
     pdl_wait();                                               // the partials come from the kernel before
     pdl_launch_dependents();
-    const int row = blockIdx.x;                               // b * Hq + h
-    if (bump.seq_lens && threadIdx.x == 0 && row % bump.Hq == 0) {
+    const int row = blockIdx.x / (D / kMergeDims);            // b * Hq + h
+    const int part = blockIdx.x % (D / kMergeDims);           // which 16 dims
+    if (bump.seq_lens && threadIdx.x == 0 && part == 0 && row % bump.Hq == 0) {
         // every block of the decode kernel has read the old length by now
         const int b = row / bump.Hq, len = bump.seq_lens[b], lp = len / kPageTokens;
         const int pidx = (len >= 0 && lp < bump.max_pages) ? bump.page_table[(size_t)b * bump.max_pages + lp] : -1;
         if (pidx >= 0 && pidx < bump.n_pages) bump.seq_lens[b] = len + 1;
     }
-    const int dd = threadIdx.x % D, grp = threadIdx.x / D;
     const size_t stride = (size_t)n_rows * (D + 2);
+    const int ln = threadIdx.x % kMergeLanes, grp = threadIdx.x / kMergeLanes;
     const float* base = partials + (size_t)row * (D + 2);
-    float l = 0.0f, o = 0.0f;
-    constexpr int kHeld = 16;                                 // splits per thread held in registers
-    if (n_splits <= kHeld * kMergeGroups) {
-        // Common case: every load of this thread is issued before anything waits on one of them (a single
-        // round trip to L2), then the maximum of the integer running maxima, then the exact rescale.
-        int Mv[kHeld];
-        float lv[kHeld], ov[kHeld];
+    const float* obase = base + 2 + part * kMergeDims + ln * 4;
+    int Ml = kMNone;                                          // this thread's splits: grp, grp + 32, ...
+    float l = 0.0f;
+    float4 o = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    for (int s0 = grp; s0 < n_splits; s0 += kMergeGroups * kMergeChunk) {
+        float2 ml[kMergeChunk], v0[kMergeChunk], v1[kMergeChunk];
 #pragma unroll
-        for (int k = 0; k < kHeld; ++k) {
-            const int s = grp + k * kMergeGroups;
-            const float* p = base + (size_t)(s < n_splits ? s : 0) * stride;
-            Mv[k] = (s < n_splits) ? __float_as_int(p[0]) : kMNone;
-            lv[k] = p[1];
-            ov[k] = p[2 + dd];
+        for (int k = 0; k < kMergeChunk; ++k) {
+            const int s = s0 + k * kMergeGroups;
+            const size_t off = (size_t)(s < n_splits ? s : s0) * stride;
+            ml[k] = *reinterpret_cast<const float2*>(base + off);
+            v0[k] = reinterpret_cast<const float2*>(obase + off)[0];
+            v1[k] = reinterpret_cast<const float2*>(obase + off)[1];
+            if (s >= n_splits) ml[k].x = __int_as_float(kMNone);
         }
-        int Ms = kMNone;
+        int Mn = Ml;
 #pragma unroll
-        for (int k = 0; k < kHeld; ++k) Ms = max(Ms, Mv[k]);
-        // the thread's splits are those of its whole group: one value per group is enough
-        if (dd == 0) m_s[grp] = Ms;
-        __syncthreads();
+        for (int k = 0; k < kMergeChunk; ++k) Mn = max(Mn, __float_as_int(ml[k].x));
+        const float fo = pow2i_neg(Ml - Mn);                  // 1 if nothing changed; 0 on the first chunk (l and o are 0 then)
+        l *= fo;
+        o.x *= fo;
+        o.y *= fo;
+        o.z *= fo;
+        o.w *= fo;
+        Ml = Mn;
 #pragma unroll
-        for (int g = 0; g < kMergeGroups; ++g) Ms = max(Ms, m_s[g]);
-#pragma unroll
-        for (int k = 0; k < kHeld; ++k) {
-            const float f = (Mv[k] == kMNone) ? 0.0f : pow2i_neg(Mv[k] - Ms);
-            l += lv[k] * f;
-            o += ov[k] * f;
-        }
-    } else {
-        // global maximum of the integer running maxima
-        int Ms = kMNone;
-        for (int s = threadIdx.x; s < n_splits; s += D * kMergeGroups) Ms = max(Ms, __float_as_int(base[s * stride]));
-#pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1) Ms = max(Ms, __shfl_xor_sync(0xffffffffu, Ms, o2));
-        if ((threadIdx.x & 31) == 0) m_s[threadIdx.x >> 5] = Ms;
-        __syncthreads();
-#pragma unroll
-        for (int w = 0; w < D * kMergeGroups / 32; ++w) Ms = max(Ms, m_s[w]);
-#pragma unroll 8
-        for (int s = grp; s < n_splits; s += kMergeGroups) {
-            const float* p = base + s * stride;
-            const int M = __float_as_int(p[0]);
-            const float f = (M == kMNone) ? 0.0f : pow2i_neg(M - Ms);
-            l += p[1] * f;
-            o += p[2 + dd] * f;
+        for (int k = 0; k < kMergeChunk; ++k) {
+            const int M = __float_as_int(ml[k].x);
+            const float f = (M == kMNone) ? 0.0f : pow2i_neg(M - Mn);     // a split that saw no key carries zeros
+            l += ml[k].y * f;
+            o.x += v0[k].x * f;
+            o.y += v0[k].y * f;
+            o.z += v1[k].x * f;
+            o.w += v1[k].y * f;
         }
     }
-    o_s[grp][dd] = o;
-    if (dd == 0) o_s[grp][D] = l;
+    int Ms = warp_max_s32(Ml);
+    if ((threadIdx.x & 31) == 0) mw_s[threadIdx.x >> 5] = Ms;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kMergeThreads / 32; ++w) Ms = max(Ms, mw_s[w]);
+    const float f = (Ml == kMNone) ? 0.0f : pow2i_neg(Ml - Ms);
+    o_s[grp][ln] = make_float4(o.x * f, o.y * f, o.z * f, o.w * f);
+    if (ln == 0) l_s[grp] = l * f;
     __syncthreads();
     if (grp == 0) {
-#pragma unroll
+        // the groups are added in a fixed order: the result does not depend on the timing of anything
+        o = o_s[0][ln];
+        l = l_s[0];
+#pragma unroll 8
         for (int g = 1; g < kMergeGroups; ++g) {
-            o += o_s[g][dd];
-            l += o_s[g][D];
+            const float4 t = o_s[g][ln];
+            o.x += t.x;
+            o.y += t.y;
+            o.z += t.z;
+            o.w += t.w;
+            l += l_s[g];
         }
         // no key at all: zeros; a poisoned partial (a bounded wait gave up) stays visible as NaN
-        O[(size_t)row * D + dd] = (l == 0.0f) ? 0.0f : o / l;
+        const float inv = 1.0f / l;
+        float4 r = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+        if (l == 0.0f) r = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        *reinterpret_cast<float4*>(O + (size_t)row * D + part * kMergeDims + ln * 4) = r;
     }
 }
 
@@ -185,6 +238,8 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
         return SA_ERR_ALIGNMENT;
     int S, GT;
     split_plan(p, c->batch, c->max_pages_per_seq, &S, &GT);
+    // the kernels place the splits with 32-bit arithmetic: tiles * (splits + 1) must stay below 2^31
+    if ((long long)c->max_pages_per_seq * (kPageTokens / kTileTokens) * (S + 1) >= (1LL << 31)) return SA_ERR_CAPACITY;
     const size_t need = (size_t)S * c->batch * p.Hq * (p.d + 2) * sizeof(float);
     if (!workspace || workspace_bytes < need) return SA_ERR_CAPACITY;
     if (mis(workspace, 16)) return SA_ERR_ALIGNMENT;
@@ -227,9 +282,9 @@ inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s
     const int rows = a.batch * a.Hq;
     BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq};
     cudaError_t err;
-    if (p.d == 64) err = launch_pdl(merge_kernel<64>, dim3(rows), dim3(64 * kMergeGroups), 0, s,
+    if (p.d == 64) err = launch_pdl(merge_kernel<64>, dim3(rows * (64 / kMergeDims)), dim3(kMergeThreads), 0, s,
                                     (const float*)a.partials, a.O, a.n_splits, rows, bump);
-    else err = launch_pdl(merge_kernel<128>, dim3(rows), dim3(128 * kMergeGroups), 0, s,
+    else err = launch_pdl(merge_kernel<128>, dim3(rows * (128 / kMergeDims)), dim3(kMergeThreads), 0, s,
                           (const float*)a.partials, a.O, a.n_splits, rows, bump);
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SA_OK : SA_ERR_CUDA;
 }

@@ -101,8 +101,8 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     if (lane == 0) {
         const int len_g = __ldcg(a.seq_lens + b) + (a.Knew ? 1 : 0);
         const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
-        const int tile_g = (int)((long long)n_tiles_g * split / a.n_splits) + warp;
-        if (tile_g < (int)((long long)n_tiles_g * (split + 1) / a.n_splits)) {
+        const int tile_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
+        if (tile_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
             const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
             if (pidx_g >= 0 && pidx_g < a.n_pages)
                 Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, (tile_g & 1) * 32);
@@ -122,8 +122,8 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         }
     }
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
-    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int tile0 = split_begin(n_tiles, split, a.n_splits);
+    const int tile1 = split_begin(n_tiles, (split + 1), a.n_splits);
     const int first = tile0 + warp;
     const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
     if (tile_new >= first && tile_new < tile1 && (tile_new - first) % 4 == 0) {      // this warp owns that tile

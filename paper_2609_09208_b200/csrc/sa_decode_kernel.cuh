@@ -96,6 +96,13 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     }
     __syncwarp();
     pdl_launch_dependents();    // the split-K merge may be scheduled as soon as blocks of this grid retire
+    // A guess at the warps' first tiles, from a length the preceding kernel may be about to change, only to ask
+    // L2 for those tiles while that kernel drains (loads that bypass L1, so nothing stale can be read back later).
+    // The length is fetched here, so that its latency hides behind the query quantisation; the dependent
+    // page-table reads and the hints themselves are left to the last warp, after the prologue's last barrier,
+    // so that no other warp waits for them.
+    int len_g = 0, tile_g = -1, pidx_g = -1;
+    if (lane == 0 || warp == NW - 1) len_g = __ldcg(a.seq_lens + b);
 
     // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register.  It reads
     // only Q, which no kernel of a decode step writes, so it runs BEFORE the wait on the preceding
@@ -110,6 +117,11 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
     }
     __syncthreads();
+    if (lane == 0) {
+        const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
+        const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
+        if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) tile_g = t_g;
+    }
     if constexpr (SM::kTable) {
         // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
         using TS = TableScore<KB, NP>;
@@ -196,22 +208,22 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     }
     __syncthreads();
 
-    // While the preceding kernel drains: a guess at this warp's first tile, from a length that kernel may be
-    // about to change, only to ask L2 for it (loads that bypass L1, so nothing stale can be read back later).
-    if (lane == 0) {
-        const int len_g = __ldcg(a.seq_lens + b) + (a.Knew ? 1 : 0);
-        const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
-        const int tile_g = (int)((long long)n_tiles_g * split / a.n_splits) + warp;
-        if (tile_g < (int)((long long)n_tiles_g * (split + 1) / a.n_splits)) {
-            const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
-            if (pidx_g >= 0 && pidx_g < a.n_pages)
-                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, (tile_g & 1) * 32, !SP);
+    if (warp == NW - 1 && lane < NW) {                        // lane w: the first tile of warp w
+        const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
+        const int t_g = split_begin(n_tiles_g, split, a.n_splits) + lane;
+        if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
+            const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
+            if (p_g >= 0 && p_g < a.n_pages)
+                Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32, !SP);
         }
     }
     pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
 
     // ---- this warp's tiles; start the first copies ----
     int len = a.seq_lens[b];
+    // the page of the guessed first tile, read again now that it is valid, at the same time as the length
+    // (one round trip instead of two when the guess holds, which it does unless the length crossed a tile boundary)
+    if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
     int tile_new = -1, pidx_new = -1;
     if (a.Knew) {
         // Fused append: the step's new token goes to position len (if its page is mapped) and is part of
@@ -225,8 +237,8 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
     }
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
-    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int tile0 = split_begin(n_tiles, split, a.n_splits);
+    const int tile1 = split_begin(n_tiles, (split + 1), a.n_splits);
     const int first = tile0 + warp;
     const int n_my = first < tile1 ? (tile1 - first + NW - 1) / NW : 0;
     if (tile_new >= first && tile_new < tile1 && (tile_new - first) % NW == 0) {      // warp-uniform: this warp owns that tile
@@ -249,7 +261,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
     auto issue = [&](int i) {
         const int tile = first + NW * i;
-        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int pidx = (tile == tile_g) ? pidx_g : a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
         const int s = i % NS;
         if (pidx < 0 || pidx >= a.n_pages) {
             mbar_arrive(mbar0 + s * 8);
@@ -263,11 +275,13 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         for (int i = 0; i < NS && i < n_my; ++i) issue(i);
 
     int M[GT];
+    float Mf[GT];            // M as a float (exact below 2^24)
     float l[GT];
     float acc[MT][4];        // O^T tiles: lane (gq, t4) holds dims 16 mt + 2 gq (+1) of queries 2 t4 (+1)
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         M[g] = kMNone;
+        Mf[g] = (float)kMNone;
         l[g] = 0.0f;
     }
 #pragma unroll
@@ -416,8 +430,6 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             // key, 8 query columns of FP32.
             __syncwarp();
             float (*p_t)[8] = reinterpret_cast<float (*)[8]>(const_cast<uint8_t*>(st));
-            bool changed = false;
-            float resc[GT];
             const float s_v = valid ? s_j : 0.0f, z_bias = valid ? 0.0f : -INFINITY;
             float pv[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};        // unused query columns stay zero
             if (a.dbg_scores && valid) {                      // parity tests only: one branch around all the stores
@@ -425,31 +437,33 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 for (int g = 0; g < GT; ++g)
                     a.dbg_scores[((size_t)b * a.Hq + h0 + g) * a.dbg_stride + (size_t)tile * 32 + lane] = A[g];
             }
+            float z[GT];
+            bool above = false;
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 // a lane without a key gets z = -inf through the addend (the product is rounded once either way)
-                const float z = fmaf((float)A[g] * qscale_s[g], s_v, z_bias);
-                // ceil of the tile's largest logit: ceil is monotone, so take the integer maximum (the
-                // conversion saturates; a lane without a key gives the smallest integer)
-                const int Mt = max(warp_max_s32(__float2int_ru(z)), -(1 << 28));
-                const int Mn = max(M[g], Mt);
-                resc[g] = pow2i_neg(M[g] - Mn);               // exact power of two; 0 while M is still "no key seen" (-2^29)
-                changed |= (Mn != M[g]);
-                M[g] = Mn;
-                const float p = ex2_approx(z - (float)Mn);     // 2^-inf = 0 for a lane without a key
-                l[g] = l[g] * resc[g] + p;
-                pv[g] = p * vscale;                                                 // weight times 2^-g_j
+                z[g] = fmaf((float)A[g] * qscale_s[g], s_v, z_bias);
+                above |= z[g] > Mf[g];
             }
-            reinterpret_cast<float4*>(&p_t[prow][0])[0] = make_float4(pv[0], pv[1], pv[2], pv[3]);
-            reinterpret_cast<float4*>(&p_t[prow][0])[1] = make_float4(pv[4], pv[5], pv[6], pv[7]);
-            if (changed) {                                    // warp-uniform
-                float r0 = 0.0f, r1 = 0.0f;                   // factors of this lane's queries 2 t4, 2 t4 + 1
+            // The running maximum M is an integer that bounds every logit seen so far from above; it has to
+            // move only when a logit of this tile exceeds it, which after the first tiles is rare.
+            if (__any_sync(0xffffffffu, above)) {             // warp-uniform
+                float r0 = 0.0f, r1 = 0.0f;                   // rescale factors of this lane's queries 2 t4, 2 t4 + 1
 #pragma unroll
-                for (int g = 0; g < GT; g += 2)
+                for (int g = 0; g < GT; ++g) {
+                    // ceiling of the tile's largest logit: ceil is monotone, so take the integer maximum (the
+                    // conversion saturates; a lane without a key gives the smallest integer)
+                    const int Mt = max(warp_max_s32(__float2int_ru(z[g])), -(1 << 28));
+                    const int Mo = __float2int_rn(Mf[g]);     // exact: M is an integer below 2^29 in magnitude
+                    const int Mn = max(Mo, Mt);
+                    const float resc = pow2i_neg(Mo - Mn);    // exact power of two; 0 while M is still "no key seen" (-2^29)
+                    l[g] *= resc;
+                    Mf[g] = (float)Mn;
                     if (t4 == g / 2) {
-                        r0 = resc[g];
-                        r1 = (g + 1 < GT) ? resc[g + 1] : 0.0f;
+                        if (g & 1) r1 = resc;
+                        else r0 = resc;
                     }
+                }
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     acc[mt][0] *= r0;
@@ -458,6 +472,14 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                     acc[mt][3] *= r1;
                 }
             }
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const float p = ex2_approx(z[g] - Mf[g]);     // at most 1; 2^-inf = 0 for a lane without a key
+                l[g] += p;
+                pv[g] = p * vscale;                           // weight times 2^-g_j
+            }
+            reinterpret_cast<float4*>(&p_t[prow][0])[0] = make_float4(pv[0], pv[1], pv[2], pv[3]);
+            reinterpret_cast<float4*>(&p_t[prow][0])[1] = make_float4(pv[4], pv[5], pv[6], pv[7]);
             __syncwarp();
 
             // ---- phase 3: O^T += V^T P^T on the tensor cores.  One 8 x 8 block of 16-bit pairs
@@ -497,6 +519,10 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             issue(i + NS);
         }
     }
+    if constexpr (!SP) {
+#pragma unroll
+        for (int g = 0; g < GT; ++g) M[g] = __float2int_rn(Mf[g]);      // exact: an integer of magnitude at most 2^29
+    }
     if (failed) {
         // A bounded wait expired: make the failure visible in the output instead of returning a
         // plausible number (no copy of this warp can still be in flight into a buffer it re-uses).
@@ -508,7 +534,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     }
 
     // ---- merge the warps of the block, write the block's partial ----
-    __syncthreads();                                           // the merge scratch re-uses the stage buffers
+    __syncthreads();
     if constexpr (SP) {
         // score pass of the shift-A.V option: the block's statistics instead of a partial
         int* stat_s = reinterpret_cast<int*>(smem + SM::kStageOff);           // [NW][GT + 1]

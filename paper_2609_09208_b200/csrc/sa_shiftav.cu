@@ -70,8 +70,8 @@ __global__ void __launch_bounds__(128) shiftav_kernel(DecodeArgs a) {
 
     const int len = a.seq_lens[b];
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = (int)((long long)n_tiles * split / a.n_splits);
-    const int tile1 = (int)((long long)n_tiles * (split + 1) / a.n_splits);
+    const int tile0 = split_begin(n_tiles, split, a.n_splits);
+    const int tile1 = split_begin(n_tiles, (split + 1), a.n_splits);
     const int first = tile0 + warp;
     const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
     auto issue = [&](int i) {

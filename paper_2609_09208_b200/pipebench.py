@@ -40,7 +40,7 @@ def main():
             ms = s.elapsed_time(e)
             if best is None or ms < best:
                 best, mhz = ms, mhz_now
-        per_thread = iters * 64 * (2 if name in ("popc+add", "i2f+fadd") else 1)
+        per_thread = iters * 64 * sa.PIPE_KIND_INSTR.get(name, 1)
         total = per_thread * 256 * blocks
         rate = total / (best * 1e-3) / (mhz * 1e6) / sms
         rows[name] = {"ms": best, "sm_mhz": mhz, "thread_instr_per_clk_per_sm": rate}
