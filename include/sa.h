@@ -68,8 +68,8 @@ typedef enum {
 
 /* Key code family: the value is k, the number of mantissa bits (eq. (2), eq. (5)). */
 enum { SA_POT4 = 0, SA_POTM1 = 1, SA_POTM2 = 2, SA_POTM4 = 4, SA_INT8 = 8, SA_KV_FP16 = 16 };
-/* SA_INT8 is the comparison code of section III / VI (an INT8 multiply-accumulate kernel "of
- * identical structure"): uniform INT8 keys, khat = round(K * 127 / amax) with the row maximum as
+/* SA_INT8 is the comparison code of section III / VI (an INT8 multiply-accumulate kernel built on the
+ * same skeleton as the shift kernels): uniform INT8 keys, khat = round(K * 127 / amax) with the row maximum as
  * scale, stored one byte per element in the byte container (132 bytes per key at d = 64, the same
  * as PoT-M4); scores are integer dot products evaluated with dp4a.  Everything else (query and
  * value quantisers, softmax, A.V, merge, cache layout) is shared with the power-of-two codes. */
@@ -92,6 +92,14 @@ enum { SA_KLAYOUT_BYTE = 0, SA_KLAYOUT_NIBBLE = 1, SA_KLAYOUT_PLANAR = 2 };
  * datapath; it is the mid-point between the shift kernels and the INT8 multiply-accumulate comparison
  * (section III), and is reported as such.  (PoT-4 has no shift left in its key loop: SA_ERR_UNSUPPORTED.) */
 #define SA_FLAG_SHIFT_BY_MULTIPLY 2u
+/* Decode kernels only, power-of-two codes only, off by default: every sign flip and add of the integer score
+ * (eq. (3)) is issued as logic and add instructions (exclusive-or with the sign mask, subtract, add) instead
+ * of one multiply-add by +1 / -1, so that no instruction of the score datapath touches the multiplier array.
+ * The INT32 scores are the same bit for bit.  It is the strictly multiplier-free form of the default kernels
+ * and is slower than them on this GPU, whose shift/logic/add pipe is the busier one; it exists to be measured
+ * beside the default, SA_FLAG_SHIFT_BY_MULTIPLY and the INT8 multiply-accumulate comparison.  Excludes
+ * SA_FLAG_SHIFT_BY_MULTIPLY. */
+#define SA_FLAG_ADD_ON_ALU 4u
 
 typedef struct {
     int head_dim;    /* 64 or 128 */
@@ -103,7 +111,7 @@ typedef struct {
                         Must satisfy F >= 6 + k (eq. (4): every shift is a left shift) and
                         head_dim * 127 * (2^(k+1) - 1) * 2^(F - k) < 2^31 (INT32 accumulator) */
     int page_tokens; /* 64 */
-    unsigned flags;  /* SA_FLAG_HADAMARD | SA_FLAG_SHIFT_BY_MULTIPLY */
+    unsigned flags;  /* SA_FLAG_HADAMARD | SA_FLAG_SHIFT_BY_MULTIPLY | SA_FLAG_ADD_ON_ALU */
 } sa_config;
 
 typedef struct {
@@ -131,8 +139,10 @@ sa_status sa_get_layout(const sa_config* cfg, sa_layout* out);
 
 /* Bytes of scratch that sa_decode_attention / sa_decode_attention_fp16 need for a cache with
  * `batch` sequences of at most `max_pages_per_seq` pages (split-K partial results, section II-F:
- * the kernel grid has a split dimension).  Host only, no CUDA call.  The scratch needs no
- * initialisation and may be shared by calls that do not overlap on the GPU. */
+ * the kernel grid has a split dimension).  Host only; the one CUDA call it may make reads the number of
+ * multiprocessors of the CURRENT device (once per device), because the split count is planned for it: ask on
+ * the device the decode calls will run on (without a device the figure of a B200 is used).  The scratch needs
+ * no initialisation and may be shared by calls that do not overlap on the GPU. */
 sa_status sa_workspace_bytes(const sa_config* cfg, int batch, int max_pages_per_seq, size_t* out);
 
 /* Key encode (eq. (2), eq. (5); nearest-in-log2 rounding, section II-D).
@@ -172,9 +182,14 @@ sa_status sa_fill_kv(const sa_config* cfg, const sa_cache* cache, const uint16_t
  *   score A = sum_m sigma * qhat * (2^k + j) << (F - k - e) is formed exactly in INT32 with
  *   shifts, sign flips and adds; logits z = A * Delta * s * 2^-F * log2(e) / sqrt(d) feed an
  *   online softmax whose running maximum is an integer in the log2 domain, so that every
- *   rescale is an exact power of two; O accumulates p * vhat * 2^-g in FP32; the key axis is
- *   split over thread blocks and the partial (M, l, O) triples are merged with exact
- *   power-of-two factors.
+ *   rescale is an exact power of two; O accumulates p * vhat * 2^-g (the paper's floating-point
+ *   A.V); the key axis is split over thread blocks and the partial (M, l, O) triples are merged
+ *   with exact power-of-two factors.
+ *   The A.V products run on the tensor cores as tf32 x tf32 with FP32 accumulation (mma.m16n8k8): the INT8
+ *   values are exact in tf32, and every weight p * 2^-g enters as the sum of two tf32 terms (its leading
+ *   11 significant bits, and the remainder cut to 11 bits), so that a weight keeps about 21 significant
+ *   bits: the relative error of one product is below 2^-21, against 2^-24 for an FP32 multiply; measured
+ *   max |dO| against the CPU oracle is 2e-8 .. 6e-7.  The integer scores never touch the tensor cores.
  * Q [batch, n_q_heads, head_dim] binary16; O [batch, n_q_heads, head_dim] float.
  * A sequence with seq_lens[b] == 0 yields zeros.
  * dbg_scores (nullable): int32 [batch, n_q_heads, max_pages_per_seq * 64]; receives A for every
@@ -273,10 +288,22 @@ sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const sa_cache* 
  *     calls that overlap on the GPU (different streams, or graphs replayed concurrently) race on
  *     it and corrupt each other's output.  Serialise them, or give the overlapping ones their own
  *     workspace through sa_decode_attention.
- *   - cfg->code must be one of the power-of-two codes (not SA_KV_FP16). */
+ *   - cfg->code must be one of the quantised key codes (the power-of-two codes or SA_INT8), not SA_KV_FP16. */
 #define SA_STATIC_SCRATCH_BYTES (4u << 20)
 sa_status sa_decode_attention_static(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                                      float* O, int32_t* dbg_scores, sa_stream stream);
+
+/* Test hook for the failure path of the staged copies (the paper has no counterpart).  sa_decode_attention
+ * in which the bulk copy of ONE tile — 32-token tile `tile` of sequence `b`, KV head `kv_head` — is never
+ * issued and every wait for a copy gives up after 2^10 polls instead of 2^18.  The warp that owns that tile
+ * finds its wait exhausted, abandons its remaining tiles and marks its block's partial result; the split-K
+ * merge carries the mark into O: the rows of the query heads of `kv_head` in sequence `b` come out as NaN,
+ * every other row is the ordinary result, and the call returns like any other (nothing is left in flight,
+ * nothing waits without a bound).  Only head_dim 64, SA_POTM4 in the byte container, 8 query heads per KV
+ * head, no flags: anything else is SA_ERR_UNSUPPORTED. */
+sa_status sa_debug_decode_lost_copy(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q, float* O,
+                                    void* workspace, size_t workspace_bytes, int b, int kv_head, int tile,
+                                    sa_stream stream);
 
 /* Instruction-throughput micro-benchmark (measurement aid; the paper has no counterpart — it stands
  * in for the paper's disassembly-based operation counts, section III and Table V).  Launches `blocks`
@@ -284,7 +311,11 @@ sa_status sa_decode_attention_static(const sa_config* cfg, const sa_cache* cache
  * independent chains.  kind: 0 variable shift, 1 three-input logic op, 2 three-input add,
  * 3 multiply-add by one (an add issued on the FMA pipe), 4 byte permute, 5 shift/multiply-add mix,
  * 6 logic/multiply-add mix, 7 FP32 FMA, 8 packed FP32x2 FMA, 9 integer multiply-add, 10 dp4a,
- * 11 population count + add, 12 int8-to-float + add, 13 shift/logic/multiply-add mix.
+ * 11 population count + add, 12 int8-to-float + add, 13 shift/logic/multiply-add mix, 14 / 15 the scalar video
+ * shift-and-add (vshl ... wrap.add / clamp.add, the paper's Table V rows), 16 shift then add as two instructions,
+ * 17 128-bit shared-memory load with every lane at one address, 18 / 25 64-bit shared-memory loads whose lanes
+ * pick entries of one 128-byte row (regularly / irregularly), 19 int32-to-float, 20 float-to-int32 rounding up,
+ * 21 ex2.approx, 22 byte-to-float, 23 the same as byte permute + FP32 add, 24 mul.hi.
  * `sink` is one device word (practically never written).  The caller times the launch. */
 sa_status sa_pipe_microbench(int kind, int iters, int blocks, uint32_t* sink, sa_stream stream);
 

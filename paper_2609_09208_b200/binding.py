@@ -17,6 +17,7 @@ SA_POT4, SA_POTM1, SA_POTM2, SA_POTM4, SA_INT8, SA_KV_FP16 = 0, 1, 2, 4, 8, 16
 SA_KLAYOUT_BYTE, SA_KLAYOUT_NIBBLE, SA_KLAYOUT_PLANAR = 0, 1, 2
 SA_FLAG_HADAMARD = 1
 SA_FLAG_SHIFT_BY_MULTIPLY = 2
+SA_FLAG_ADD_ON_ALU = 4
 PAGE_TOKENS = 64
 
 EXPORTS = [
@@ -24,7 +25,7 @@ EXPORTS = [
     "sa_quantise_query", "sa_quantise_values", "sa_append_kv", "sa_fill_kv", "sa_decode_attention",
     "sa_decode_attention_fp16", "sa_decode_attention_stages", "sa_decode_attention_fp16_stages", "sa_debug_unpack", "sa_staging_bytes", "sa_decode_step_host",
     "sa_decode_attention_static", "sa_pipe_microbench", "sa_shiftav_workspace_bytes", "sa_decode_attention_shiftav",
-    "sa_decode_step",
+    "sa_decode_step", "sa_debug_decode_lost_copy",
 ]
 
 
@@ -77,15 +78,18 @@ def _check(st: int, where: str):
 
 
 def make_config(head_dim: int, n_q_heads: int, n_kv_heads: int, code: int, *, nibble: bool = False,
-                headroom_F: int = 0, hadamard: bool = False, shift_by_multiply: bool = False) -> SaConfig:
+                headroom_F: int = 0, hadamard: bool = False, shift_by_multiply: bool = False,
+                add_on_alu: bool = False) -> SaConfig:
     """nibble=True selects the dense sub-byte container of the code: two 4-bit codes per byte for PoT-4,
     nibbles plus mantissa bit planes (5 / 6 bits per element) for PoT-M1 / PoT-M2.  shift_by_multiply=True
-    selects the non-default decode kernels whose shifts run on the integer multiplier (same scores)."""
+    selects the non-default decode kernels whose shifts run on the integer multiplier, add_on_alu=True the
+    non-default ones without any multiply-add in the score datapath (same scores either way)."""
     klayout = SA_KLAYOUT_BYTE
     if nibble:
         klayout = SA_KLAYOUT_NIBBLE if code == SA_POT4 else SA_KLAYOUT_PLANAR
     return SaConfig(head_dim, n_q_heads, n_kv_heads, code, klayout, headroom_F, PAGE_TOKENS,
-                    (SA_FLAG_HADAMARD if hadamard else 0) | (SA_FLAG_SHIFT_BY_MULTIPLY if shift_by_multiply else 0))
+                    (SA_FLAG_HADAMARD if hadamard else 0) | (SA_FLAG_SHIFT_BY_MULTIPLY if shift_by_multiply else 0) |
+                    (SA_FLAG_ADD_ON_ALU if add_on_alu else 0))
 
 
 def get_layout(cfg: SaConfig) -> SaLayout:
@@ -220,6 +224,13 @@ def decode_attention_static(cfg, cache: SaCache, Q, O, dbg_scores=None):
     problem needs more than STATIC_SCRATCH_BYTES.  Calls sharing a device must not overlap on the GPU."""
     _check(lib().sa_decode_attention_static(C.byref(cfg), C.byref(cache), _ptr(Q), _ptr(O), _ptr(dbg_scores),
                                             _stream()), "sa_decode_attention_static")
+
+
+def debug_decode_lost_copy(cfg, cache: SaCache, Q, O, workspace, b: int, kv_head: int, tile: int):
+    """Test hook: decode attention in which the copy of one 32-token tile is never issued (its rows come out NaN)."""
+    _check(lib().sa_debug_decode_lost_copy(C.byref(cfg), C.byref(cache), _ptr(Q), _ptr(O), _ptr(workspace),
+                                           C.c_size_t(workspace.numel() * workspace.element_size()), C.c_int(b),
+                                           C.c_int(kv_head), C.c_int(tile), _stream()), "sa_debug_decode_lost_copy")
 
 
 def debug_unpack(cfg, cache: SaCache, b: int, n_tokens: int, codes=None, scales=None, v_hat=None, g=None):

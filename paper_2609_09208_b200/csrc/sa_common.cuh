@@ -22,7 +22,7 @@ constexpr int half_block_bytes(int d, int kb, bool nib) {
     return kTileTokens * (nib ? d / 2 : d) + ((nib && kb > 0) ? kb * kTileTokens * (d / 8) : 0) + kTileTokens * 4 + kTileTokens * d;
 }
 constexpr int half_block_bytes_fp16(int d) { return 2 * kTileTokens * d * 2; }
-constexpr int kNumSMs = 148;              // B200
+constexpr int kNumSMsB200 = 148;          // the split plan's SM count where no device can be asked (see sm_count())
 constexpr int kEmax = 6;                  // largest exponent of the 3-bit field
 constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no key seen yet"
 
@@ -32,6 +32,7 @@ constexpr int kMNone = -(1 << 29);        // running-maximum value meaning "no k
 struct Plan {
     int d, Hq, Hkv, G, k;     // k = mantissa bits (0 for SA_KV_FP16)
     bool mulshift;            // SA_FLAG_SHIFT_BY_MULTIPLY: the scores' shifts run on the integer multiplier
+    bool addalu;              // SA_FLAG_ADD_ON_ALU: sign flips and adds as logic/add instructions, no multiply-add
     bool fp16, nibble, hadamard, int8;   // nibble: 4-bit sign/exponent codes (PoT-4 nibble container, or with k = 1, 2
                                          // the dense planar container); int8: the uniform INT8 comparison code
     int F;                    // head-room actually used
@@ -59,6 +60,9 @@ constexpr KernelShape decode_shape(int d, int kb) {
                                 : KernelShape{4, 5};
 }
 constexpr KernelShape kFp16Shape{4, 3};
+// Streaming multiprocessors of the current device (cudaDevAttrMultiProcessorCount, asked once per device; 148,
+// a B200, where no device answers, so that the size queries also work on a machine without a GPU).
+int sm_count();
 // number of splits of the key axis for a cache of this shape, and queries handled per block
 void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt);
 

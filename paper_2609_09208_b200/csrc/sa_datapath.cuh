@@ -35,6 +35,18 @@ SA_HD uint32_t shl_clamp_hd(uint32_t x, uint32_t n) {
     return n >= 32u ? 0u : (x << n);
 #endif
 }
+// Ablation only (SA_ABLATE_SIGNED_SHIFT): a shift whose direction is decided per term, as a datapath without
+// head-room would need: amount r - 3, left when that is non-negative, else arithmetic right (dropping bits).
+SA_HD uint32_t shl_signed_hd(uint32_t x, uint32_t r) {
+    const int rs = (int)r - 3;
+    const uint32_t left = shl_clamp_hd(x, (uint32_t)rs), right = (uint32_t)((int32_t)x >> ((-rs) & 31));
+    return rs >= 0 ? left : right;
+}
+#ifdef SA_ABLATE_SIGNED_SHIFT
+#define SA_TERM_SHIFT shl_signed_hd
+#else
+#define SA_TERM_SHIFT shl_clamp_hd
+#endif
 SA_HD int popc_hd(uint32_t x) {
 #ifdef __CUDA_ARCH__
     return __popc(x);
@@ -102,6 +114,10 @@ SA_HD uint32_t mad_fma(uint32_t a, uint32_t w, uint32_t c) {
 #endif
 }
 
+// c + x with the sign flip of x chosen by the mask s (0: +x, 0xffffffff: -x) done as exclusive-or and
+// subtract: logic and add instructions only, no multiplier.
+SA_HD uint32_t flip_add(uint32_t x, uint32_t s, uint32_t c) { return c + ((x ^ s) - s); }
+
 SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (uint32_t)q_lo; }
 
 // Accumulators for 2 * NP queries against one PoT-4 key.
@@ -112,7 +128,9 @@ SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (
 // and at the end  lower-query sum = tot - (hit << 16) - bias  (exact: the true value is far below
 // 2^32) and  upper-query sum = hit.  That is one ALU instruction and two FMA-pipe adds per window
 // register.
-template <int NP>
+// ALU (SA_FLAG_ADD_ON_ALU, not the default): sg is a sign MASK (0 / 0xffffffff) and every sign flip and add
+// is an exclusive-or, a subtract and an add on the ALU pipe; the multiplier array is not used at all.
+template <int NP, bool ALU = false>
 struct PackedShift {
     uint32_t win[NP];           // window sums, lower half biased by 0x8000
     uint32_t tot[NP], hit[NP];  // running totals, see above
@@ -125,22 +143,22 @@ struct PackedShift {
 #pragma unroll
         for (int p = 0; p < NP; ++p) tot[p] = hit[p] = 0;
     }
-    // sg: +1 or -1; x: the element's packed pairs, already shifted (an entry of ShiftTable)
+    // sg: +1 or -1 (ALU: the sign mask); x: the element's packed pairs, already shifted (an entry of ShiftTable)
     SA_HD void entry_first(uint32_t sg, const uint32_t (&x)[NP]) {
 #pragma unroll
-        for (int p = 0; p < NP; ++p) win[p] = mad_fma(x[p], sg, 0x8000u);
+        for (int p = 0; p < NP; ++p) win[p] = ALU ? flip_add(x[p], sg, 0x8000u) : mad_fma(x[p], sg, 0x8000u);
     }
     SA_HD void entry_next(uint32_t sg, const uint32_t (&x)[NP]) {
 #pragma unroll
-        for (int p = 0; p < NP; ++p) win[p] = mad_fma(x[p], sg, win[p]);
+        for (int p = 0; p < NP; ++p) win[p] = ALU ? flip_add(x[p], sg, win[p]) : mad_fma(x[p], sg, win[p]);
     }
     SA_HD void window_end() {
         ++n_windows;
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
             const uint32_t h = (uint32_t)((int32_t)win[p] >> 16);      // exact upper half
-            tot[p] = add_fma(win[p], tot[p], one);
-            hit[p] = add_fma(h, hit[p], one);
+            tot[p] = ALU ? win[p] + tot[p] : add_fma(win[p], tot[p], one);
+            hit[p] = ALU ? h + hit[p] : add_fma(h, hit[p], one);
         }
     }
     // score of query g (g even: lower half of register g / 2), before the final head-room shift
@@ -197,45 +215,46 @@ SA_HD void shift_gather(const uint8_t* base, uint32_t offs, int i, uint32_t (&x)
 
 // Elements I .. 3 of one window: element E0 + STEP * I of the group, byte I of offs and of sw (sign at the
 // byte's top bit).
-template <int NP, int E0, int STEP, int I, typename Base>
-SA_HD void shift_window(PackedShift<NP>& pl, uint32_t sw, uint32_t offs, Base grp) {
+template <int NP, int E0, int STEP, int I, bool ALU, typename Base>
+SA_HD void shift_window(PackedShift<NP, ALU>& pl, uint32_t sw, uint32_t offs, Base grp) {
     if constexpr (I < 4) {
         using ST = ShiftTable<NP>;
         constexpr int e = E0 + STEP * I;
         uint32_t x[NP];
         shift_gather<NP, ST::high(e)>(grp, offs, I, x);
-        const uint32_t sg = mad_fma(prmt_hd(sw, 0u, 0x8888u | (0x1111u * I)), pl.one + pl.one, pl.one);   // +1 / -1
+        const uint32_t sm = prmt_hd(sw, 0u, 0x8888u | (0x1111u * I));                 // sign mask: 0 / 0xffffffff
+        const uint32_t sg = ALU ? sm : mad_fma(sm, pl.one + pl.one, pl.one);          // +1 / -1
         if (I == 0) pl.entry_first(sg, x);
         else pl.entry_next(sg, x);
-        shift_window<NP, E0, STEP, I + 1>(pl, sw, offs, grp);
+        shift_window<NP, E0, STEP, I + 1, ALU>(pl, sw, offs, grp);
     }
 }
 
 // One 32-bit word of the byte container = 4 elements: word W4 (0 .. 3) of a group of 16 elements whose
 // table rows start at grp (256-byte aligned).
-template <int NP, int W4, typename Base>
-SA_HD void accumulate_word_bytes_tab(PackedShift<NP>& pl, uint32_t w, Base grp) {
+template <int NP, int W4, bool ALU, typename Base>
+SA_HD void accumulate_word_bytes_tab(PackedShift<NP, ALU>& pl, uint32_t w, Base grp) {
     using ST = ShiftTable<NP>;
     constexpr uint32_t pattern = ST::low(W4 * 4) | (ST::low(W4 * 4 + 1) << 8) | (ST::low(W4 * 4 + 2) << 16) | (ST::low(W4 * 4 + 3) << 24);
     const uint32_t offs = ((w << ST::kShift) & (0x07070707u << ST::kShift)) | pattern;      // g * entry bytes + row
-    shift_window<NP, W4 * 4, 1, 0>(pl, w, offs, grp);
+    shift_window<NP, W4 * 4, 1, 0, ALU>(pl, w, offs, grp);
     pl.window_end();
 }
 
 // One 32-bit word of the nibble container = 8 elements (low nibble = even element), two windows: the even
 // and the odd elements (the order of the terms within the exact sum is free).  grp: the rows of the word's
 // first element (256-byte aligned).
-template <int NP, typename Base>
-SA_HD void accumulate_word_nibbles_tab(PackedShift<NP>& pl, uint32_t w, Base grp) {
+template <int NP, bool ALU, typename Base>
+SA_HD void accumulate_word_nibbles_tab(PackedShift<NP, ALU>& pl, uint32_t w, Base grp) {
     using ST = ShiftTable<NP>;
     constexpr uint32_t pat_e = ST::low(0) | (ST::low(2) << 8) | (ST::low(4) << 16) | (ST::low(6) << 24);
     constexpr uint32_t pat_o = ST::low(1) | (ST::low(3) << 8) | (ST::low(5) << 16) | (ST::low(7) << 24);
     const uint32_t we = w << 4;                                          // even elements' sign at the byte's top bit
     const uint32_t offs_e = ((w << ST::kShift) & (0x07070707u << ST::kShift)) | pat_e;
     const uint32_t offs_o = ((w >> (4 - ST::kShift)) & (0x07070707u << ST::kShift)) | pat_o;
-    shift_window<NP, 0, 2, 0>(pl, we, offs_e, grp);
+    shift_window<NP, 0, 2, 0, ALU>(pl, we, offs_e, grp);
     pl.window_end();
-    shift_window<NP, 1, 2, 0>(pl, w, offs_o, grp);
+    shift_window<NP, 1, 2, 0, ALU>(pl, w, offs_o, grp);
     pl.window_end();
 }
 
@@ -280,8 +299,11 @@ SA_HD void table_gather(const uint8_t* base, uint32_t offs, int i, uint32_t& x, 
 
 // MUL (SA_FLAG_SHIFT_BY_MULTIPLY, not the default): sigma * 2^r is formed once per key element and the
 // update is one multiply-add of the table entry by it.
-template <int KB, int NGP, bool MUL = false>
+// ALU (SA_FLAG_ADD_ON_ALU, not the default): the sign flip and the add are an exclusive-or, a subtract and an
+// add on the ALU pipe (sg is then the sign mask 0 / 0xffffffff); the multiplier array is not used at all.
+template <int KB, int NGP, bool MUL = false, bool ALU = false>
 struct TableScore {
+    static_assert(!(MUL && ALU), "the two variants exclude one another");
     static constexpr int kRowBytes = 8 << KB;              // one (element, query pair) row
     static constexpr int kElemBytes = NGP * kRowBytes;     // all query pairs of one element
     static constexpr int kGroupBytes = 16 * kElemBytes;    // 16 elements = 4 code words; a multiple of 256
@@ -300,8 +322,10 @@ struct TableScore {
         if constexpr (GP < NGP) {
             uint32_t x, y;
             table_gather<IMM + GP * kRowBytes>(grp, offs, i, x, y);
-            acc[2 * GP] = MUL ? mad_fma(x, sg, acc[2 * GP]) : mad_fma(shl_clamp_hd(x, r), sg, acc[2 * GP]);
-            acc[2 * GP + 1] = MUL ? mad_fma(y, sg, acc[2 * GP + 1]) : mad_fma(shl_clamp_hd(y, r), sg, acc[2 * GP + 1]);
+            acc[2 * GP] = MUL ? mad_fma(x, sg, acc[2 * GP])
+                          : ALU ? flip_add(SA_TERM_SHIFT(x, r), sg, acc[2 * GP]) : mad_fma(SA_TERM_SHIFT(x, r), sg, acc[2 * GP]);
+            acc[2 * GP + 1] = MUL ? mad_fma(y, sg, acc[2 * GP + 1])
+                              : ALU ? flip_add(SA_TERM_SHIFT(y, r), sg, acc[2 * GP + 1]) : mad_fma(SA_TERM_SHIFT(y, r), sg, acc[2 * GP + 1]);
             element_pairs<IMM, GP + 1>(grp, offs, i, r, sg);
         }
     }
@@ -309,7 +333,8 @@ struct TableScore {
     SA_HD void elements(uint32_t w, uint32_t rw, uint32_t offs, Base grp) {
         if constexpr (I < 4) {
             const uint32_t r = prmt_hd(rw, 0u, 0x4440u | I);
-            const uint32_t sg = mad_fma(prmt_hd(w, 0u, 0x8888u | (0x1111u * I)), two, one);   // sigma: 0 / -1 -> +1 / -1
+            const uint32_t sm = prmt_hd(w, 0u, 0x8888u | (0x1111u * I));                      // sign mask: 0 / 0xffffffff
+            const uint32_t sg = ALU ? sm : mad_fma(sm, two, one);                             // sigma: +1 / -1
             element_pairs<(W4 * 4 + I) * kElemBytes, 0>(grp, offs, I, r, MUL ? shl_clamp_hd(sg, r) : sg);
             elements<W4, I + 1>(w, rw, offs, grp);
         }
@@ -333,7 +358,8 @@ struct TableScore {
         if constexpr (NI < 8) {
             constexpr int byte = NI >> 1;
             const uint32_t r = prmt_hd((NI & 1) ? ro : re, 0u, 0x4440u | byte);
-            const uint32_t sg = mad_fma(prmt_hd((NI & 1) ? w : we, 0u, 0x8888u | (0x1111u * byte)), two, one);
+            const uint32_t sm = prmt_hd((NI & 1) ? w : we, 0u, 0x8888u | (0x1111u * byte));
+            const uint32_t sg = ALU ? sm : mad_fma(sm, two, one);
             element_pairs<(W8 * 8 + NI) * kElemBytes, 0>(grp, (NI & 1) ? offs_o : offs_e, byte, r, MUL ? shl_clamp_hd(sg, r) : sg);
             nibble_elements<W8, NI + 1>(w, we, re, ro, offs_e, offs_o, grp);
         }

@@ -9,7 +9,7 @@ void launch_decode_fp16_main(const Plan& p, const DecodeArgs& a, int GT, cudaStr
 // The decode kernel for these arguments (the score pass of the shift-A.V option when a.zr is set).
 void launch_decode_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s) {
     const dim3 grid((unsigned)a.n_splits, (unsigned)(p.Hkv * (p.G / GT)), (unsigned)a.batch);
-    const int mode = a.zr ? 2 : (p.mulshift ? 1 : 0);            // a.zr: score pass of the shift-based A.V option
+    const int mode = a.zr ? 2 : (p.mulshift ? 1 : (p.addalu ? 3 : 0));   // a.zr: score pass of the shift-based A.V option
     if (p.int8) launch_decode_int8(p.d, a, GT, grid, s);
     else if (p.k == 0) launch_decode_pot4(p.nibble, p.d, mode, a, GT, grid, s);
     else if (p.k == 1) launch_decode_potm1(p.nibble, p.d, mode, a, GT, grid, s);
@@ -44,6 +44,28 @@ extern "C" sa_status sa_decode_attention_stages(const sa_config* cfg, const sa_c
     return (stages & 2) ? launch_merge(p, a, s) : SA_OK;
 }
 
+extern "C" sa_status sa_debug_decode_lost_copy(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q, float* O,
+                                               void* workspace, size_t workspace_bytes, int b, int kv_head, int tile,
+                                               sa_stream stream) {
+    Plan p;
+    sa_status st = make_plan(cfg, &p);
+    if (st != SA_OK) return st;
+    if (p.fp16 || p.int8 || p.nibble || p.d != 64 || p.k != 4 || p.G != 8 || p.mulshift || p.addalu) return SA_ERR_UNSUPPORTED;
+    DecodeArgs a;
+    int GT;
+    st = make_decode_args(p, cache, Q, O, workspace, workspace_bytes, &a, &GT);
+    if (st != SA_OK) return st;
+    if (b < 0 || b >= a.batch || kv_head < 0 || kv_head >= p.Hkv || tile < 0) return SA_ERR_INVALID_ARG;
+    a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / (double)(1LL << p.F));
+    a.lost_b = b;
+    a.lost_kvh = kv_head;
+    a.lost_tile = tile;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    launch_decode_potm4_lost_copy(a, dim3((unsigned)a.n_splits, (unsigned)p.Hkv, (unsigned)a.batch), s);
+    if (cudaGetLastError() != cudaSuccess) return SA_ERR_CUDA;
+    return launch_merge(p, a, s);
+}
+
 extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                                     const uint16_t* K_new, const uint16_t* V_new, float* O, void* workspace,
                                     size_t workspace_bytes, sa_stream stream) {
@@ -56,7 +78,12 @@ extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache,
     if (cache && cache->batch > 0 && cache->max_pages_per_seq > 0) split_plan(p, cache->batch, cache->max_pages_per_seq, &S, &GT);
     else GT = 0;
     if (GT != p.G) {
-        // a query group wider than one block: the separate append kernel
+        // a query group wider than one block: the separate append kernel.  Everything the decode call will check
+        // is checked first, so that a call that fails has neither written the token nor moved the length.
+        DecodeArgs probe;
+        int gt_probe;
+        st = make_decode_args(p, cache, Q, O, workspace, workspace_bytes, &probe, &gt_probe);
+        if (st != SA_OK) return st;
         st = sa_append_kv(cfg, cache, K_new, V_new, 1, stream);
         if (st != SA_OK) return st;
         return p.fp16 ? sa_decode_attention_fp16(cfg, cache, Q, O, workspace, workspace_bytes, stream)

@@ -29,6 +29,8 @@ struct DecodeArgs {
     // Fused cache append (sa_decode_step); null on the plain decode path.
     const uint16_t* Knew;     // [batch][Hkv][D] binary16: the step's new token, written at position seq_lens[b]
     const uint16_t* Vnew;
+    // Test hook (sa_debug_decode_lost_copy): the copy of this tile of this (sequence, KV head) is never issued.
+    int lost_b, lost_kvh, lost_tile;
 };
 
 // red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace
@@ -64,7 +66,7 @@ SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2]
 template <int D, int GT, int NW>
 SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], const int (&M)[GT],
                                 float (&l)[GT], float (&acc)[D / 16][4], int lane, int warp, int b, int h0,
-                                int split) {
+                                int split, bool failed = false) {
     const int gq = lane >> 2, t4 = lane & 3;
     float lsum[GT];
 #pragma unroll
@@ -72,7 +74,10 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
         lsum[g] = warp_sum_f32(l[g]);
         if (lane == 0) red_s[warp][g][0] = __int_as_float(M[g]);
     }
-    __syncthreads();
+    // A warp whose bounded wait for a copy expired makes the block's whole partial a marked one: l = NaN is
+    // written below from a register, not through the scratch rows, which alias the stage buffers — a copy that
+    // was merely late could still land in them.
+    const bool poisoned = __syncthreads_or(failed ? 1 : 0) != 0;
     if (threadIdx.x < GT) {
         int Mb = kMNone;
 #pragma unroll
@@ -115,6 +120,7 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
 #pragma unroll
             for (int w = 1; w < NW; ++w) v += red_s[w][g][c];
         }
+        if (poisoned && c <= 1) v = (c == 0) ? __int_as_float(0) : __int_as_float(0x7fc00000);   // M = 0, l = NaN
         a.partials[(((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2) + c] = v;
     }
 }
@@ -274,6 +280,7 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->k_max = 0;
     a->Knew = nullptr;
     a->Vnew = nullptr;
+    a->lost_b = a->lost_kvh = a->lost_tile = -1;
     *gt = GT;
     return SA_OK;
 }

@@ -14,6 +14,15 @@
 // values are exact, every weight is split into two tf32 terms, accumulation in FP32).  The warps'
 // states and then the blocks' partial results are merged with exact power-of-two factors.
 // For sa_decode_step the warp that owns the new token's tile writes the token first (section II-F).
+//
+// Compile-time switches for ablation measurements only (section V-F of the paper lists the three design choices;
+// each switch removes one of them from every instantiation, `python -m paper_2609_09208_b200.build -DNAME`):
+//   SA_ABLATE_WORD_STAGING   a warp stages its tile itself with 32-bit loads and stores instead of one 16-byte
+//                            aligned bulk-async copy, and reads the key codes back 32 bits at a time instead of 128
+//   SA_ABLATE_SIGNED_SHIFT   the mantissa codes' shift without head-room: a signed amount (here F = 3 instead of
+//                            6 + k), the direction decided per term — a right shift drops bits, so the scores of
+//                            such a build are NOT the exact ones and its tests fail by design
+//   SA_ABLATE_NO_MIN_BLOCKS  __launch_bounds__ without the resident-blocks clause (the register cap)
 #include "sa_common.cuh"
 #include "sa_cache_write.cuh"
 #include "sa_datapath.cuh"
@@ -58,10 +67,16 @@ struct DecodeSmem {
 };
 
 template <int D, int KB, bool NIB, int GT, int MODE = 0>
+#ifdef SA_ABLATE_NO_MIN_BLOCKS
+__global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW)) decode_kernel(DecodeArgs a) {
+#else
 __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (DecodeSmem<D, KB, NIB, GT>::kBlocksPerSM)) decode_kernel(DecodeArgs a) {
+#endif
     // MODE 0: the decode kernel; 1: the same with SA_FLAG_SHIFT_BY_MULTIPLY; 2: the score pass of the shift-based
     // A.V option (a.zr set: rounded logits and statistics instead of softmax and A.V), kept out of the other two
-    constexpr bool MUL = (MODE == 1), SP = (MODE == 2);
+    // 3: the same with SA_FLAG_ADD_ON_ALU; 4: the test hook that never issues one chosen tile's copy (sa_debug_decode_lost_copy)
+    constexpr bool MUL = (MODE == 1), SP = (MODE == 2), ALUO = (MODE == 3), LOST = (MODE == 4);
+    constexpr uint32_t kPolls = LOST ? (1u << 10) : kWaitLimit;
     // KB = 0: PoT-4 (packed shift datapath); KB = 1, 2, 4: mantissa codes (table datapath);
     // KB = 8: uniform INT8 comparison code (dp4a).  MUL: the shifts run on the integer multiplier
     // (SA_FLAG_SHIFT_BY_MULTIPLY; same scores, reported separately from the shift kernels).
@@ -259,10 +274,12 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     }
     // Lane 0: start the copies of my i-th tile into stage i % NS.  A tile whose page is not
     // mapped gets a plain arrival instead (the phase completes, the tile is skipped below).
+#ifndef SA_ABLATE_WORD_STAGING
     auto issue = [&](int i) {
         const int tile = first + NW * i;
         const int pidx = (tile == tile_g) ? pidx_g : a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
         const int s = i % NS;
+        if (LOST && tile == a.lost_tile && b == a.lost_b && kvh == a.lost_kvh) return;   // test hook: this copy never starts
         if (pidx < 0 || pidx >= a.n_pages) {
             mbar_arrive(mbar0 + s * 8);
         } else {
@@ -273,6 +290,23 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     };
     if (lane == 0)
         for (int i = 0; i < NS && i < n_my; ++i) issue(i);
+#else
+    // ablation: the whole warp copies the tile word by word; lane 0 then completes the stage's barrier phase
+    auto issue = [&](int i) {
+        const int tile = first + NW * i;
+        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int s = i % NS;
+        if (pidx >= 0 && pidx < a.n_pages) {
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(a.pages + ((size_t)pidx * a.Hkv + kvh) * a.page_bytes +
+                                                                    (size_t)(tile & 1) * Stage::kBytes);
+            uint32_t* dst = reinterpret_cast<uint32_t*>(smem + SM::kStageOff + (warp * NS + s) * Stage::kBytes);
+            for (int w = lane; w < Stage::kBytes / 4; w += 32) dst[w] = __ldcg(src + w);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(mbar0 + s * 8);
+    };
+    for (int i = 0; i < NS && i < n_my; ++i) issue(i);
+#endif
 
     int M[GT];
     float Mf[GT];            // M as a float (exact below 2^24)
@@ -299,11 +333,11 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         const int s = i % NS;
         const uint32_t parity = (uint32_t)(i / NS) & 1u;
         // the decision is made warp-uniform: a lane must never leave the loop alone
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(mbar0 + s * 8, parity))) {
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(mbar0 + s * 8, parity, kPolls))) {
             failed = true;
             // give the other stage's copy (already issued) a bounded chance to land before this
             // warp's buffers are re-used by the block merge
-            if (NS > 1 && i + 1 < n_my) (void)mbar_wait_bounded(mbar0 + ((i + 1) % NS) * 8, (uint32_t)((i + 1) / NS) & 1u);
+            if (NS > 1 && i + 1 < n_my) (void)mbar_wait_bounded(mbar0 + ((i + 1) % NS) * 8, (uint32_t)((i + 1) / NS) & 1u, kPolls);
             break;
         }
         const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
@@ -317,14 +351,14 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             int32_t A[GT];
             const uint32_t* cw = reinterpret_cast<const uint32_t*>(st) + lane * 4;
             if constexpr (SM::kTable) {
-                using TS = TableScore<KB, NP, MUL>;
+                using TS = TableScore<KB, NP, MUL, ALUO>;
                 uint32_t grp = smem_addr(smem + SM::kQpOff);    // table of the next 16 elements (256-byte aligned)
                 TS ts;
                 ts.begin(a.one);
                 if constexpr (!NIB) {
 #pragma unroll 1
                     for (int c = 0; c < WORDS / 4; ++c, grp += TS::kGroupBytes) {
-                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        const uint4 w4 = load_code_chunk(cw + c * 128);
                         ts.template accumulate_word<0>(w4.x, grp);
                         ts.template accumulate_word<1>(w4.y, grp);
                         ts.template accumulate_word<2>(w4.z, grp);
@@ -336,7 +370,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                     const uint32_t* pw = reinterpret_cast<const uint32_t*>(st + Stage::kPlaneOff) + lane * (D / 32);
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
-                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        const uint4 w4 = load_code_chunk(cw + c * 128);
                         uint32_t pb[KB];
 #pragma unroll
                         for (int bit = 0; bit < KB; ++bit) pb[bit] = pw[bit * (Stage::kPlaneBytes / 4) + c];
@@ -362,13 +396,13 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             } else if constexpr (KB != 8) {
                 // PoT-4: the packed pairs, shifted ahead of the loop, are looked up by the key's exponent field
                 using ST = ShiftTable<NP>;
-                PackedShift<NP> pl;
+                PackedShift<NP, ALUO> pl;
                 pl.begin(a.one);
                 uint32_t grp = smem_addr(smem + SM::kQpOff);     // rows of the next group of elements (256-byte aligned)
                 if constexpr (!NIB) {
 #pragma unroll 1
                     for (int c = 0; c < D / 16; ++c, grp += 16 * ST::kRowBytes) {
-                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        const uint4 w4 = load_code_chunk(cw + c * 128);
                         accumulate_word_bytes_tab<NP, 0>(pl, w4.x, grp);
                         accumulate_word_bytes_tab<NP, 1>(pl, w4.y, grp);
                         accumulate_word_bytes_tab<NP, 2>(pl, w4.z, grp);
@@ -377,7 +411,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 } else {
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c, grp += 32 * ST::kRowBytes) {
-                        const uint4 w4 = *reinterpret_cast<const uint4*>(cw + c * 128);
+                        const uint4 w4 = load_code_chunk(cw + c * 128);
                         accumulate_word_nibbles_tab<NP>(pl, w4.x, grp);
                         accumulate_word_nibbles_tab<NP>(pl, w4.y, grp + 8 * ST::kRowBytes);
                         accumulate_word_nibbles_tab<NP>(pl, w4.z, grp + 16 * ST::kRowBytes);
@@ -420,10 +454,14 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
                 }
                 g_min = min(g_min, valid ? g_j : 0x7fffffff);
                 __syncwarp();
+#ifndef SA_ABLATE_WORD_STAGING
                 if (lane == 0 && i + NS < n_my) {
                     fence_proxy_async();
                     issue(i + NS);
                 }
+#else
+                if (i + NS < n_my) issue(i + NS);
+#endif
                 continue;
             }
             // The weights go where the tile's key codes were (every lane is done with them): row =
@@ -514,10 +552,14 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
             }
         }
         __syncwarp();                                         // every lane is done with this stage
+#ifndef SA_ABLATE_WORD_STAGING
         if (lane == 0 && i + NS < n_my) {
             fence_proxy_async();
             issue(i + NS);
         }
+#else
+        if (i + NS < n_my) issue(i + NS);
+#endif
     }
     if constexpr (!SP) {
 #pragma unroll
@@ -556,7 +598,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
         return;
     }
-    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, b, h0, split);
+    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, b, h0, split, failed);
 }
 
 template <int D, int KB, bool NIB, int GT, int MODE>
@@ -583,17 +625,19 @@ static void launch_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
 
 // All instantiations of one key code and container: head_dim 64 / 128, the queries per block, and the
 // kernel's mode (0 decode; 1 the same with the shifts on the integer multiplier, mantissa codes only;
-// 2 the score pass of the shift-based A.V option, power-of-two codes only).
+// 2 the score pass of the shift-based A.V option, 3 sign flips and adds on the ALU pipe: power-of-two codes only).
 template <int KB, bool NIB>
 static void launch_code(int d, int mode, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     constexpr bool kPot = (KB != 8);
     constexpr bool kMul = (KB == 1 || KB == 2 || KB == 4);
     if (d == 64) {
         if (kPot && mode == 2) launch_gt<64, KB, NIB, kPot ? 2 : 0>(a, GT, grid, s);
+        else if (kPot && mode == 3) launch_gt<64, KB, NIB, kPot ? 3 : 0>(a, GT, grid, s);
         else if (kMul && mode == 1) launch_gt<64, KB, NIB, kMul ? 1 : 0>(a, GT, grid, s);
         else launch_gt<64, KB, NIB, 0>(a, GT, grid, s);
     } else {
         if (kPot && mode == 2) launch_gt<128, KB, NIB, kPot ? 2 : 0>(a, GT, grid, s);
+        else if (kPot && mode == 3) launch_gt<128, KB, NIB, kPot ? 3 : 0>(a, GT, grid, s);
         else if (kMul && mode == 1) launch_gt<128, KB, NIB, kMul ? 1 : 0>(a, GT, grid, s);
         else launch_gt<128, KB, NIB, 0>(a, GT, grid, s);
     }
@@ -604,6 +648,7 @@ void launch_decode_pot4(bool nib, int d, int mode, const DecodeArgs& a, int GT, 
 void launch_decode_potm1(bool nib, int d, int mode, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s);
 void launch_decode_potm2(bool nib, int d, int mode, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s);
 void launch_decode_potm4(int d, int mode, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s);
+void launch_decode_potm4_lost_copy(const DecodeArgs& a, dim3 grid, cudaStream_t s);   // test hook: head_dim 64, 8 queries per block
 void launch_decode_int8(int d, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s);
 
 }  // namespace sa

@@ -5,4 +5,7 @@ namespace sa {
 void launch_decode_potm4(int d, int mode, const DecodeArgs& a, int GT, dim3 grid, cudaStream_t s) {
     launch_code<4, false>(d, mode, a, GT, grid, s);
 }
+void launch_decode_potm4_lost_copy(const DecodeArgs& a, dim3 grid, cudaStream_t s) {
+    launch_one<64, 4, false, 8, 4>(a, grid, s);
+}
 }  // namespace sa

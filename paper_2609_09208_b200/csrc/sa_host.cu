@@ -1,6 +1,6 @@
 // Host side of the C ABI: configuration validation, page layout, split plan, and the
 // host-buffer convenience entry.  No kernels live here.
-#include "sa_common.cuh"
+#include "sa_decode_common.cuh"
 #include <cmath>
 
 namespace sa {
@@ -12,8 +12,11 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
         return SA_ERR_INVALID_ARG;
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return SA_ERR_UNSUPPORTED;
     if (cfg->page_tokens != kPageTokens) return SA_ERR_UNSUPPORTED;
-    if (cfg->flags & ~(SA_FLAG_HADAMARD | SA_FLAG_SHIFT_BY_MULTIPLY)) return SA_ERR_INVALID_ARG;
+    if (cfg->flags & ~(SA_FLAG_HADAMARD | SA_FLAG_SHIFT_BY_MULTIPLY | SA_FLAG_ADD_ON_ALU)) return SA_ERR_INVALID_ARG;
     p.mulshift = (cfg->flags & SA_FLAG_SHIFT_BY_MULTIPLY) != 0;
+    p.addalu = (cfg->flags & SA_FLAG_ADD_ON_ALU) != 0;
+    if (p.mulshift && p.addalu) return SA_ERR_INVALID_ARG;
+    if (p.addalu && (cfg->code == SA_KV_FP16 || cfg->code == SA_INT8)) return SA_ERR_UNSUPPORTED;   // no shift-and-add datapath there
     // no shift in the key loop to move: FP16 and INT8 have none, PoT-4 looks its shifted queries up
     if (p.mulshift && (cfg->code == SA_KV_FP16 || cfg->code == SA_INT8 || cfg->code == SA_POT4)) return SA_ERR_UNSUPPORTED;
     p.d = cfg->head_dim;
@@ -85,6 +88,24 @@ sa_status make_plan(const sa_config* cfg, Plan* out) {
     return SA_OK;
 }
 
+int sm_count() {
+    static int cached[64] = {};                               // 0: not asked yet (benign race: every thread stores the same value)
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        (void)cudaGetLastError();
+        return kNumSMsB200;
+    }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = kNumSMsB200;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt) {
     int GT = 1;
     for (int c = 8; c >= 1; c >>= 1)
@@ -95,14 +116,15 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
     //   * a block lasts about  r + c_fix  with r between tiles / (warps S) and its ceiling (warps that
     //     run out of tiles leave their issue slots to the others, but not all of the time), and
     //     c_fix for the prologue (query quantisation, table) and the block merge;
-    //   * blocks run in waves of 148 x resident-blocks-per-SM; a last wave whose SMs hold only the
+    //   * blocks run in waves of (SMs of the current device) x resident-blocks-per-SM; a last wave whose SMs hold only the
     //     fraction f of that takes 0.1 + 0.9 f of a full wave's time, a single partial wave f^0.2
     //     (an SM's throughput falls almost in proportion to its resident warps).
     // The sequence lengths live on the device, so the model uses the cache's capacity.
     const long long units = (long long)batch * p.Hkv * (p.G / GT);
     const KernelShape shape = p.fp16 ? kFp16Shape : decode_shape(p.d, p.int8 ? 8 : p.k);
     const int bps = shape.blocks_per_sm, nw = shape.warps;
-    const long long slots = (long long)kNumSMs * bps;
+    const int n_sms = sm_count();
+    const long long slots = (long long)n_sms * bps;
     const long long tiles = (long long)max_pages * (kPageTokens / 32);
     long long cap = tiles / 2;                      // at least two tiles per block (short caches: spread them over the SMs)
     if (cap < 1) cap = 1;
@@ -117,7 +139,7 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
         const long long full = blocks / slots, rest = blocks % slots;
         double cost = (double)full * block_time;
         if (rest) {
-            const double fill = (double)((rest + kNumSMs - 1) / kNumSMs) / (double)bps;
+            const double fill = (double)((rest + n_sms - 1) / n_sms) / (double)bps;
             // behind full waves a partial one overlaps their stragglers; on its own it does not
             cost += block_time * (full ? 0.1 + 0.9 * fill : pow(fill, 0.2));
         }
@@ -235,7 +257,16 @@ sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const
                         cudaHostGetDevicePointer(&mo, O_host, 0) == cudaSuccess;
     (void)cudaGetLastError();                                    // a pageable buffer is not an error here
     auto al16 = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; };
-    if (mapped && al16(mq) && al16(mk) && al16(mv) && al16(mo) && q % 16 == 0 && kv % 16 == 0) {
+    const bool direct = mapped && al16(mq) && al16(mk) && al16(mv) && al16(mo) && q % 16 == 0 && kv % 16 == 0;
+    {
+        // everything sa_decode_step will check, checked before a kernel or a copy is enqueued: a call that
+        // returns an error has launched nothing
+        DecodeArgs probe;
+        int gt_probe;
+        st = make_decode_args(p, cache, dQ, direct ? static_cast<float*>(mo) : dO, workspace, workspace_bytes, &probe, &gt_probe);
+        if (st != SA_OK) return st;
+    }
+    if (direct) {
         const int nq = (int)(q / 16), nkv = (int)(kv / 16);
         const unsigned blocks = (unsigned)((nq + 2 * nkv + 255) / 256);
         if (launch_pdl(stage_in_kernel, dim3(blocks), dim3(256), 0, s, (const uint4*)mq, (const uint4*)mk, (const uint4*)mv,

@@ -41,11 +41,26 @@ SA_D bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait for a phase; false if it did not complete within kWaitLimit polls.
-SA_D bool mbar_wait_bounded(uint32_t mbar, uint32_t parity) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it)
+// Bounded wait for a phase; false if it did not complete within `limit` polls.
+SA_D bool mbar_wait_bounded(uint32_t mbar, uint32_t parity, uint32_t limit = kWaitLimit) {
+    for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(mbar, parity)) return true;
     return false;
+}
+// The 16 bytes of key codes of this lane's key in one chunk of a staged tile (one 128-bit load; with
+// SA_ABLATE_WORD_STAGING four 32-bit loads that the compiler may not merge).
+SA_D uint4 load_code_chunk(const uint32_t* p) {
+#ifndef SA_ABLATE_WORD_STAGING
+    return *reinterpret_cast<const uint4*>(p);
+#else
+    uint4 v;
+    const uint32_t addr = smem_addr(p);
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v.x) : "r"(addr));
+    asm volatile("ld.shared.u32 %0, [%1+4];" : "=r"(v.y) : "r"(addr));
+    asm volatile("ld.shared.u32 %0, [%1+8];" : "=r"(v.z) : "r"(addr));
+    asm volatile("ld.shared.u32 %0, [%1+12];" : "=r"(v.w) : "r"(addr));
+    return v;
+#endif
 }
 // global -> shared bulk copy; size and both addresses are multiples of 16 bytes
 SA_D void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {

@@ -7,6 +7,7 @@ using namespace sa;
 
 // Scores of one PoT-4 key (canonical code bytes) against 8 queries, through the same packed
 // datapath and word decoders the decode kernel uses (byte container: phys_byte; nibbles: canonical nibble ^ 7).
+template <bool ALU>
 static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool nibble_path, int32_t* out) {
     using ST = ShiftTable<4>;
     alignas(256) static uint8_t tab[128 * ST::kRowBytes];          // S[m][g][pair]: the shifted packed pairs
@@ -15,7 +16,7 @@ static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool ni
             for (int p = 0; p < 4; ++p)
                 reinterpret_cast<uint32_t*>(tab)[(m * 8 + g) * 4 + p] =
                     ST::entry(pack_pair(q8[(2 * p) * d + m], q8[(2 * p + 1) * d + m]), g);
-    PackedShift<4> pl;
+    PackedShift<4, ALU> pl;
     pl.begin(1u);
     if (!nibble_path) {
         for (int m0 = 0; m0 < d; m0 += 16) {
@@ -39,9 +40,10 @@ static void score8_packed(const uint8_t* canon, const int8_t* q8, int d, bool ni
 
 // The scores of a mantissa code (k = 1, 2, 4) through the table datapath.
 // The same scores through the table datapath of the mantissa codes.
-template <int K, bool MUL>
+// VAR 0: the default datapath; 1: the shifts as multiplications by 2^r; 2: sign flips and adds on the ALU pipe only
+template <int K, int VAR>
 static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
-    using TS = TableScore<K, 4, MUL>;
+    using TS = TableScore<K, 4, VAR == 1, VAR == 2>;
     alignas(256) static uint8_t tab[128 * TS::kElemBytes];
     for (int m = 0; m < d; ++m)
         for (int gp = 0; gp < 4; ++gp)
@@ -62,9 +64,9 @@ static void score8_table(const uint8_t* canon, const int8_t* q8, int d, int32_t*
 
 // The same through the dense planar container (k = 1, 2): sign/exponent nibbles, two per byte, and the
 // mantissa bits in k separate bit planes.
-template <int K, bool MUL>
+template <int K, int VAR>
 static void score8_planar(const uint8_t* canon, const int8_t* q8, int d, int32_t* out) {
-    using TS = TableScore<K, 4, MUL>;
+    using TS = TableScore<K, 4, VAR == 1, VAR == 2>;
     alignas(256) static uint8_t tab[128 * TS::kElemBytes];
     for (int m = 0; m < d; ++m)
         for (int gp = 0; gp < 4; ++gp)
@@ -88,23 +90,25 @@ static void score8_planar(const uint8_t* canon, const int8_t* q8, int d, int32_t
     for (int g = 0; g < 8; ++g) out[g] = ts.score(g);
 }
 
-template <bool MUL>
+template <int VAR>
 static void score8_any(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) {
     // path 0: byte container (packed datapath for k = 0, table datapath otherwise); 1: nibble container
     // (k = 0) or dense planar container (k = 1, 2)
-    if (k == 0) score8_packed(canon, q8, d, path != 0, out);            // PoT-4 has one datapath
-    else if (path != 0 && k == 1) score8_planar<1, MUL>(canon, q8, d, out);
-    else if (path != 0 && k == 2) score8_planar<2, MUL>(canon, q8, d, out);
-    else if (k == 1) score8_table<1, MUL>(canon, q8, d, out);
-    else if (k == 2) score8_table<2, MUL>(canon, q8, d, out);
-    else score8_table<4, MUL>(canon, q8, d, out);
+    if (k == 0) score8_packed<VAR == 2>(canon, q8, d, path != 0, out);  // PoT-4 has no multiply variant
+    else if (path != 0 && k == 1) score8_planar<1, VAR>(canon, q8, d, out);
+    else if (path != 0 && k == 2) score8_planar<2, VAR>(canon, q8, d, out);
+    else if (k == 1) score8_table<1, VAR>(canon, q8, d, out);
+    else if (k == 2) score8_table<2, VAR>(canon, q8, d, out);
+    else score8_table<4, VAR>(canon, q8, d, out);
 }
 
 extern "C" {
-void hh_score8_planar(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) { score8_any<false>(k, canon, q8, d, 1, out); }
-void hh_score8_table(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) { score8_any<false>(k, canon, q8, d, 0, out); }
+void hh_score8_planar(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) { score8_any<0>(k, canon, q8, d, 1, out); }
+void hh_score8_table(int k, const uint8_t* canon, const int8_t* q8, int d, int32_t* out) { score8_any<0>(k, canon, q8, d, 0, out); }
 // the same datapaths with the shifts executed as multiplications by 2^r
-void hh_score8_mul(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) { score8_any<true>(k, canon, q8, d, path, out); }
+void hh_score8_mul(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) { score8_any<1>(k, canon, q8, d, path, out); }
+// ... and with every sign flip and add on the ALU pipe (exclusive-or, subtract, add)
+void hh_score8_alu(int k, const uint8_t* canon, const int8_t* q8, int d, int path, int32_t* out) { score8_any<2>(k, canon, q8, d, path, out); }
 int hh_encode_element(int k, unsigned a_bits, unsigned s_bits) {
     switch (k) {
         case 0: return encode_element<0>(a_bits, s_bits);
@@ -118,6 +122,6 @@ void hh_encode_many(int k, const uint16_t* a_bits, int64_t n, unsigned s_bits, u
 }
 int hh_value_exponent(unsigned amax_bits) { return value_exponent(amax_bits); }
 void hh_score8(int k, const uint8_t* canon, const int8_t* q8, int d, int nibble_path, int32_t* out) {
-    score8_any<false>(k, canon, q8, d, k == 0 ? nibble_path : 0, out);
+    score8_any<0>(k, canon, q8, d, k == 0 ? nibble_path : 0, out);
 }
 }

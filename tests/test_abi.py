@@ -136,6 +136,64 @@ def test_entry_points_reject_bad_arguments_before_any_cuda_call():
     assert lib.sa_debug_unpack(C.byref(cfg), C.byref(cache), C.c_int(0), C.c_int(4 * 64 + 1), null, null, null, null, null) == 4
 
 
+def test_step_entries_check_the_decode_arguments_before_they_launch_anything():
+    """sa_decode_step with a query group wider than one block appends with a separate kernel, and sa_decode_step_host
+    stages its inputs first: both must have checked the decode call's arguments before that.  Without a GPU a
+    launch attempt would come back as a CUDA error (5); the argument errors must win."""
+    lib = sa.lib()
+    null, one = C.c_void_p(0), C.c_void_p(256)
+    wide = sa.make_config(64, 32, 2, sa.SA_POTM4)            # 16 query heads per KV head: the separate append
+    cache = sa.SaCache(256, 256, 256, 1, 4, 4)
+    need = sa.workspace_bytes(wide, 1, 4)
+    step = lambda cfg, ws, nbytes, O=one: lib.sa_decode_step(C.byref(cfg), C.byref(cache), one, one, one, O, ws,
+                                                             C.c_size_t(nbytes), null)
+    assert step(wide, one, need - 1) == 4                    # short workspace
+    assert step(wide, null, need) == 4
+    assert step(wide, one, need, null) == 1                  # no output
+    assert step(wide, C.c_void_p(260), need) == 3            # misaligned workspace
+    ok = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    assert step(ok, one, sa.workspace_bytes(ok, 1, 4) - 1) == 4
+    # the host-buffer entry: cache pointers, alignment and workspace are checked before the staging transfers
+    stg = sa.staging_bytes(ok, 1)
+    host = lambda c, ws_bytes: lib.sa_decode_step_host(C.byref(ok), C.byref(c), one, one, one, one, one, C.c_size_t(stg),
+                                                        one, C.c_size_t(ws_bytes), null)
+    assert host(sa.SaCache(0, 256, 256, 1, 4, 4), 1 << 30) == 1
+    assert host(sa.SaCache(264, 256, 256, 1, 4, 4), 1 << 30) == 3
+    assert host(cache, 8) == 4
+
+
+def test_flag_combinations():
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POTM4, add_on_alu=True)) == 0
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POT4, nibble=True, add_on_alu=True)) == 0
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_POTM4, add_on_alu=True, shift_by_multiply=True)) == 1
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_INT8, add_on_alu=True)) == 2
+    assert _status(sa.get_layout, sa.make_config(64, 32, 4, sa.SA_KV_FP16, add_on_alu=True)) == 2
+
+
+def test_lost_copy_hook_validates_on_the_host():
+    lib = sa.lib()
+    null, one = C.c_void_p(0), C.c_void_p(256)
+    cache = sa.SaCache(256, 256, 256, 2, 4, 8)
+    ok = sa.make_config(64, 32, 4, sa.SA_POTM4)
+    call = lambda cfg, b, h, t, nbytes=1 << 30: lib.sa_debug_decode_lost_copy(
+        C.byref(cfg), C.byref(cache), one, one, one, C.c_size_t(nbytes), C.c_int(b), C.c_int(h), C.c_int(t), null)
+    assert call(sa.make_config(64, 32, 4, sa.SA_POTM1), 0, 0, 0) == 2
+    assert call(sa.make_config(128, 32, 4, sa.SA_POTM4), 0, 0, 0) == 2
+    assert call(sa.make_config(64, 16, 4, sa.SA_POTM4), 0, 0, 0) == 2
+    assert call(ok, 2, 0, 0) == 1 and call(ok, 0, 4, 0) == 1 and call(ok, 0, 0, -1) == 1
+    assert call(ok, 0, 0, 0, 8) == 4
+
+
+def test_static_scratch_holds_the_headline_shape_at_any_length():
+    """sa_decode_attention_static documents that batch 1, 32 query heads, head_dim 64 fits its fixed scratch at any
+    cache length, for every code it accepts: the split count is capped, so the workspace is bounded."""
+    for code, nib in [(sa.SA_POT4, False), (sa.SA_POT4, True), (sa.SA_POTM1, False), (sa.SA_POTM1, True), (sa.SA_POTM2, False),
+                      (sa.SA_POTM4, False), (sa.SA_INT8, False)]:
+        cfg = sa.make_config(64, 32, 4, code, nibble=nib)
+        for pages in (1, 2, 7, 64, 512, 513, 4096, 1 << 16, 1 << 20):
+            assert sa.workspace_bytes(cfg, 1, pages) <= sa.STATIC_SCRATCH_BYTES, (code, nib, pages)
+
+
 def test_shiftav_entry_validates_on_the_host():
     """The shift-based A.V option: workspace = partials + rounded logits + per-split statistics; the
     constants N and k_max, the code and the workspace are checked before anything is launched."""

@@ -28,10 +28,11 @@ def t16(x, dev):
     return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev)
 
 
-def cfg_of(case, *, code=None, F=0, shift_by_multiply=False):
+def cfg_of(case, *, code=None, F=0, shift_by_multiply=False, add_on_alu=False):
     code = case.code_k if code is None else code
     return sa.make_config(case.head_dim, case.n_q_heads, case.n_kv_heads, code, nibble=case.nibble,
-                          headroom_F=F, hadamard=case.hadamard, shift_by_multiply=shift_by_multiply)
+                          headroom_F=F, hadamard=case.hadamard, shift_by_multiply=shift_by_multiply,
+                          add_on_alu=add_on_alu)
 
 
 def build_cache(case, dev, *, cfg=None, permute_seed=None, extra_tokens=0):
@@ -43,9 +44,9 @@ def build_cache(case, dev, *, cfg=None, permute_seed=None, extra_tokens=0):
     return cfg, cache
 
 
-def run_decode(case, dev, *, F=0, want_scores=True, permute_seed=None, shift_by_multiply=False):
+def run_decode(case, dev, *, F=0, want_scores=True, permute_seed=None, shift_by_multiply=False, add_on_alu=False):
     import torch
-    cfg = cfg_of(case, F=F, shift_by_multiply=shift_by_multiply)
+    cfg = cfg_of(case, F=F, shift_by_multiply=shift_by_multiply, add_on_alu=add_on_alu)
     cfg, cache = build_cache(case, dev, cfg=cfg, permute_seed=permute_seed)
     O = torch.full((case.batch, case.n_q_heads, case.head_dim), float("nan"), dtype=torch.float32, device=dev)
     dbg = None
@@ -670,3 +671,58 @@ def test_shift_by_multiply_step_matches_the_shift_kernel_bitwise(dev):
     assert np.array_equal(outs[0][0].view(np.uint32), outs[1][0].view(np.uint32))
     assert np.array_equal(outs[0][1], outs[1][1])
     check_against_oracle(case, outs[1][0], None)
+
+
+# ------------------------------------------- sign flips and adds on the ALU pipe only (non-default option)
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 32, 4), (128, 8, 2), (64, 6, 2)])
+@pytest.mark.parametrize("k,nibble", [(0, False), (0, True), (1, True), (2, False), (4, False)])
+def test_add_on_alu_gives_the_same_scores(dev, d, Hq, Hkv, k, nibble):
+    """SA_FLAG_ADD_ON_ALU (no multiply-add anywhere in the score datapath): INT32 scores bit-exact against the
+    oracle, outputs within the tolerance; ragged batch with an empty sequence, head-room above the default."""
+    F = 6 + k + (2 if d == 64 else 0)
+    case = synth.make_case("addalu", [700, 0, 33, 129], Hq, Hkv, d, k, outliers=True, seed=4900 + 10 * k + d, nibble=nibble)
+    O, dbg, _ = run_decode(case, dev, F=F, permute_seed=11, add_on_alu=True)
+    check_against_oracle(case, O, dbg, F=F)
+
+
+def test_add_on_alu_excludes_shift_by_multiply(dev):
+    case = synth.make_case("addalu2", [64], 32, 4, 64, 4, seed=1)
+    cfg = cfg_of(case, shift_by_multiply=True, add_on_alu=True)
+    with pytest.raises(sa.SaError):
+        sa.get_layout(cfg)
+
+
+# ------------------------------------------------------------------ a staged copy that never arrives
+@pytest.mark.parametrize("lost", [(1, 2, 3), (0, 0, 0), (2, 3, 9)])
+def test_lost_copy_marks_exactly_its_rows_and_returns(dev, lost):
+    """The bounded wait of the staged copies, made to run out: the copy of one tile of one (sequence, KV head) is
+    never issued (test hook, 2^10 polls).  The call returns, the rows of that KV head's query heads in that
+    sequence are NaN, every other row is the ordinary result, and an ordinary call afterwards is unaffected."""
+    import torch
+    b, kvh, tile = lost
+    case = synth.make_case("lost", [300, 513, 777], 32, 4, 64, 4, outliers=True, seed=5100)
+    cfg, cache = build_cache(case, dev, permute_seed=3)
+    Q = t16(case.Q, dev)
+    O = torch.zeros((case.batch, 32, 64), dtype=torch.float32, device=dev)
+    sa.debug_decode_lost_copy(cfg, cache.handle, Q, O, cache.workspace, b, kvh, tile)
+    torch.cuda.synchronize()                                # the call comes back: nothing waits without a bound
+    got = O.cpu().numpy()
+    ref = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, 4, 10, n_threads=8)["O"]
+    hit = np.zeros((case.batch, 32), dtype=bool)
+    hit[b, kvh * 8:(kvh + 1) * 8] = True
+    assert np.isnan(got[hit]).all(), "the rows of the lost tile must be marked"
+    assert np.isfinite(got[~hit]).all()
+    assert np.max(np.abs(got[~hit] - ref[~hit])) <= TOL_O
+    O2 = torch.zeros_like(O)
+    sa.decode_attention(cfg, cache.handle, Q, O2, cache.workspace, None)
+    torch.cuda.synchronize()
+    assert np.max(np.abs(O2.cpu().numpy() - ref)) <= TOL_O
+
+
+def test_lost_copy_hook_refuses_other_shapes(dev):
+    import torch
+    case = synth.make_case("lost2", [100], 32, 4, 64, 1, seed=5101)
+    cfg, cache = build_cache(case, dev)
+    O = torch.zeros((1, 32, 64), dtype=torch.float32, device=dev)
+    with pytest.raises(sa.SaError):
+        sa.debug_decode_lost_copy(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, 0, 0, 0)

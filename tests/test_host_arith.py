@@ -115,3 +115,8 @@ def test_score_datapaths_equal_oracle_scores(hh, k, d):
             hh.hh_score8_mul(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
                              C.c_int(path), out.ctypes.data_as(C.c_void_p))
             assert np.array_equal(out.astype(np.int64), want[:, 0]), ("shift by multiply", path, trial, out, want[:, 0])
+        # the non-default kernels without any multiply-add (sign flip and add as logic and add instructions)
+        for path in ((0, 1) if k in (0, 1, 2) else (0,)):
+            hh.hh_score8_alu(C.c_int(k), codes.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), C.c_int(d),
+                             C.c_int(path), out.ctypes.data_as(C.c_void_p))
+            assert np.array_equal(out.astype(np.int64), want[:, 0]), ("adds on the ALU pipe", path, trial, out, want[:, 0])
