@@ -33,6 +33,31 @@ struct DecodeArgs {
     int lost_b, lost_kvh, lost_tile;
 };
 
+// Ragged batches: the grid's sequence coordinate is taken as a RANK by cached length, longest first, so that the
+// blocks of the long sequences are dispatched first and the launch ends on the short ones instead of on whichever
+// long sequence happens to come last in the batch.  Every block of the grid must read the same lengths, so this
+// runs after the wait on the preceding kernels; ties go to the lower index (the map is a fixed function of the
+// lengths).  One thread per sequence counts the sequences that precede its own: batches up to kRankedBatchMax.
+constexpr int kRankedBatchMax = 128;
+SA_D bool batch_is_ranked(int batch) { return batch > 1 && batch <= kRankedBatchMax; }
+SA_D int sequence_of_rank(const int32_t* seq_lens, int batch, int rank, int* scratch /* shared, batch + 1 ints */) {
+    for (int i = threadIdx.x; i < batch; i += blockDim.x) scratch[i] = seq_lens[i];
+    __syncthreads();
+    for (int i = threadIdx.x; i < batch; i += blockDim.x) {
+        const int li = scratch[i];
+        int before = 0;
+        for (int j = 0; j < batch; ++j) {
+            const int lj = scratch[j];
+            before += (lj > li || (lj == li && j < i)) ? 1 : 0;
+        }
+        if (before == rank) scratch[batch] = i;
+    }
+    __syncthreads();
+    const int b = scratch[batch];
+    __syncthreads();                                          // the scratch is about to be used for something else
+    return b;
+}
+
 // red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace
 // (used by the kernels whose warps write their states to shared memory themselves).
 template <int D, int GT, int NW = 4>

@@ -67,7 +67,12 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     const int chunks = a.G / GT;
     const int kvh = blockIdx.y / chunks;
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;
-    const int b = blockIdx.z;
+    const bool ranked = batch_is_ranked(a.batch);             // ragged batches: longest sequence first (see the quantised kernel)
+    int b = blockIdx.z;
+    if (ranked) {
+        pdl_wait();
+        b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
+    }
     const int split = blockIdx.x;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
