@@ -842,8 +842,8 @@ def oracle_rate(lens, Hq, Hkv, d, code, hadamard, outliers, token_cap=1 << 17):
         v1, _ = smp.time_layers(reps, 1)
         vm, _ = smp.time_layers(reps, threads)
         _ORACLE_CACHE[key] = {"oracle_keys_per_s_1thread": v1, "oracle_keys_per_s_threads": vm, "oracle_threads": threads,
-                              "oracle_sample_tokens": tot, "oracle_extrapolated": tot < sum(lens)}
-    return _ORACLE_CACHE[key]
+                              "oracle_sample_tokens": tot}
+    return dict(_ORACLE_CACHE[key], oracle_extrapolated=tot < sum(lens))
 
 
 def run_sweep(args):

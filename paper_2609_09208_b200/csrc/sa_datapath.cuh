@@ -116,7 +116,17 @@ SA_HD uint32_t mad_fma(uint32_t a, uint32_t w, uint32_t c) {
 
 // c + x with the sign flip of x chosen by the mask s (0: +x, 0xffffffff: -x) done as exclusive-or and
 // subtract: logic and add instructions only, no multiplier.
-SA_HD uint32_t flip_add(uint32_t x, uint32_t s, uint32_t c) { return c + ((x ^ s) - s); }
+SA_HD uint32_t flip_add(uint32_t x, uint32_t s, uint32_t c) {
+#ifdef __CUDA_ARCH__
+    // one opaque unit, like the multiply-add it stands in for (left as plain C the three operations of the many
+    // independent updates are interleaved so freely that the kernel spills)
+    uint32_t d;
+    asm("{\n\t.reg .b32 t;\n\txor.b32 t, %1, %2;\n\tsub.s32 t, t, %2;\n\tadd.s32 %0, t, %3;\n\t}" : "=r"(d) : "r"(x), "r"(s), "r"(c));
+    return d;
+#else
+    return c + ((x ^ s) - s);
+#endif
+}
 
 SA_HD uint32_t pack_pair(int q_lo, int q_hi) { return ((uint32_t)q_hi << 16) + (uint32_t)q_lo; }
 

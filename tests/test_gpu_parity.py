@@ -726,3 +726,28 @@ def test_lost_copy_hook_refuses_other_shapes(dev):
     O = torch.zeros((1, 32, 64), dtype=torch.float32, device=dev)
     with pytest.raises(sa.SaError):
         sa.debug_decode_lost_copy(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, 0, 0, 0)
+
+
+# ------------------------------------------------------------------ ragged batches: longest sequence first
+@pytest.mark.parametrize("batch", [2, 17, 128, 129])
+def test_length_ranked_batches_cover_every_sequence_once(dev, batch):
+    """Batches up to 128 sequences are dispatched by rank of their cached length (ties by index), larger ones in
+    index order: either way every sequence must come out exactly as the oracle's, whatever the mix of equal, empty
+    and distinct lengths; and twice in a row bit for bit (the rank is a fixed function of the lengths)."""
+    import torch
+    rng = np.random.default_rng(6000 + batch)
+    lens = rng.integers(0, 200, size=batch)
+    lens[rng.integers(0, batch, size=max(1, batch // 4))] = 97          # ties
+    lens[0] = 0
+    lens[-1] = 199
+    case = synth.make_case("ranked", lens, 8, 2, 64, 4, outliers=True, seed=6100 + batch)
+    cfg, cache = build_cache(case, dev, permute_seed=5)
+    outs = []
+    for _ in range(2):
+        O = torch.full((case.batch, 8, 64), float("nan"), dtype=torch.float32, device=dev)
+        dbg = torch.full((case.batch, 8, cache.max_pages * 64), -7, dtype=torch.int32, device=dev)
+        sa.decode_attention(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, dbg)
+        torch.cuda.synchronize()
+        outs.append(O.cpu().numpy())
+    check_against_oracle(case, outs[0], dbg.cpu().numpy())
+    assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
