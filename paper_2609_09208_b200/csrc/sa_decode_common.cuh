@@ -154,16 +154,18 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
 // dims times 32 groups of splits; a thread's loads (three splits at a time) are all in flight
 // together, so up to 96 splits cost one round trip to L2.  Each thread merges its splits with a local
 // maximum, the block takes the maximum M* of those, every thread rescales its sum by the exact
-// 2^(M_local - M*), and the groups are added in a fixed order (deterministic).  The block is kept this
+// 2^(M_local - M*), and the groups are added in a fixed order, in two levels (deterministic).  The block is kept this
 // small — 128 threads, at most 32 registers, 2.7 KB of shared memory — so that it fits on an SM beside
 // two resident blocks of the decode kernel: the next decode kernel is launched while this one runs
 // (programmatic dependent launch), and a merge block that took the place of one of its blocks would make
 // that block, and with it the whole grid, finish late.
-constexpr int kMergeThreads = 128;
+// With more than 96 splits (the FP16 kernel at batch 1: 111) the block has 256 threads = 64 groups instead, so that
+// the partials are still fetched in one round trip; it then no longer fits beside the quantised kernels' two blocks,
+// whose split counts stay below that.
 constexpr int kMergeDims = 16;                                // output dims per block
 constexpr int kMergeLanes = kMergeDims / 4;                   // float4 lanes
-constexpr int kMergeGroups = kMergeThreads / kMergeLanes;     // groups of splits
 constexpr int kMergeChunk = 3;                                // splits per thread whose loads are in flight together
+constexpr int kMergeSmallSplits = (128 / kMergeLanes) * kMergeChunk;   // most splits a 128-thread block takes in one pass
 
 // A sequence's length grows by one when the decode kernel appended the step's token itself (the token's
 // page must be mapped, exactly the condition the decode kernel used).
@@ -173,10 +175,11 @@ struct BumpArgs {
     int max_pages, n_pages, Hq;
 };
 
-template <int D>
-__global__ void __launch_bounds__(kMergeThreads, 16) merge_kernel(const float* __restrict__ partials,
-                                                                  float* __restrict__ O, int n_splits, int n_rows,
-                                                                  BumpArgs bump) {
+template <int D, int kMergeThreads>
+__global__ void __launch_bounds__(kMergeThreads, 2048 / kMergeThreads) merge_kernel(const float* __restrict__ partials,
+                                                                                    float* __restrict__ O, int n_splits,
+                                                                                    int n_rows, BumpArgs bump) {
+    constexpr int kMergeGroups = kMergeThreads / kMergeLanes;     // groups of splits
     __shared__ int mw_s[kMergeThreads / 32];
     __shared__ float4 o_s[kMergeGroups][kMergeLanes];
     __shared__ float l_s[kMergeGroups];
@@ -238,12 +241,33 @@ __global__ void __launch_bounds__(kMergeThreads, 16) merge_kernel(const float* _
     o_s[grp][ln] = make_float4(o.x * f, o.y * f, o.z * f, o.w * f);
     if (ln == 0) l_s[grp] = l * f;
     __syncthreads();
+    // the groups are added in a fixed order, in two levels (eight groups per thread, then the eighths): the result
+    // does not depend on the timing of anything
+    constexpr int kFan = 8;
+    if (grp < kMergeGroups / kFan) {
+        o = o_s[grp * kFan][ln];
+        l = l_s[grp * kFan];
+#pragma unroll
+        for (int g = 1; g < kFan; ++g) {
+            const float4 t = o_s[grp * kFan + g][ln];
+            o.x += t.x;
+            o.y += t.y;
+            o.z += t.z;
+            o.w += t.w;
+            l += l_s[grp * kFan + g];
+        }
+    }
+    __syncthreads();                                          // every first-level read is done: the rows can be overwritten
+    if (grp < kMergeGroups / kFan) {
+        o_s[grp][ln] = o;
+        if (ln == 0) l_s[grp] = l;
+    }
+    __syncthreads();
     if (grp == 0) {
-        // the groups are added in a fixed order: the result does not depend on the timing of anything
         o = o_s[0][ln];
         l = l_s[0];
-#pragma unroll 8
-        for (int g = 1; g < kMergeGroups; ++g) {
+#pragma unroll
+        for (int g = 1; g < kMergeGroups / kFan; ++g) {
             const float4 t = o_s[g][ln];
             o.x += t.x;
             o.y += t.y;
@@ -314,10 +338,13 @@ inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s
     const int rows = a.batch * a.Hq;
     BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq};
     cudaError_t err;
-    if (p.d == 64) err = launch_pdl(merge_kernel<64>, dim3(rows * (64 / kMergeDims)), dim3(kMergeThreads), 0, s,
-                                    (const float*)a.partials, a.O, a.n_splits, rows, bump);
-    else err = launch_pdl(merge_kernel<128>, dim3(rows * (128 / kMergeDims)), dim3(kMergeThreads), 0, s,
-                          (const float*)a.partials, a.O, a.n_splits, rows, bump);
+    const bool small = a.n_splits <= kMergeSmallSplits;
+    const dim3 grid(rows * (p.d / kMergeDims));
+    const float* part = a.partials;
+    if (p.d == 64) err = small ? launch_pdl(merge_kernel<64, 128>, grid, dim3(128), 0, s, part, a.O, a.n_splits, rows, bump)
+                               : launch_pdl(merge_kernel<64, 256>, grid, dim3(256), 0, s, part, a.O, a.n_splits, rows, bump);
+    else err = small ? launch_pdl(merge_kernel<128, 128>, grid, dim3(128), 0, s, part, a.O, a.n_splits, rows, bump)
+                     : launch_pdl(merge_kernel<128, 256>, grid, dim3(256), 0, s, part, a.O, a.n_splits, rows, bump);
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SA_OK : SA_ERR_CUDA;
 }
 
