@@ -751,3 +751,24 @@ def test_length_ranked_batches_cover_every_sequence_once(dev, batch):
         outs.append(O.cpu().numpy())
     check_against_oracle(case, outs[0], dbg.cpu().numpy())
     assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
+
+
+# ------------------------------------------------------------------ split-K merge: every block shape and pass count
+@pytest.mark.parametrize("code,Hq,Hkv,T", [(4, 8, 1, 20000), (1, 8, 1, 20000), (0, 32, 4, 3000)])
+def test_split_merge_with_many_splits(dev, code, Hq, Hkv, T):
+    """A single KV head spreads one sequence over up to 295 splits: the merge then runs with its 256-thread blocks
+    and (above 192 splits) takes the partials in two passes; 32/4 heads at a short length stay below 96 splits
+    (128-thread blocks).  Outputs against the oracle, and identical twice in a row."""
+    import torch
+    case = synth.make_case("merge", [T], Hq, Hkv, 64, code, outliers=True, seed=7000 + code)
+    cfg, cache = build_cache(case, dev, permute_seed=9)
+    n_splits = sa.workspace_bytes(cfg, 1, cache.max_pages) // (Hq * 66 * 4)
+    assert (n_splits > 192) == (code == 1) and (n_splits <= 96) == (code == 0)
+    outs = []
+    for _ in range(2):
+        O = torch.full((1, Hq, 64), float("nan"), dtype=torch.float32, device=dev)
+        sa.decode_attention(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, None)
+        torch.cuda.synchronize()
+        outs.append(O.cpu().numpy())
+    check_against_oracle(case, outs[0], None)
+    assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
