@@ -198,7 +198,10 @@ sa_status sa_fill_kv(const sa_config* cfg, const sa_cache* cache, const uint16_t
  * The kernels are launched with programmatic stream serialisation; the decode kernel reads Q
  * (and nothing else) before it waits for the preceding kernel in the stream, so Q must not be
  * written by a kernel that signals programmatic launch completion before it has written Q
- * (ordinary launches, copies and every kernel of this library satisfy that). */
+ * (ordinary launches, copies and every kernel of this library satisfy that).  The split-K merge that ends
+ * the call may release its dependents before it has written O: a following kernel that the CALLER launches
+ * with the programmatic-serialisation attribute must execute its own grid-dependency wait before it reads O
+ * or seq_lens (as that attribute always requires); ordinary launches and copies are ordered as usual. */
 sa_status sa_decode_attention(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                               float* O, void* workspace, size_t workspace_bytes,
                               int32_t* dbg_scores, sa_stream stream);

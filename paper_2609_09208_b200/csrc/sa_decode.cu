@@ -69,6 +69,14 @@ extern "C" sa_status sa_debug_decode_lost_copy(const sa_config* cfg, const sa_ca
 extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q,
                                     const uint16_t* K_new, const uint16_t* V_new, float* O, void* workspace,
                                     size_t workspace_bytes, sa_stream stream) {
+    return sa::decode_step_impl(cfg, cache, Q, K_new, V_new, O, workspace, workspace_bytes, stream, false);
+}
+
+// sa_decode_step; with q_after_wait the decode kernel reads Q only after its wait on the preceding kernel (the
+// host-buffer entry, whose staging kernel writes Q and releases its dependents early).
+sa_status sa::decode_step_impl(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q, const uint16_t* K_new,
+                               const uint16_t* V_new, float* O, void* workspace, size_t workspace_bytes,
+                               sa_stream stream, bool q_after_wait) {
     Plan p;
     sa_status st = make_plan(cfg, &p);
     if (st != SA_OK) return st;
@@ -94,6 +102,7 @@ extern "C" sa_status sa_decode_step(const sa_config* cfg, const sa_cache* cache,
     if (st != SA_OK) return st;
     a.Knew = K_new;
     a.Vnew = V_new;
+    a.wait_first = q_after_wait ? 1 : 0;
     a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / (double)(1LL << p.F));
     if (p.int8) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d) / 127.0);
     if (p.fp16) a.zscale = (float)(1.4426950408889634 / sqrt((double)p.d));

@@ -31,6 +31,9 @@ struct DecodeArgs {
     const uint16_t* Vnew;
     // Test hook (sa_debug_decode_lost_copy): the copy of this tile of this (sequence, KV head) is never issued.
     int lost_b, lost_kvh, lost_tile;
+    // The block waits for the preceding kernels before it reads anything, Q included (set when the kernel before
+    // this one writes Q and releases its dependents early: the host-buffer entry's staging kernel).
+    int wait_first;
 };
 
 // Ragged batches: the grid's sequence coordinate is taken as a RANK by cached length, longest first, so that the
@@ -173,6 +176,7 @@ struct BumpArgs {
     int32_t* seq_lens;        // null: no fused append
     const int32_t* page_table;
     int max_pages, n_pages, Hq;
+    int early_release;        // release the dependents of the merge kernel before its own wait (see merge_kernel)
 };
 
 template <int D, int kMergeThreads>
@@ -183,8 +187,15 @@ __global__ void __launch_bounds__(kMergeThreads, 2048 / kMergeThreads) merge_ker
     __shared__ int mw_s[kMergeThreads / 32];
     __shared__ float4 o_s[kMergeGroups][kMergeLanes];
     __shared__ float l_s[kMergeGroups];
+    // With early_release the kernel after this one may be scheduled at once — while the decode kernel whose
+    // partials this block is about to wait for is still running — so that its blocks move in as that kernel's
+    // blocks retire and are already waiting when this one completes.  That is safe because every kernel of this
+    // library reads, ahead of its own wait, nothing that this kernel or its predecessors write (the decode kernels:
+    // only Q and hints).  It pays for the ten-warp decode kernels at batch 1 (3–6 % of a step); with the four-warp
+    // kernels (PoT-M1 / M2, d = 128, FP16) the early arrivals slow the running kernel down by more than they gain.
+    if (bump.early_release) pdl_launch_dependents();
     pdl_wait();                                               // the partials come from the kernel before
-    pdl_launch_dependents();
+    if (!bump.early_release) pdl_launch_dependents();
     const int row = blockIdx.x / (D / kMergeDims);            // b * Hq + h
     const int part = blockIdx.x % (D / kMergeDims);           // which 16 dims
     if (bump.seq_lens && threadIdx.x == 0 && part == 0 && row % bump.Hq == 0) {
@@ -283,6 +294,10 @@ __global__ void __launch_bounds__(kMergeThreads, 2048 / kMergeThreads) merge_ker
     }
 }
 
+sa_status decode_step_impl(const sa_config* cfg, const sa_cache* cache, const uint16_t* Q, const uint16_t* K_new,
+                           const uint16_t* V_new, float* O, void* workspace, size_t workspace_bytes, sa_stream stream,
+                           bool q_after_wait);
+
 inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16_t* Q, float* O,
                                   void* workspace, size_t workspace_bytes, DecodeArgs* a, int* gt) {
     if (!c || !c->pages || !c->page_table || !c->seq_lens || !Q || !O) return SA_ERR_INVALID_ARG;
@@ -330,13 +345,15 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->Knew = nullptr;
     a->Vnew = nullptr;
     a->lost_b = a->lost_kvh = a->lost_tile = -1;
+    a->wait_first = 0;
     *gt = GT;
     return SA_OK;
 }
 
 inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s) {
     const int rows = a.batch * a.Hq;
-    BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq};
+    const int early = (!p.fp16 && decode_shape(p.d, p.int8 ? 8 : p.k).warps >= 8) ? 1 : 0;
+    BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq, early};
     cudaError_t err;
     const bool small = a.n_splits <= kMergeSmallSplits;
     const dim3 grid(rows * (p.d / kMergeDims));

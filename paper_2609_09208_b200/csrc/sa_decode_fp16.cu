@@ -69,10 +69,8 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;
     const bool ranked = batch_is_ranked(a.batch);             // ragged batches: longest sequence first (see the quantised kernel)
     int b = blockIdx.z;
-    if (ranked) {
-        pdl_wait();
-        b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
-    }
+    if (ranked || a.wait_first) pdl_wait();
+    if (ranked) b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
     const int split = blockIdx.x;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
@@ -103,19 +101,24 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
 
     // While the preceding kernel drains: ask L2 for this warp's first tile, guessed from a length that kernel
     // may be about to change (loads that bypass L1; a hint only).
+    int tile_g = -1, pidx_g = -1;
     if (lane == 0) {
         const int len_g = __ldcg(a.seq_lens + b) + (a.Knew ? 1 : 0);
         const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
-        const int tile_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
-        if (tile_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
-            const int pidx_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (tile_g >> 1));
-            if (pidx_g >= 0 && pidx_g < a.n_pages)
-                Stage::prefetch(a.pages + ((size_t)pidx_g * a.Hkv + kvh) * a.page_bytes, (tile_g & 1) * 32);
+        const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
+        if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
+            tile_g = t_g;
+            const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
+            if (p_g >= 0 && p_g < a.n_pages)
+                Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32);
         }
     }
     pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
 
     int len = a.seq_lens[b];
+    // the page of the guessed first tile, read again now that it is valid, together with the length (one round trip
+    // instead of two when the guess holds)
+    if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
     int tile_new = -1, pidx_new = -1;
     if (a.Knew) {
         // fused append (see the quantised kernel): the step's new token goes to position len if its page is mapped
@@ -144,7 +147,7 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     }
     auto issue = [&](int i) {
         const int tile = first + 4 * i;
-        const int pidx = a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
+        const int pidx = (tile == tile_g) ? pidx_g : a.page_table[(size_t)b * a.max_pages + (tile >> 1)];
         const int s = i % kStages;
         if (pidx < 0 || pidx >= a.n_pages) {
             mbar_arrive(mbar0 + s * 8);

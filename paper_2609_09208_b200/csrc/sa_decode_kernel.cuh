@@ -101,10 +101,8 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     // in that case the block waits for the preceding kernels right here, before the lengths are read.
     const bool ranked = batch_is_ranked(a.batch);
     int b = blockIdx.z;
-    if (ranked) {
-        pdl_wait();
-        b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
-    }
+    if (ranked || a.wait_first) pdl_wait();
+    if (ranked) b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
     const int split = blockIdx.x;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * NS * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * NS * Stage::kBytes;

@@ -157,9 +157,11 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
 __global__ void __launch_bounds__(256) stage_in_kernel(const uint4* __restrict__ q, const uint4* __restrict__ k,
                                                        const uint4* __restrict__ v, uint4* __restrict__ dq,
                                                        uint4* __restrict__ dk, uint4* __restrict__ dv, int nq, int nkv) {
-    // The staging buffer may still be read by the step before.  No early launch_dependents here: the decode
-    // kernel reads Q ahead of its own wait, so it must not start before this kernel has completed.
+    // The staging buffer may still be read by the step before.  The kernel after this one — the decode kernel in its
+    // wait-first form, or the append kernel, which waits before anything else — may be scheduled at once: neither
+    // reads the staging buffer before its own wait.
     pdl_wait();
+    pdl_launch_dependents();
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i < nq) dq[i] = q[i];
     else if (i < nq + nkv) dk[i - nq] = k[i - nq];
@@ -272,7 +274,7 @@ sa_status sa_decode_step_host(const sa_config* cfg, const sa_cache* cache, const
         if (launch_pdl(stage_in_kernel, dim3(blocks), dim3(256), 0, s, (const uint4*)mq, (const uint4*)mk, (const uint4*)mv,
                        (uint4*)dQ, (uint4*)dK, (uint4*)dV, nq, nkv) != cudaSuccess || cudaGetLastError() != cudaSuccess)
             return SA_ERR_CUDA;
-        return sa_decode_step(cfg, cache, dQ, dK, dV, static_cast<float*>(mo), workspace, workspace_bytes, stream);
+        return decode_step_impl(cfg, cache, dQ, dK, dV, static_cast<float*>(mo), workspace, workspace_bytes, stream, true);
     }
     const char* hq = reinterpret_cast<const char*>(Q_host);
     if (up(q) == q && up(kv) == kv && reinterpret_cast<const char*>(K_new_host) == hq + q &&

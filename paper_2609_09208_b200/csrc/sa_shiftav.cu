@@ -9,7 +9,7 @@
 // Both M and g_ref are those of the whole sequence, so the option runs as two passes over the
 // key axis instead of one streaming pass with running values (whose truncations would depend on
 // the order of the tiles):
-//   pass 1  the decode kernel's score phase (sa_decode.cu, DecodeArgs::zr != null): integer
+//   pass 1  the decode kernel's score phase (sa_decode_kernel.cuh, DecodeArgs::zr != null): integer
 //           scores, rounded logits to memory, per block the ceiling of its largest logit and its
 //           smallest value exponent;
 //   pass 2  shiftav_kernel below: reduces those statistics to M and g_ref, then per 32-key tile
@@ -229,7 +229,7 @@ static void launch_shiftav_gt(const DecodeArgs& a, int GT, dim3 grid, cudaStream
     }
 }
 
-// defined in sa_decode.cu: the decode kernel for these arguments (score pass when a.zr is set)
+// defined in sa_decode.cu: launches the decode kernel for these arguments (score pass when a.zr is set)
 void launch_decode_main(const Plan& p, const DecodeArgs& a, int GT, cudaStream_t s);
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
