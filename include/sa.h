@@ -339,7 +339,10 @@ sa_status sa_debug_unpack(const sa_config* cfg, const sa_cache* cache, int b, in
  * Everything is asynchronous on `stream`; synchronise it before reading O_host.
  * If all four host buffers are pinned and device-addressable (cudaHostAlloc / cudaHostRegister
  * memory under unified addressing), no copy engine is used: a small kernel fetches the inputs
- * and the merge kernel stores O directly into host memory.  Otherwise the buffers are copied
+ * and the merge kernel stores O directly into host memory.  That kernel reads the three input buffers
+ * without waiting for kernels enqueued earlier on `stream` (they are host inputs): their contents must
+ * be in place when the call is enqueued (or the graph holding it is launched), written by the host or by
+ * work that has completed, not produced by a kernel still pending on the same stream.  Otherwise the buffers are copied
  * with cudaMemcpyAsync (a single copy for the inputs if Q_host, K_new_host and V_new_host follow
  * one another in one host buffer and their sizes are multiples of 256 bytes).
  * `staging` is device scratch of at least sa_staging_bytes(); not shared between overlapping calls. */

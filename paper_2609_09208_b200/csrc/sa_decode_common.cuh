@@ -38,13 +38,16 @@ struct DecodeArgs {
 
 // Ragged batches: the grid's sequence coordinate is taken as a RANK by cached length, longest first, so that the
 // blocks of the long sequences are dispatched first and the launch ends on the short ones instead of on whichever
-// long sequence happens to come last in the batch.  Every block of the grid must read the same lengths, so this
-// runs after the wait on the preceding kernels; ties go to the lower index (the map is a fixed function of the
-// lengths).  One thread per sequence counts the sequences that precede its own: batches up to kRankedBatchMax.
+// long sequence happens to come last in the batch.  Every block of the grid must map ranks from the same lengths, so
+// the map that counts is taken after the wait on the preceding kernels (a call before that wait is a guess); ties
+// go to the lower index (the map is a fixed function of the lengths).  The lengths are read past L1, so that a
+// guess leaves nothing stale behind.  One thread per sequence counts the sequences that precede its own: batches
+// up to kRankedBatchMax.
 constexpr int kRankedBatchMax = 128;
 SA_D bool batch_is_ranked(int batch) { return batch > 1 && batch <= kRankedBatchMax; }
-SA_D int sequence_of_rank(const int32_t* seq_lens, int batch, int rank, int* scratch /* shared, batch + 1 ints */) {
-    for (int i = threadIdx.x; i < batch; i += blockDim.x) scratch[i] = seq_lens[i];
+SA_D int sequence_of_rank(const int32_t* seq_lens, int batch, int rank, int* scratch /* shared, batch + 1 ints */,
+                          int* len_out = nullptr /* that sequence's length, as read here */) {
+    for (int i = threadIdx.x; i < batch; i += blockDim.x) scratch[i] = __ldcg(seq_lens + i);
     __syncthreads();
     for (int i = threadIdx.x; i < batch; i += blockDim.x) {
         const int li = scratch[i];
@@ -57,6 +60,7 @@ SA_D int sequence_of_rank(const int32_t* seq_lens, int batch, int rank, int* scr
     }
     __syncthreads();
     const int b = scratch[batch];
+    if (len_out) *len_out = scratch[b];
     __syncthreads();                                          // the scratch is about to be used for something else
     return b;
 }

@@ -67,10 +67,12 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     const int chunks = a.G / GT;
     const int kvh = blockIdx.y / chunks;
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;
-    const bool ranked = batch_is_ranked(a.batch);             // ragged batches: longest sequence first (see the quantised kernel)
-    int b = blockIdx.z;
-    if (ranked || a.wait_first) pdl_wait();
-    if (ranked) b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
+    // ragged batches: longest sequence first, the rank guessed ahead of the dependency wait and settled after it
+    // (see the quantised kernel)
+    const bool ranked = batch_is_ranked(a.batch);
+    int b = blockIdx.z, len_ranked = 0;
+    if (a.wait_first) pdl_wait();
+    if (ranked) b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff), &len_ranked);
     const int split = blockIdx.x;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
@@ -89,36 +91,48 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     // Q fragments (A operand, rows = query heads; rows >= GT are zero): for 16-dim block kb the lane
     // holds dims 16kb + 2*quad + {0,1} and + 8 of query `row`.
     uint32_t qa[KB16][2];
+    int tile_g, pidx_g;
+    bool again;
+#pragma unroll 1
+    do {
 #pragma unroll
-    for (int kb = 0; kb < KB16; ++kb) {
-        qa[kb][0] = qa[kb][1] = 0u;
-        if (row < GT) {
-            const uint32_t* q32 = reinterpret_cast<const uint32_t*>(a.Q + ((size_t)b * a.Hq + h0 + row) * D);
-            qa[kb][0] = __ldg(q32 + kb * 8 + quad);
-            qa[kb][1] = __ldg(q32 + kb * 8 + 4 + quad);
+        for (int kb = 0; kb < KB16; ++kb) {
+            qa[kb][0] = qa[kb][1] = 0u;
+            if (row < GT) {
+                const uint32_t* q32 = reinterpret_cast<const uint32_t*>(a.Q + ((size_t)b * a.Hq + h0 + row) * D);
+                qa[kb][0] = __ldg(q32 + kb * 8 + quad);
+                qa[kb][1] = __ldg(q32 + kb * 8 + 4 + quad);
+            }
         }
-    }
 
-    // While the preceding kernel drains: ask L2 for this warp's first tile, guessed from a length that kernel
-    // may be about to change (loads that bypass L1; a hint only).
-    int tile_g = -1, pidx_g = -1;
-    if (lane == 0) {
-        const int len_g = __ldcg(a.seq_lens + b) + (a.Knew ? 1 : 0);
-        const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
-        const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
-        if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
-            tile_g = t_g;
-            const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
-            if (p_g >= 0 && p_g < a.n_pages)
-                Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32);
+        // While the preceding kernel drains: ask L2 for this warp's first tile, guessed from a length that kernel
+        // may be about to change (loads that bypass L1; a hint only).
+        tile_g = -1, pidx_g = -1;
+        if (lane == 0) {
+            const int len_g = (ranked ? len_ranked : __ldcg(a.seq_lens + b)) + (a.Knew ? 1 : 0);
+            const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
+            const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
+            if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
+                tile_g = t_g;
+                const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
+                if (p_g >= 0 && p_g < a.n_pages)
+                    Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32);
+            }
         }
-    }
-    pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
+        pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
+        // the page of the guessed first tile, read again now that it is valid, together with the length(s) (one round
+        // trip instead of two when the guess holds)
+        if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
+        again = false;
+        if (ranked && !a.wait_first) {
+            const int b_now = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff),
+                                               &len_ranked);
+            again = b_now != b;
+            b = b_now;
+        }
+    } while (again);
 
-    int len = a.seq_lens[b];
-    // the page of the guessed first tile, read again now that it is valid, together with the length (one round trip
-    // instead of two when the guess holds)
-    if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
+    int len = ranked ? len_ranked : a.seq_lens[b];
     int tile_new = -1, pidx_new = -1;
     if (a.Knew) {
         // fused append (see the quantised kernel): the step's new token goes to position len if its page is mapped

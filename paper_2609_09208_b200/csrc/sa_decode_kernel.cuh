@@ -97,12 +97,18 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     const int chunks = a.G / GT;
     const int kvh = blockIdx.y / chunks;
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;     // first query head of this block
-    // Sequence of this block: grid coordinate z itself, or (ragged batches) the sequence whose length has rank z;
-    // in that case the block waits for the preceding kernels right here, before the lengths are read.
+    // Sequence of this block: grid coordinate z itself, or (ragged batches) the sequence whose length has rank z.
+    // The rank taken here, from lengths the preceding kernel may be about to change, is a guess that lets the
+    // query prologue run ahead of the dependency wait; the rank taken after the wait decides, and the prologue is
+    // repeated in the rare case that the two differ (a step adds one token to every sequence, which keeps the order).
+    // The test-hook instantiation guesses wrong on purpose, so that its tests walk the repeat.
     const bool ranked = batch_is_ranked(a.batch);
     int b = blockIdx.z;
-    if (ranked || a.wait_first) pdl_wait();
-    if (ranked) b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff));
+    if (a.wait_first) pdl_wait();
+    int len_ranked = 0;                                        // the length that came with the rank
+    if (ranked)
+        b = sequence_of_rank(a.seq_lens, a.batch, LOST ? (blockIdx.z + 1) % a.batch : blockIdx.z,
+                             reinterpret_cast<int*>(smem + SM::kStageOff), &len_ranked);
     const int split = blockIdx.x;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * NS * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * NS * Stage::kBytes;
@@ -121,129 +127,142 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     // The length is fetched here, so that its latency hides behind the query quantisation; the dependent
     // page-table reads and the hints themselves are left to the last warp, after the prologue's last barrier,
     // so that no other warp waits for them.
-    int len_g = 0, tile_g = -1, pidx_g = -1;
-    if (lane == 0 || warp == NW - 1) len_g = __ldcg(a.seq_lens + b);
+    int len_g, tile_g, pidx_g;
+    bool again;
+#pragma unroll 1
+    do {
+        len_g = 0, tile_g = -1, pidx_g = -1;
+        if (ranked) len_g = len_ranked;
+        else if (lane == 0 || warp == NW - 1) len_g = __ldcg(a.seq_lens + b);
 
-    // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register.  It reads
-    // only Q, which no kernel of a decode step writes, so it runs BEFORE the wait on the preceding
-    // kernel (the cache append) and overlaps it. ----
-    for (int g = warp; g < GT; g += NW) {
-        uint32_t bits[EPL];
-        load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
-        int q[EPL];
-        const float delta = quantise_query_vec<EPL>(bits, lane, a.hadamard != 0, q);
+        // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register.  It reads
+        // only Q, which no kernel of a decode step writes, so it runs BEFORE the wait on the preceding
+        // kernel (the cache append) and overlaps it. ----
+        for (int g = warp; g < GT; g += NW) {
+            uint32_t bits[EPL];
+            load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
+            int q[EPL];
+            const float delta = quantise_query_vec<EPL>(bits, lane, a.hadamard != 0, q);
 #pragma unroll
-        for (int i = 0; i < EPL; ++i) q_s[lane * EPL + i][g] = q[i];
-        if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
-    }
-    __syncthreads();
-    if (lane == 0) {
-        const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
-        const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
-        if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) tile_g = t_g;
-    }
-    if constexpr (SM::kTable) {
-        // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
-        using TS = TableScore<KB, NP>;
-        uint8_t* tab = smem + SM::kQpOff;
-        // One thread per row (element, query pair) and pass; it walks the row's 2^KB entries by
-        // repeated addition of the pair, starting at an entry that depends on its lane so that the
-        // lanes of a half-warp always write different banks, and wraps around once.
-        constexpr int ROWS = D * NP;
-        constexpr int PASSES = (ROWS + NT - 1) / NT;
-        constexpr uint32_t MASK = (1u << KB) - 1u;
-        int qlo[PASSES], qhi[PASSES];
-#pragma unroll
-        for (int k = 0; k < PASSES; ++k) {
-            const int row = threadIdx.x + k * NT;              // = m * NP + p
-            const int m = row / NP, p = row % NP;
-            qlo[k] = (row < ROWS) ? q_s[m][2 * p] : 0;
-            qhi[k] = (row < ROWS && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
+            for (int i = 0; i < EPL; ++i) q_s[lane * EPL + i][g] = q[i];
+            if (lane == 0) qscale_s[g] = delta * a.zscale;        // Delta * 2^-F * log2(e) / sqrt(d)
         }
-        __syncthreads();                                       // q_s is about to be overwritten
-        const uint32_t mu0 = ((uint32_t)lane >> (4 - KB)) & MASK;
+        __syncthreads();
+        if (lane == 0) {
+            const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
+            const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
+            if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) tile_g = t_g;
+        }
+        if constexpr (SM::kTable) {
+            // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
+            using TS = TableScore<KB, NP>;
+            uint8_t* tab = smem + SM::kQpOff;
+            // One thread per row (element, query pair) and pass; it walks the row's 2^KB entries by
+            // repeated addition of the pair, starting at an entry that depends on its lane so that the
+            // lanes of a half-warp always write different banks, and wraps around once.
+            constexpr int ROWS = D * NP;
+            constexpr int PASSES = (ROWS + NT - 1) / NT;
+            constexpr uint32_t MASK = (1u << KB) - 1u;
+            int qlo[PASSES], qhi[PASSES];
 #pragma unroll
-        for (int k = 0; k < PASSES; ++k) {
-            const int row = threadIdx.x + k * NT;
-            if (row < ROWS) {
-                uint2* dst = reinterpret_cast<uint2*>(tab + (size_t)row * TS::kRowBytes);
-                const uint32_t lo = (uint32_t)qlo[k], hi = (uint32_t)qhi[k];
-                uint32_t x = lo << KB, y = hi << KB;           // entry mu0: (2^KB + mu0) times the pair, by shift-and-add
+            for (int k = 0; k < PASSES; ++k) {
+                const int row = threadIdx.x + k * NT;              // = m * NP + p
+                const int m = row / NP, p = row % NP;
+                qlo[k] = (row < ROWS) ? q_s[m][2 * p] : 0;
+                qhi[k] = (row < ROWS && 2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0;
+            }
+            __syncthreads();                                       // q_s is about to be overwritten
+            const uint32_t mu0 = ((uint32_t)lane >> (4 - KB)) & MASK;
 #pragma unroll
-                for (int bit = 0; bit < KB; ++bit)
-                    if (mu0 & (1u << bit)) { x += lo << bit; y += hi << bit; }
+            for (int k = 0; k < PASSES; ++k) {
+                const int row = threadIdx.x + k * NT;
+                if (row < ROWS) {
+                    uint2* dst = reinterpret_cast<uint2*>(tab + (size_t)row * TS::kRowBytes);
+                    const uint32_t lo = (uint32_t)qlo[k], hi = (uint32_t)qhi[k];
+                    uint32_t x = lo << KB, y = hi << KB;           // entry mu0: (2^KB + mu0) times the pair, by shift-and-add
 #pragma unroll
-                for (uint32_t st = 0; st <= MASK; ++st) {
-                    const uint32_t mu = (mu0 + st) & MASK;
-                    if (mu == 0u) { x = lo << KB; y = hi << KB; }
-                    dst[mu] = make_uint2(x, y);
-                    x += lo;
-                    y += hi;
+                    for (int bit = 0; bit < KB; ++bit)
+                        if (mu0 & (1u << bit)) { x += lo << bit; y += hi << bit; }
+#pragma unroll
+                    for (uint32_t st = 0; st <= MASK; ++st) {
+                        const uint32_t mu = (mu0 + st) & MASK;
+                        if (mu == 0u) { x = lo << KB; y = hi << KB; }
+                        dst[mu] = make_uint2(x, y);
+                        x += lo;
+                        y += hi;
+                    }
                 }
             }
-        }
-    } else if constexpr (KB != 8) {
-        uint32_t qp_reg[(D * NP + NT - 1) / NT];
+        } else if constexpr (KB != 8) {
+            uint32_t qp_reg[(D * NP + NT - 1) / NT];
 #pragma unroll
-        for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
-            const int idx = threadIdx.x + k * NT;
-            const int m = idx / NP, p = idx % NP;
-            qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
-        }
-        __syncthreads();                                       // q_s is about to be overwritten
-        // S[m][g][pair] = the packed pair shifted by g - 1 (0 for g = 0); the entries of one pair are written
-        // starting at a g that depends on the element, so that the lanes of a warp use different banks
-        uint32_t* tab = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
+            for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
+                const int idx = threadIdx.x + k * NT;
+                const int m = idx / NP, p = idx % NP;
+                qp_reg[k] = (idx < D * NP) ? pack_pair(q_s[m][2 * p], (2 * p + 1 < GT) ? q_s[m][2 * p + 1] : 0) : 0u;
+            }
+            __syncthreads();                                       // q_s is about to be overwritten
+            // S[m][g][pair] = the packed pair shifted by g - 1 (0 for g = 0); the entries of one pair are written
+            // starting at a g that depends on the element, so that the lanes of a warp use different banks
+            uint32_t* tab = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
 #pragma unroll
-        for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
-            const int idx = threadIdx.x + k * NT;
-            const int m = idx / NP, p = idx % NP;
-            if (idx < D * NP) {
+            for (int k = 0; k < (D * NP + NT - 1) / NT; ++k) {
+                const int idx = threadIdx.x + k * NT;
+                const int m = idx / NP, p = idx % NP;
+                if (idx < D * NP) {
 #pragma unroll
-                for (int st = 0; st < 8; ++st) {
-                    const int g = (st + m) & 7;
-                    tab[(m * 8 + g) * NP + p] = ShiftTable<NP>::entry(qp_reg[k], g);
+                    for (int st = 0; st < 8; ++st) {
+                        const int g = (st + m) & 7;
+                        tab[(m * 8 + g) * NP + p] = ShiftTable<NP>::entry(qp_reg[k], g);
+                    }
                 }
             }
-        }
-    } else {
-        // four consecutive elements of one query per word, in the byte order of the key words
-        uint32_t* q4_s = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
-        uint32_t q4_reg[(D / 4 * GT + NT - 1) / NT];
+        } else {
+            // four consecutive elements of one query per word, in the byte order of the key words
+            uint32_t* q4_s = reinterpret_cast<uint32_t*>(smem + SM::kQpOff);
+            uint32_t q4_reg[(D / 4 * GT + NT - 1) / NT];
 #pragma unroll
-        for (int k = 0; k < (D / 4 * GT + NT - 1) / NT; ++k) {
-            const int idx = threadIdx.x + k * NT;
-            const int w = idx / GT, g = idx % GT;
-            q4_reg[k] = 0u;
-            if (idx < D / 4 * GT)
-                q4_reg[k] = (uint32_t)(q_s[4 * w][g] & 0xff) | ((uint32_t)(q_s[4 * w + 1][g] & 0xff) << 8) |
-                            ((uint32_t)(q_s[4 * w + 2][g] & 0xff) << 16) | ((uint32_t)(q_s[4 * w + 3][g] & 0xff) << 24);
-        }
-        __syncthreads();                                       // q_s is about to be overwritten
+            for (int k = 0; k < (D / 4 * GT + NT - 1) / NT; ++k) {
+                const int idx = threadIdx.x + k * NT;
+                const int w = idx / GT, g = idx % GT;
+                q4_reg[k] = 0u;
+                if (idx < D / 4 * GT)
+                    q4_reg[k] = (uint32_t)(q_s[4 * w][g] & 0xff) | ((uint32_t)(q_s[4 * w + 1][g] & 0xff) << 8) |
+                                ((uint32_t)(q_s[4 * w + 2][g] & 0xff) << 16) | ((uint32_t)(q_s[4 * w + 3][g] & 0xff) << 24);
+            }
+            __syncthreads();                                       // q_s is about to be overwritten
 #pragma unroll
-        for (int k = 0; k < (D / 4 * GT + NT - 1) / NT; ++k) {
-            const int idx = threadIdx.x + k * NT;
-            if (idx < D / 4 * GT) q4_s[idx] = q4_reg[k];
+            for (int k = 0; k < (D / 4 * GT + NT - 1) / NT; ++k) {
+                const int idx = threadIdx.x + k * NT;
+                if (idx < D / 4 * GT) q4_s[idx] = q4_reg[k];
+            }
         }
-    }
-    __syncthreads();
+        __syncthreads();
 
-    if (warp == NW - 1 && lane < NW) {                        // lane w: the first tile of warp w
-        const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
-        const int t_g = split_begin(n_tiles_g, split, a.n_splits) + lane;
-        if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
-            const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
-            if (p_g >= 0 && p_g < a.n_pages)
-                Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32, !SP);
+        if (warp == NW - 1 && lane < NW) {                        // lane w: the first tile of warp w
+            const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
+            const int t_g = split_begin(n_tiles_g, split, a.n_splits) + lane;
+            if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
+                const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
+                if (p_g >= 0 && p_g < a.n_pages)
+                    Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32, !SP);
+            }
         }
-    }
-    pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
+        pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
+        // the page of the guessed first tile, read again now that it is valid, at the same time as the length(s)
+        // (one round trip instead of two when the guess holds, which it does unless the length crossed a tile boundary)
+        if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
+        again = false;
+        if (ranked && !a.wait_first) {                            // the rank that counts; wait_first took it after the wait already
+            const int b_now = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff),
+                                               &len_ranked);
+            again = b_now != b;
+            b = b_now;
+        }
+    } while (again);
 
     // ---- this warp's tiles; start the first copies ----
-    int len = a.seq_lens[b];
-    // the page of the guessed first tile, read again now that it is valid, at the same time as the length
-    // (one round trip instead of two when the guess holds, which it does unless the length crossed a tile boundary)
-    if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
+    int len = ranked ? len_ranked : a.seq_lens[b];
     int tile_new = -1, pidx_new = -1;
     if (a.Knew) {
         // Fused append: the step's new token goes to position len (if its page is mapped) and is part of

@@ -157,15 +157,28 @@ void split_plan(const Plan& p, int batch, int max_pages, int* n_splits, int* gt)
 __global__ void __launch_bounds__(256) stage_in_kernel(const uint4* __restrict__ q, const uint4* __restrict__ k,
                                                        const uint4* __restrict__ v, uint4* __restrict__ dq,
                                                        uint4* __restrict__ dk, uint4* __restrict__ dv, int nq, int nkv) {
-    // The staging buffer may still be read by the step before.  The kernel after this one — the decode kernel in its
-    // wait-first form, or the append kernel, which waits before anything else — may be scheduled at once: neither
-    // reads the staging buffer before its own wait.
-    pdl_wait();
+    // The inputs sit in host memory that no kernel writes, so they are fetched before the wait and the trip over the
+    // bus runs beside the step before; that step may still read the staging buffer, so the stores come after the
+    // wait.  The kernel after this one (the decode kernel in its wait-first form, or the append kernel, which waits
+    // before anything else) may be scheduled at once: neither reads the staging buffer before its own wait.
     pdl_launch_dependents();
     const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i < nq) dq[i] = q[i];
-    else if (i < nq + nkv) dk[i - nq] = k[i - nq];
-    else if (i < nq + 2 * nkv) dv[i - nq - nkv] = v[i - nq - nkv];
+    const uint4* src = nullptr;
+    uint4* dst = nullptr;
+    if (i < nq) {
+        src = q + i;
+        dst = dq + i;
+    } else if (i < nq + nkv) {
+        src = k + (i - nq);
+        dst = dk + (i - nq);
+    } else if (i < nq + 2 * nkv) {
+        src = v + (i - nq - nkv);
+        dst = dv + (i - nq - nkv);
+    }
+    uint4 x = make_uint4(0u, 0u, 0u, 0u);
+    if (src) x = __ldcv(src);             // host memory: never from a cache line of an earlier step
+    pdl_wait();
+    if (dst) *dst = x;
 }
 
 }  // namespace sa

@@ -99,16 +99,17 @@ __global__ void __launch_bounds__(256) pipe_kernel(int iters, uint32_t one, uint
                 } else if (KIND == PK_SHL_ADD) {
                     asm volatile("{ .reg .u32 t; shl.b32 t, %0, %1; add.u32 %0, t, %2; }" : "+r"(x[i]) : "r"(r), "r"(a));
                 } else if (KIND == PK_LDS128_BCAST) {
-                    // the address depends on the value loaded before (always 0), all lanes read the same 16 bytes
+                    // the address depends on the value loaded before (always 0), all lanes read the same 16 bytes;
+                    // volatile, here and below, so that the access keeps its width although only its first word is used
                     uint32_t y, z, w;
-                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x[i]), "=r"(y), "=r"(z), "=r"(w) : "r"(tab + i * 128 + x[i]));
+                    asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x[i]), "=r"(y), "=r"(z), "=r"(w) : "r"(tab + i * 128 + x[i]));
                 } else if (KIND == PK_LDS64_GATHER) {
                     uint32_t y;
-                    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(x[i]), "=r"(y) : "r"(tab + i * 128 + ((threadIdx.x * 5u) & 15u) * 8u + x[i]));
+                    asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(x[i]), "=r"(y) : "r"(tab + i * 128 + ((threadIdx.x * 5u) & 15u) * 8u + x[i]));
                 } else if (KIND == PK_LDS64_SCATTERED) {
                     uint32_t y;
                     const uint32_t e = ((threadIdx.x * 2654435761u) >> 13) & 15u;      // 11 distinct entries per warp, unevenly spread
-                    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(x[i]), "=r"(y) : "r"(tab + i * 128 + e * 8u + x[i]));
+                    asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(x[i]), "=r"(y) : "r"(tab + i * 128 + e * 8u + x[i]));
                 } else if (KIND == PK_CVT_F32_S32) {
                     asm volatile("{ .reg .f32 t; cvt.rn.f32.s32 t, %0; mov.b32 %0, t; }" : "+r"(x[i]));
                 } else if (KIND == PK_CVT_S32_F32) {

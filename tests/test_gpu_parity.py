@@ -697,7 +697,9 @@ def test_add_on_alu_excludes_shift_by_multiply(dev):
 def test_lost_copy_marks_exactly_its_rows_and_returns(dev, lost):
     """The bounded wait of the staged copies, made to run out: the copy of one tile of one (sequence, KV head) is
     never issued (test hook, 2^10 polls).  The call returns, the rows of that KV head's query heads in that
-    sequence are NaN, every other row is the ordinary result, and an ordinary call afterwards is unaffected."""
+    sequence are NaN, every other row is the ordinary result, and an ordinary call afterwards is unaffected.
+    The hook's kernel also takes its first guess at the length ranks wrong on purpose, so every block here repeats
+    its query prologue for the sequence the ranks after the dependency wait give it."""
     import torch
     b, kvh, tile = lost
     case = synth.make_case("lost", [300, 513, 777], 32, 4, 64, 4, outliers=True, seed=5100)
@@ -751,6 +753,32 @@ def test_length_ranked_batches_cover_every_sequence_once(dev, batch):
         outs.append(O.cpu().numpy())
     check_against_oracle(case, outs[0], dbg.cpu().numpy())
     assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
+
+
+def test_rank_follows_lengths_rewritten_by_the_preceding_kernel(dev):
+    """The decode kernel ranks the sequences twice: ahead of its dependency wait (a guess, so that the query prologue
+    can run early) and after it (the rank that counts; a differing guess repeats the prologue).  Here the kernel in
+    front of every call rewrites the lengths so that the order of the sequences flips, back to back with no
+    synchronisation in between: each call must come out as the oracle's for the lengths then in force, whichever
+    lengths its guess saw."""
+    import dataclasses
+    import torch
+    full = synth.make_case("flip", [700, 400, 450, 700], 32, 4, 64, 4, outliers=True, seed=6200)
+    cfg, cache = build_cache(full, dev, permute_seed=9)
+    Q = t16(full.Q, dev)
+    orders = [[700, 400, 150, 90], [60, 200, 450, 700], [33, 400, 31, 64], [700, 1, 450, 2]]
+    lens_dev = [torch.tensor(o, dtype=torch.int32, device=dev) for o in orders]
+    outs = [torch.full((4, 32, 64), float("nan"), dtype=torch.float32, device=dev) for _ in range(12)]
+    for i, O in enumerate(outs):                               # nothing synchronises inside this loop
+        cache.seq_lens.copy_(lens_dev[i % len(orders)])
+        sa.decode_attention(cfg, cache.handle, Q, O, cache.workspace, None)
+    torch.cuda.synchronize()
+    for j, lens in enumerate(orders):
+        rows = np.concatenate([np.arange(full.cu_lens[b], full.cu_lens[b] + lens[b]) for b in range(4)])
+        cut = dataclasses.replace(full, K=full.K[rows], V=full.V[rows], cu_lens=np.concatenate([[0], np.cumsum(lens)]))
+        ref = ora.decode_attention(cut.Q, cut.K, cut.V, cut.cu_lens, 4, 10, n_threads=8)["O"]
+        for i in range(j, len(outs), len(orders)):
+            assert np.max(np.abs(outs[i].cpu().numpy() - ref)) <= TOL_O, "call %d" % i
 
 
 # ------------------------------------------------------------------ split-K merge: every block shape and pass count
