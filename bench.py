@@ -667,6 +667,20 @@ def run_ours(args):
                                 "achieved": alu_peak * row["alu_pipe_pct"] / 100.0, "issue_slots_frac": row["issue_slots_pct"] / 100.0,
                                 "source": "ncu sm__inst_executed_pipe_alu of the capture at batch %d, kernel sources %s (profiles/); "
                                           "not measured by this run" % (row["batch"], pipes.get("kernel_source_hash"))}
+    code_k = VARIANTS[args.variant][0]
+    if code_k in (1, 2, 4) and not wl.fp16:
+        # The floor of the table datapath of the mantissa codes, measured live: every (key, element, query pair) update
+        # gathers one 8-byte table entry from shared memory, and an SM's shared-memory pipe moves 128 bytes per clock
+        # (profiles/instruction_throughput_b200.md: a 64-bit gather is two wavefronts wherever its lanes point).
+        pairs = (group + 1) // 2
+        table_bytes = wl.batch * wl.T * wl.Hkv * wl.d * pairs * 8.0      # per launch: one layer's cached keys
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        smem_peak = sms * 128.0 * (clocks.get("sm_mhz") or 1965.0) * 1e6
+        line["roofline_shared"] = {"bound": "shared-memory pipe", "unit": "B/s", "peak": smem_peak,
+                                   "achieved": table_bytes / (main_us * 1e-6), "frac": table_bytes / (main_us * 1e-6) / smem_peak,
+                                   "what": "table entries gathered per launch (keys x head_dim x query pairs x 8 B) / main kernel "
+                                           "time, against SMs x 128 B/clk x sampled SM clock; the kernel's other shared-memory "
+                                           "traffic (key codes, values, weights) is not counted"}
     if rank == 0 and args.gpus == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args.variant, args.seq_len, args.batch)
     if rank == 0 and args.gpus == 1 and not args.no_context:
