@@ -662,7 +662,8 @@ def run_ours(args):
         # The resource that actually binds the shift kernels is the integer ALU pipe (shift, logic, permute):
         # 64 lanes per SM and clock.  Fraction from the recorded capture of the nearest batch size.
         row = min(pipes["rows"], key=lambda r: abs(r["batch"] - wl.batch))
-        alu_peak = 148 * 64 * (clocks.get("sm_mhz") or 1965.0) * 1e6      # no clock sample in a very short run: the maximum
+        n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        alu_peak = n_sms * 64 * (clocks.get("sm_mhz") or 1965.0) * 1e6    # no clock sample in a very short run: the maximum
         line["roofline_alu"] = {"bound": "alu", "peak": alu_peak, "unit": "thread-instr/s", "frac": row["alu_pipe_pct"] / 100.0,
                                 "achieved": alu_peak * row["alu_pipe_pct"] / 100.0, "issue_slots_frac": row["issue_slots_pct"] / 100.0,
                                 "source": "ncu sm__inst_executed_pipe_alu of the capture at batch %d, kernel sources %s (profiles/); "
