@@ -755,28 +755,37 @@ def test_length_ranked_batches_cover_every_sequence_once(dev, batch):
     assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
 
 
-def test_rank_follows_lengths_rewritten_by_the_preceding_kernel(dev):
-    """The decode kernel ranks the sequences twice: ahead of its dependency wait (a guess, so that the query prologue
+@pytest.mark.parametrize("fp16", [False, True])
+def test_rank_follows_lengths_rewritten_by_the_preceding_kernel(dev, fp16):
+    """The decode kernels rank the sequences twice: ahead of their dependency wait (a guess, so that the query prologue
     can run early) and after it (the rank that counts; a differing guess repeats the prologue).  Here the kernel in
     front of every call rewrites the lengths so that the order of the sequences flips, back to back with no
     synchronisation in between: each call must come out as the oracle's for the lengths then in force, whichever
     lengths its guess saw."""
     import dataclasses
     import torch
-    full = synth.make_case("flip", [700, 400, 450, 700], 32, 4, 64, 4, outliers=True, seed=6200)
-    cfg, cache = build_cache(full, dev, permute_seed=9)
+    full = synth.make_case("flip", [700, 400, 450, 700], 32, 4, 64, 4, outliers=not fp16, seed=6200)
+    cfg = sa.make_config(64, 32, 4, sa.SA_KV_FP16) if fp16 else None
+    cfg, cache = build_cache(full, dev, cfg=cfg, permute_seed=9)
     Q = t16(full.Q, dev)
     orders = [[700, 400, 150, 90], [60, 200, 450, 700], [33, 400, 31, 64], [700, 1, 450, 2]]
     lens_dev = [torch.tensor(o, dtype=torch.int32, device=dev) for o in orders]
     outs = [torch.full((4, 32, 64), float("nan"), dtype=torch.float32, device=dev) for _ in range(12)]
     for i, O in enumerate(outs):                               # nothing synchronises inside this loop
         cache.seq_lens.copy_(lens_dev[i % len(orders)])
-        sa.decode_attention(cfg, cache.handle, Q, O, cache.workspace, None)
+        if fp16:
+            sa.decode_attention_fp16(cfg, cache.handle, Q, O, cache.workspace)
+        else:
+            sa.decode_attention(cfg, cache.handle, Q, O, cache.workspace, None)
     torch.cuda.synchronize()
     for j, lens in enumerate(orders):
         rows = np.concatenate([np.arange(full.cu_lens[b], full.cu_lens[b] + lens[b]) for b in range(4)])
         cut = dataclasses.replace(full, K=full.K[rows], V=full.V[rows], cu_lens=np.concatenate([[0], np.cumsum(lens)]))
-        ref = ora.decode_attention(cut.Q, cut.K, cut.V, cut.cu_lens, 4, 10, n_threads=8)["O"]
+        if fp16:
+            ref = np.stack([ora.sdpa_fp16(cut.Q[b], cut.K[cut.cu_lens[b]:cut.cu_lens[b + 1]], cut.V[cut.cu_lens[b]:cut.cu_lens[b + 1]])
+                            for b in range(4)])
+        else:
+            ref = ora.decode_attention(cut.Q, cut.K, cut.V, cut.cu_lens, 4, 10, n_threads=8)["O"]
         for i in range(j, len(outs), len(orders)):
             assert np.max(np.abs(outs[i].cpu().numpy() - ref)) <= TOL_O, "call %d" % i
 
