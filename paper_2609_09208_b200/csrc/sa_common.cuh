@@ -49,14 +49,17 @@ sa_status make_plan(const sa_config* cfg, Plan* out);
 // multiples, and for every code fewer, larger blocks mean fewer prologues and partials, which is
 // most of the time of a batch-1 step.  PoT-M1 / M2 keep four blocks of four warps: their finer
 // granularity serves the short and ragged batches those codes are specified for (measured: 16 %
-// faster there, 6 % slower at T = 32768, batch 1).
+// faster there, 6 % slower at T = 32768, batch 1).  At d = 128 (8 KB tiles, one stage buffer per
+// warp) PoT-M4 runs two blocks of eight warps beside their 32 KB tables (16 warps at 128 registers;
+// measured 3 - 22 % faster than three blocks of four); the other codes keep blocks of four warps
+// (larger blocks measured 2 - 13 % slower for them from batch 8 on).
 struct KernelShape {
     int warps, blocks_per_sm;
 };
 constexpr KernelShape decode_shape(int d, int kb) {
     return (kb == 1 || kb == 2) ? KernelShape{4, 4}
            : (d == 64)          ? KernelShape{10, 2}
-           : (kb == 4)          ? KernelShape{4, 3}
+           : (kb == 4)          ? KernelShape{8, 2}
                                 : KernelShape{4, 5};
 }
 constexpr KernelShape kFp16Shape{4, 3};

@@ -169,7 +169,7 @@ extern "C" sa_status sa_decode_attention_static(const sa_config* cfg, const sa_c
     if (!cache || cache->batch <= 0 || cache->max_pages_per_seq <= 0) return SA_ERR_INVALID_ARG;
     int S, GT;
     split_plan(p, cache->batch, cache->max_pages_per_seq, &S, &GT);
-    const size_t need = (size_t)S * cache->batch * p.Hq * (p.d + 2) * sizeof(float);
+    const size_t need = decode_workspace_bytes(p, cache->batch, S);
     if (need > (size_t)SA_STATIC_SCRATCH_BYTES) return SA_ERR_CAPACITY;   // problem too large for the fixed scratch
     void* scratch = nullptr;
     st = static_scratch_address(&scratch);

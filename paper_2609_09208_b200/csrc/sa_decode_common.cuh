@@ -14,7 +14,8 @@ struct DecodeArgs {
     const int32_t* seq_lens;
     const uint16_t* Q;
     float* O;
-    float* partials;          // [n_splits][batch][Hq][D + 2]: {M (int bits), l, O[D]}
+    float* partials;          // [slot][Hq][D + 2]: {M (int bits), l, O[D]}; slot = split * batch + sequence, or, where
+                              // `plan` is set, the block's place among the (sequence, split) pairs of its batch
     int32_t* dbg_scores;
     size_t dbg_stride;
     int batch, Hq, Hkv, G, max_pages, n_pages, n_splits, f_extra, hadamard;
@@ -34,41 +35,119 @@ struct DecodeArgs {
     // The block waits for the preceding kernels before it reads anything, Q included (set when the kernel before
     // this one writes Q and releases its dependents early: the host-buffer entry's staging kernel).
     int wait_first;
+    // Batches of 2 .. kRankedBatchMax sequences (plan_block below): `plan` receives {first slot, splits} of every
+    // sequence for the merge kernel; bal_target is the number of (sequence, split) blocks per grid row that a batch
+    // of unequal lengths is cut into (0: every sequence keeps n_splits).  Null / 0 elsewhere.
+    int32_t* plan;
+    int bal_target;
 };
 
-// Ragged batches: the grid's sequence coordinate is taken as a RANK by cached length, longest first, so that the
-// blocks of the long sequences are dispatched first and the launch ends on the short ones instead of on whichever
-// long sequence happens to come last in the batch.  Every block of the grid must map ranks from the same lengths, so
-// the map that counts is taken after the wait on the preceding kernels (a call before that wait is a guess); ties
-// go to the lower index (the map is a fixed function of the lengths).  The lengths are read past L1, so that a
-// guess leaves nothing stale behind.  One thread per sequence counts the sequences that precede its own: batches
-// up to kRankedBatchMax.
+// Batches of 2 .. kRankedBatchMax sequences: which (sequence, split) a block of the grid works on is decided on the
+// device, from the cached lengths, by every block in the same way.
+//   * The sequences are taken longest first (ties by index), so that the blocks of the long sequences are
+//     dispatched first and the launch ends on the short ones.
+//   * Sequences of equal tile counts keep the host's n_splits each.  Otherwise the grid's x * z blocks of a row are
+//     dealt out in proportion to the lengths: the smallest tiles-per-block is searched for which the sequences'
+//     split counts, ceil(tiles / tiles-per-block) and at least one each, fit into bal_target blocks (the host's
+//     grid, rounded down to whole waves of resident blocks); a sequence's tiles are then cut evenly into its splits.
+//     Blocks of about equal work fill the machine whatever the mix of lengths — with the same n_splits for all, the
+//     blocks of a batch's longest sequences set the time of the launch while the others' slots idle.
+// Block i = z * n_splits + x of a grid row takes the i-th (sequence, split) pair in that order; its partial goes to
+// slot i, and {first slot, splits} of every sequence is left in `plan` for the merge kernel.  Blocks beyond the last
+// pair have nothing to do (b = -1).
+// Every block must work from the same lengths, so the plan that counts is made after the wait on the preceding
+// kernels; one made before that wait is a guess (lengths read past L1, so that it leaves nothing stale behind).
+// `scratch` keeps the guess's lengths and counts: if the lengths read after the wait are the same, the guess stands.
 constexpr int kRankedBatchMax = 128;
-SA_D bool batch_is_ranked(int batch) { return batch > 1 && batch <= kRankedBatchMax; }
-SA_D int sequence_of_rank(const int32_t* seq_lens, int batch, int rank, int* scratch /* shared, batch + 1 ints */,
-                          int* len_out = nullptr /* that sequence's length, as read here */) {
-    for (int i = threadIdx.x; i < batch; i += blockDim.x) scratch[i] = __ldcg(seq_lens + i);
+constexpr int kPlanScratchInts = 3 * kRankedBatchMax + 48;
+SA_HD bool batch_is_ranked(int batch) { return batch > 1 && batch <= kRankedBatchMax; }
+struct BlockPlan {
+    int b, split, n_splits, slot, len;
+};
+// sum of v over the block (every thread gets it); red: 2 x 16 ints, phase alternates between calls
+SA_D int plan_block_sum(int v, int* red, int& phase) {
+    v = __reduce_add_sync(0xffffffffu, v);
+    if ((threadIdx.x & 31) == 0) red[phase * 16 + (threadIdx.x >> 5)] = v;
     __syncthreads();
-    for (int i = threadIdx.x; i < batch; i += blockDim.x) {
-        const int li = scratch[i];
-        int before = 0;
-        for (int j = 0; j < batch; ++j) {
-            const int lj = scratch[j];
-            before += (lj > li || (lj == li && j < i)) ? 1 : 0;
+    int total = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) total += red[phase * 16 + w];
+    phase ^= 1;
+    return total;
+}
+// z, x: the block's grid coordinates (z may be falsified by a test hook's guess); recheck: a plan made from `scratch`
+// earlier (prev) stands if the lengths have not changed; counts: this is the plan that counts (it is left for the merge)
+SA_D BlockPlan plan_block(const DecodeArgs& a, int z, int x, bool recheck, bool counts, const BlockPlan& prev, int* scratch) {
+    const int B = a.batch, S = a.n_splits, j = threadIdx.x;     // one thread per sequence (a block has >= 128 threads)
+    int* len_s = scratch;
+    int* cnt_s = scratch + kRankedBatchMax;
+    int* pre_s = scratch + 2 * kRankedBatchMax;
+    int* red_s = scratch + 3 * kRankedBatchMax;                 // 32 ints
+    int* out_s = red_s + 32;                                    // 4 ints
+    const bool writer = counts && a.plan != nullptr && z == 0 && x == 0 && blockIdx.y == 0;
+    const int len_now = (j < B) ? __ldcg(a.seq_lens + j) : 0;
+    if (recheck) {
+        if (!__syncthreads_or((j < B && len_now != len_s[j]) ? 1 : 0)) {
+            if (writer && j < B) {
+                a.plan[2 * j] = pre_s[j];
+                a.plan[2 * j + 1] = cnt_s[j];
+            }
+            return prev;
         }
-        if (before == rank) scratch[batch] = i;
+    }
+    if (j < B) len_s[j] = len_now;
+    if (j == 0) out_s[0] = -1;
+    const int cap = a.max_pages * kPageTokens;
+    const int tiles = (j < B) ? (min(max(len_now + (a.Knew ? 1 : 0), 0), cap) + 31) >> 5 : 0;
+    __syncthreads();
+    const int tiles0 = (min(max(len_s[0] + (a.Knew ? 1 : 0), 0), cap) + 31) >> 5;
+    int cnt = S;                                                // splits of sequence j
+    if (a.bal_target > 0 && !__syncthreads_and((j >= B || tiles == tiles0) ? 1 : 0)) {
+        int phase = 0;
+        const int G = a.bal_target, N = plan_block_sum(tiles, red_s, phase);
+        int tpb = max(1, (N + G - 1) / G);
+        for (int it = 0; it < 48; ++it) {                       // (the first guess is at most a few per cent short)
+            cnt = (j < B) ? max(1, (tiles + tpb - 1) / tpb) : 0;
+            const int total = plan_block_sum(cnt, red_s, phase);
+            if (total <= G) break;
+            tpb = max(tpb + 1, (int)(((long long)tpb * total + G - 1) / G));
+            cnt = (j < B) ? S : 0;                              // (if the search ran out: the host's plan, which always fits)
+        }
+    }
+    if (j < B) cnt_s[j] = cnt;
+    __syncthreads();
+    if (j < B) {
+        int pre = 0;                                            // blocks of the sequences ahead of this one
+        for (int k = 0; k < B; ++k) {
+            const int lk = len_s[k];
+            if (lk > len_now || (lk == len_now && k < j)) pre += cnt_s[k];
+        }
+        pre_s[j] = pre;
+        const int i = z * S + x;
+        if (i >= pre && i < pre + cnt) {
+            out_s[0] = j;
+            out_s[1] = i - pre;
+            out_s[2] = cnt;
+        }
+        if (writer) {
+            a.plan[2 * j] = pre;
+            a.plan[2 * j + 1] = cnt;
+        }
     }
     __syncthreads();
-    const int b = scratch[batch];
-    if (len_out) *len_out = scratch[b];
-    __syncthreads();                                          // the scratch is about to be used for something else
-    return b;
+    BlockPlan r;
+    r.b = out_s[0];
+    r.split = out_s[1];
+    r.n_splits = out_s[2];
+    r.slot = z * S + x;
+    r.len = r.b >= 0 ? len_s[r.b] : 0;
+    __syncthreads();                                            // out_s may be written again by a later call
+    return r;
 }
 
 // red_s[w][g] = {M (int bits), l, O[D]} of warp w (NW warps per block) -> the block's partial in the workspace
 // (used by the kernels whose warps write their states to shared memory themselves).
 template <int D, int GT, int NW = 4>
-SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], int b, int h0, int split) {
+SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], int slot, int h0) {
     for (int idx = threadIdx.x; idx < GT * (D + 1); idx += 32 * NW) {
         const int g = idx / (D + 1), c = idx % (D + 1);       // c = 0: l, c >= 1: O[c - 1]
         int Ms = kMNone;
@@ -80,7 +159,7 @@ SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2]
             const int Mw = __float_as_int(red_s[w][g][0]);
             if (Mw != kMNone) v += red_s[w][g][1 + c] * pow2i_neg(Mw - Ms);
         }
-        float* dst = a.partials + (((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2);
+        float* dst = a.partials + ((size_t)slot * a.Hq + h0 + g) * (D + 2);
         dst[1 + c] = v;
         if (c == 0) dst[0] = __int_as_float(Ms);
     }
@@ -97,8 +176,8 @@ SA_D void block_combine_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2]
 // 2 t4 + 1 (c1, c3).
 template <int D, int GT, int NW>
 SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], const int (&M)[GT],
-                                float (&l)[GT], float (&acc)[D / 16][4], int lane, int warp, int b, int h0,
-                                int split, bool failed = false) {
+                                float (&l)[GT], float (&acc)[D / 16][4], int lane, int warp, int slot, int h0,
+                                bool failed = false) {
     const int gq = lane >> 2, t4 = lane & 3;
     float lsum[GT];
 #pragma unroll
@@ -153,7 +232,7 @@ SA_D void block_merge_and_store(const DecodeArgs& a, float (*red_s)[GT][D + 2], 
             for (int w = 1; w < NW; ++w) v += red_s[w][g][c];
         }
         if (poisoned && c <= 1) v = (c == 0) ? __int_as_float(0) : __int_as_float(0x7fc00000);   // M = 0, l = NaN
-        a.partials[(((size_t)split * a.batch + b) * a.Hq + h0 + g) * (D + 2) + c] = v;
+        a.partials[((size_t)slot * a.Hq + h0 + g) * (D + 2) + c] = v;
     }
 }
 
@@ -181,6 +260,7 @@ struct BumpArgs {
     const int32_t* page_table;
     int max_pages, n_pages, Hq;
     int early_release;        // release the dependents of the merge kernel before its own wait (see merge_kernel)
+    const int32_t* plan;      // {first slot, splits} per sequence (plan_block), or null: slots split * batch + sequence
 };
 
 template <int D, int kMergeThreads>
@@ -208,9 +288,16 @@ __global__ void __launch_bounds__(kMergeThreads, 2048 / kMergeThreads) merge_ker
         const int pidx = (len >= 0 && lp < bump.max_pages) ? bump.page_table[(size_t)b * bump.max_pages + lp] : -1;
         if (pidx >= 0 && pidx < bump.n_pages) bump.seq_lens[b] = len + 1;
     }
-    const size_t stride = (size_t)n_rows * (D + 2);
+    size_t stride = (size_t)n_rows * (D + 2);
     const int ln = threadIdx.x % kMergeLanes, grp = threadIdx.x / kMergeLanes;
     const float* base = partials + (size_t)row * (D + 2);
+    if (bump.plan) {                                          // the sequence's splits sit in consecutive slots
+        const int b = row / bump.Hq;
+        const int first = bump.plan[2 * b];
+        n_splits = bump.plan[2 * b + 1];
+        stride = (size_t)bump.Hq * (D + 2);
+        base = partials + ((size_t)first * bump.Hq + row % bump.Hq) * (D + 2);
+    }
     const float* obase = base + 2 + part * kMergeDims + ln * 4;
     int Ml = kMNone;                                          // this thread's splits: grp, grp + 32, ...
     float l = 0.0f;
@@ -302,8 +389,15 @@ sa_status decode_step_impl(const sa_config* cfg, const sa_cache* cache, const ui
                            const uint16_t* V_new, float* O, void* workspace, size_t workspace_bytes, sa_stream stream,
                            bool q_after_wait);
 
+// Bytes of the split-K workspace: the partials and, for the batches whose blocks are planned on the device, the plan.
+inline size_t decode_workspace_bytes(const Plan& p, int batch, int S, bool with_plan = true) {
+    const size_t partials = (size_t)S * batch * p.Hq * (p.d + 2) * sizeof(float);
+    return partials + ((with_plan && batch_is_ranked(batch)) ? (((size_t)batch * 8 + 15) & ~(size_t)15) : 0);
+}
+
+// with_plan = false: the caller's kernels index the partials by (split, sequence) themselves (the shift-based A.V option)
 inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16_t* Q, float* O,
-                                  void* workspace, size_t workspace_bytes, DecodeArgs* a, int* gt) {
+                                  void* workspace, size_t workspace_bytes, DecodeArgs* a, int* gt, bool with_plan = true) {
     if (!c || !c->pages || !c->page_table || !c->seq_lens || !Q || !O) return SA_ERR_INVALID_ARG;
     if (c->batch <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return SA_ERR_INVALID_ARG;
     if (c->batch > 65535) return SA_ERR_CAPACITY;
@@ -314,7 +408,7 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     split_plan(p, c->batch, c->max_pages_per_seq, &S, &GT);
     // the kernels place the splits with 32-bit arithmetic: tiles * (splits + 1) must stay below 2^31
     if ((long long)c->max_pages_per_seq * (kPageTokens / kTileTokens) * (S + 1) >= (1LL << 31)) return SA_ERR_CAPACITY;
-    const size_t need = (size_t)S * c->batch * p.Hq * (p.d + 2) * sizeof(float);
+    const size_t need = decode_workspace_bytes(p, c->batch, S, with_plan);
     if (!workspace || workspace_bytes < need) return SA_ERR_CAPACITY;
     if (mis(workspace, 16)) return SA_ERR_ALIGNMENT;
     a->pages = static_cast<const uint8_t*>(c->pages);
@@ -350,6 +444,18 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
     a->Vnew = nullptr;
     a->lost_b = a->lost_kvh = a->lost_tile = -1;
     a->wait_first = 0;
+    a->plan = nullptr;
+    a->bal_target = 0;
+    if (with_plan && batch_is_ranked(c->batch)) {
+        a->plan = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + (size_t)S * c->batch * p.Hq * (p.d + 2) * sizeof(float));
+        // blocks per grid row that a batch of unequal lengths is cut into: the grid, rounded down to whole waves of
+        // resident blocks (equal blocks gain nothing from a last, partly filled wave)
+        const KernelShape shape = p.fp16 ? kFp16Shape : decode_shape(p.d, p.int8 ? 8 : p.k);
+        const long long rows = (long long)p.Hkv * (p.G / GT), slots = (long long)sm_count() * shape.blocks_per_sm;
+        long long per_row = (long long)S * c->batch;
+        if (per_row * rows > slots) per_row = ((per_row * rows) / slots) * slots / rows;
+        a->bal_target = (int)(per_row < c->batch ? c->batch : per_row);
+    }
     *gt = GT;
     return SA_OK;
 }
@@ -357,7 +463,7 @@ inline sa_status make_decode_args(const Plan& p, const sa_cache* c, const uint16
 inline sa_status launch_merge(const Plan& p, const DecodeArgs& a, cudaStream_t s) {
     const int rows = a.batch * a.Hq;
     const int early = (!p.fp16 && decode_shape(p.d, p.int8 ? 8 : p.k).warps >= 8) ? 1 : 0;
-    BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq, early};
+    BumpArgs bump{a.Knew ? const_cast<int32_t*>(a.seq_lens) : nullptr, a.page_table, a.max_pages, a.n_pages, a.Hq, early, a.plan};
     cudaError_t err;
     const bool small = a.n_splits <= kMergeSmallSplits;
     const dim3 grid(rows * (p.d / kMergeDims));

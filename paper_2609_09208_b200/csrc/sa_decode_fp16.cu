@@ -67,13 +67,14 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     const int chunks = a.G / GT;
     const int kvh = blockIdx.y / chunks;
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;
-    // ragged batches: longest sequence first, the rank guessed ahead of the dependency wait and settled after it
-    // (see the quantised kernel)
+    // batches of 2 .. 128 sequences: the block's (sequence, split) is dealt by plan_block from the cached lengths,
+    // guessed ahead of the dependency wait and settled after it (see the quantised kernel)
     const bool ranked = batch_is_ranked(a.batch);
-    int b = blockIdx.z, len_ranked = 0;
+    int* plan_scratch = reinterpret_cast<int*>(smem + SM::kStageOff);
+    BlockPlan bp{(int)blockIdx.z, (int)blockIdx.x, a.n_splits, (int)(blockIdx.x * a.batch + blockIdx.z), 0};
     if (a.wait_first) pdl_wait();
-    if (ranked) b = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff), &len_ranked);
-    const int split = blockIdx.x;
+    if (ranked) bp = plan_block(a, blockIdx.z, blockIdx.x, false, a.wait_first != 0, bp, plan_scratch);
+    int b = bp.b;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
     const uint8_t* stage_ptr0 = smem + SM::kStageOff + warp * kStages * Stage::kBytes;
@@ -95,11 +96,13 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     bool again;
 #pragma unroll 1
     do {
+        const int split_g = bp.split, nsp_g = bp.n_splits;         // what the hint below is computed for
+        const int bq = b < 0 ? 0 : b;                              // (a block without work so far prepares sequence 0)
 #pragma unroll
         for (int kb = 0; kb < KB16; ++kb) {
             qa[kb][0] = qa[kb][1] = 0u;
             if (row < GT) {
-                const uint32_t* q32 = reinterpret_cast<const uint32_t*>(a.Q + ((size_t)b * a.Hq + h0 + row) * D);
+                const uint32_t* q32 = reinterpret_cast<const uint32_t*>(a.Q + ((size_t)bq * a.Hq + h0 + row) * D);
                 qa[kb][0] = __ldg(q32 + kb * 8 + quad);
                 qa[kb][1] = __ldg(q32 + kb * 8 + 4 + quad);
             }
@@ -109,12 +112,12 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         // may be about to change (loads that bypass L1; a hint only).
         tile_g = -1, pidx_g = -1;
         if (lane == 0) {
-            const int len_g = (ranked ? len_ranked : __ldcg(a.seq_lens + b)) + (a.Knew ? 1 : 0);
+            const int len_g = (ranked ? bp.len : __ldcg(a.seq_lens + bq)) + (a.Knew ? 1 : 0);
             const int n_tiles_g = (min(max(len_g, 0), a.max_pages * kPageTokens) + 31) >> 5;
-            const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
-            if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
+            const int t_g = split_begin(n_tiles_g, bp.split, bp.n_splits) + warp;
+            if (t_g < split_begin(n_tiles_g, (bp.split + 1), bp.n_splits)) {
                 tile_g = t_g;
-                const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
+                const int p_g = __ldcg(a.page_table + (size_t)bq * a.max_pages + (t_g >> 1));
                 if (p_g >= 0 && p_g < a.n_pages)
                     Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32);
             }
@@ -122,17 +125,19 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
         // the page of the guessed first tile, read again now that it is valid, together with the length(s) (one round
         // trip instead of two when the guess holds)
-        if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
+        if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)bq * a.max_pages + (tile_g >> 1)];
         again = false;
         if (ranked && !a.wait_first) {
-            const int b_now = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff),
-                                               &len_ranked);
-            again = b_now != b;
-            b = b_now;
+            bp = plan_block(a, blockIdx.z, blockIdx.x, true, true, bp, plan_scratch);
+            again = bp.b != bq && bp.b >= 0;
+            if (bp.split != split_g || bp.n_splits != nsp_g) tile_g = -1;     // the hint was for other tiles
+            b = bp.b;
         }
     } while (again);
+    if (b < 0) return;                                            // more blocks than (sequence, split) pairs
+    const int split = bp.split, n_splits = bp.n_splits;
 
-    int len = ranked ? len_ranked : a.seq_lens[b];
+    int len = ranked ? bp.len : a.seq_lens[b];
     int tile_new = -1, pidx_new = -1;
     if (a.Knew) {
         // fused append (see the quantised kernel): the step's new token goes to position len if its page is mapped
@@ -144,8 +149,8 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         }
     }
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = split_begin(n_tiles, split, a.n_splits);
-    const int tile1 = split_begin(n_tiles, (split + 1), a.n_splits);
+    const int tile0 = split_begin(n_tiles, split, n_splits);
+    const int tile1 = split_begin(n_tiles, (split + 1), n_splits);
     const int first = tile0 + warp;
     const int n_my = first < tile1 ? (tile1 - first + 3) >> 2 : 0;
     if (tile_new >= first && tile_new < tile1 && (tile_new - first) % 4 == 0) {      // this warp owns that tile
@@ -291,7 +296,7 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         }
     }
     __syncthreads();
-    block_combine_and_store<D, GT>(a, red_s, b, h0, split);
+    block_combine_and_store<D, GT>(a, red_s, bp.slot, h0);
 }
 
 }  // namespace sa

@@ -3,7 +3,7 @@
 #pragma once
 // Decode attention over the power-of-two key cache: the hot path.
 //
-// Grid (split, KV head x query chunk, sequence); 4 or 10 warps per block (decode_shape).  A block
+// Grid (split, KV head x query chunk, sequence); 4, 8 or 10 warps per block (decode_shape).  A block
 // quantises its GT query heads into shared memory (ahead of its wait on the preceding kernel),
 // then each of its warps walks its own 32-key tiles of the block's slice of the key axis with a
 // private online-softmax state, so the main loop has no block-wide barrier.  Per tile: lane = key
@@ -97,19 +97,19 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     const int chunks = a.G / GT;
     const int kvh = blockIdx.y / chunks;
     const int h0 = kvh * a.G + (blockIdx.y % chunks) * GT;     // first query head of this block
-    // Sequence of this block: grid coordinate z itself, or (ragged batches) the sequence whose length has rank z.
-    // The rank taken here, from lengths the preceding kernel may be about to change, is a guess that lets the
-    // query prologue run ahead of the dependency wait; the rank taken after the wait decides, and the prologue is
-    // repeated in the rare case that the two differ (a step adds one token to every sequence, which keeps the order).
-    // The test-hook instantiation guesses wrong on purpose, so that its tests walk the repeat.
+    // What this block works on: sequence z and split x of the host's n_splits, or (batches of 2 .. 128 sequences)
+    // what plan_block deals it from the cached lengths.  The plan made here, from lengths the preceding kernel may be
+    // about to change, is a guess that lets the query prologue run ahead of the dependency wait; the plan made after
+    // the wait decides, and the prologue is repeated in the rare case that it names another sequence (a step adds
+    // one token to every sequence, which keeps their order).  The test-hook instantiation guesses wrong on purpose, so
+    // that its tests walk the repeat.
     const bool ranked = batch_is_ranked(a.batch);
-    int b = blockIdx.z;
+    int* plan_scratch = reinterpret_cast<int*>(smem + SM::kStageOff);
+    BlockPlan bp{(int)blockIdx.z, (int)blockIdx.x, a.n_splits, (int)(blockIdx.x * a.batch + blockIdx.z), 0};
     if (a.wait_first) pdl_wait();
-    int len_ranked = 0;                                        // the length that came with the rank
     if (ranked)
-        b = sequence_of_rank(a.seq_lens, a.batch, LOST ? (blockIdx.z + 1) % a.batch : blockIdx.z,
-                             reinterpret_cast<int*>(smem + SM::kStageOff), &len_ranked);
-    const int split = blockIdx.x;
+        bp = plan_block(a, LOST ? (blockIdx.z + 1) % a.batch : blockIdx.z, blockIdx.x, false, a.wait_first != 0, bp, plan_scratch);
+    int b = bp.b;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * NS * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * NS * Stage::kBytes;
     const uint8_t* stage_ptr0 = smem + SM::kStageOff + warp * NS * Stage::kBytes;
@@ -132,15 +132,17 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 #pragma unroll 1
     do {
         len_g = 0, tile_g = -1, pidx_g = -1;
-        if (ranked) len_g = len_ranked;
-        else if (lane == 0 || warp == NW - 1) len_g = __ldcg(a.seq_lens + b);
+        const int split_g = bp.split, nsp_g = bp.n_splits;         // what the hints below are computed for
+        const int bq = b < 0 ? 0 : b;                              // (a block without work so far prepares sequence 0)
+        if (ranked) len_g = bp.len;
+        else if (lane == 0 || warp == NW - 1) len_g = __ldcg(a.seq_lens + bq);
 
         // ---- prologue: quantise the GT query heads (eq. (2)) and pack them two per register.  It reads
         // only Q, which no kernel of a decode step writes, so it runs BEFORE the wait on the preceding
         // kernel (the cache append) and overlaps it. ----
         for (int g = warp; g < GT; g += NW) {
             uint32_t bits[EPL];
-            load_vec_bits<EPL>(a.Q + ((size_t)b * a.Hq + h0 + g) * D, lane, bits);
+            load_vec_bits<EPL>(a.Q + ((size_t)bq * a.Hq + h0 + g) * D, lane, bits);
             int q[EPL];
             const float delta = quantise_query_vec<EPL>(bits, lane, a.hadamard != 0, q);
 #pragma unroll
@@ -150,8 +152,8 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         __syncthreads();
         if (lane == 0) {
             const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
-            const int t_g = split_begin(n_tiles_g, split, a.n_splits) + warp;
-            if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) tile_g = t_g;
+            const int t_g = split_begin(n_tiles_g, bp.split, bp.n_splits) + warp;
+            if (t_g < split_begin(n_tiles_g, (bp.split + 1), bp.n_splits)) tile_g = t_g;
         }
         if constexpr (SM::kTable) {
             // table of query multiples, built by repeated addition: row (m, pair) = {q_lo, q_hi} * (2^KB + mu)
@@ -241,9 +243,9 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
 
         if (warp == NW - 1 && lane < NW) {                        // lane w: the first tile of warp w
             const int n_tiles_g = (min(max(len_g + (a.Knew ? 1 : 0), 0), a.max_pages * kPageTokens) + 31) >> 5;
-            const int t_g = split_begin(n_tiles_g, split, a.n_splits) + lane;
-            if (t_g < split_begin(n_tiles_g, (split + 1), a.n_splits)) {
-                const int p_g = __ldcg(a.page_table + (size_t)b * a.max_pages + (t_g >> 1));
+            const int t_g = split_begin(n_tiles_g, bp.split, bp.n_splits) + lane;
+            if (t_g < split_begin(n_tiles_g, (bp.split + 1), bp.n_splits)) {
+                const int p_g = __ldcg(a.page_table + (size_t)bq * a.max_pages + (t_g >> 1));
                 if (p_g >= 0 && p_g < a.n_pages)
                     Stage::prefetch(a.pages + ((size_t)p_g * a.Hkv + kvh) * a.page_bytes, (t_g & 1) * 32, !SP);
             }
@@ -251,18 +253,20 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         pdl_wait();                 // everything below reads what the preceding kernels in the stream wrote (the cache)
         // the page of the guessed first tile, read again now that it is valid, at the same time as the length(s)
         // (one round trip instead of two when the guess holds, which it does unless the length crossed a tile boundary)
-        if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)b * a.max_pages + (tile_g >> 1)];
+        if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)bq * a.max_pages + (tile_g >> 1)];
         again = false;
-        if (ranked && !a.wait_first) {                            // the rank that counts; wait_first took it after the wait already
-            const int b_now = sequence_of_rank(a.seq_lens, a.batch, blockIdx.z, reinterpret_cast<int*>(smem + SM::kStageOff),
-                                               &len_ranked);
-            again = b_now != b;
-            b = b_now;
+        if (ranked && !a.wait_first) {                            // the plan that counts; wait_first made it after the wait already
+            bp = plan_block(a, blockIdx.z, blockIdx.x, true, true, bp, plan_scratch);
+            again = bp.b != bq && bp.b >= 0;
+            if (bp.split != split_g || bp.n_splits != nsp_g) tile_g = -1;     // the hint was for other tiles
+            b = bp.b;
         }
     } while (again);
+    if (b < 0) return;                                            // more blocks than (sequence, split) pairs
+    const int split = bp.split, n_splits = bp.n_splits;
 
     // ---- this warp's tiles; start the first copies ----
-    int len = ranked ? len_ranked : a.seq_lens[b];
+    int len = ranked ? bp.len : a.seq_lens[b];
     int tile_new = -1, pidx_new = -1;
     if (a.Knew) {
         // Fused append: the step's new token goes to position len (if its page is mapped) and is part of
@@ -276,8 +280,8 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
     }
     const int n_tiles = (min(len, a.max_pages * kPageTokens) + 31) >> 5;
-    const int tile0 = split_begin(n_tiles, split, a.n_splits);
-    const int tile1 = split_begin(n_tiles, (split + 1), a.n_splits);
+    const int tile0 = split_begin(n_tiles, split, n_splits);
+    const int tile1 = split_begin(n_tiles, (split + 1), n_splits);
     const int first = tile0 + warp;
     const int n_my = first < tile1 ? (tile1 - first + NW - 1) / NW : 0;
     if (tile_new >= first && tile_new < tile1 && (tile_new - first) % NW == 0) {      // warp-uniform: this warp owns that tile
@@ -622,7 +626,7 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
         return;
     }
-    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, b, h0, split, failed);
+    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, bp.slot, h0, failed);
 }
 
 template <int D, int KB, bool NIB, int GT, int MODE>

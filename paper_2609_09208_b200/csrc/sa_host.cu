@@ -217,7 +217,7 @@ sa_status sa_workspace_bytes(const sa_config* cfg, int batch, int max_pages_per_
     if (st != SA_OK) return st;
     int S, GT;
     split_plan(p, batch, max_pages_per_seq, &S, &GT);
-    *out = (size_t)S * batch * p.Hq * (p.d + 2) * sizeof(float);
+    *out = decode_workspace_bytes(p, batch, S);
     return SA_OK;
 }
 

@@ -210,7 +210,7 @@ __global__ void __launch_bounds__(128) shiftav_kernel(DecodeArgs a) {
         for (int c = 0; c < DPL; ++c) red_s[warp][g][2 + lane * DPL + c] = O[g][c] * vs;
     }
     __syncthreads();
-    block_combine_and_store<D, GT, 4>(a, red_s, b, h0, split);
+    block_combine_and_store<D, GT, 4>(a, red_s, split * a.batch + b, h0);
 }
 
 template <int D, int GT>
@@ -276,7 +276,7 @@ extern "C" sa_status sa_decode_attention_shiftav(const sa_config* cfg, const sa_
     if (n_bits < 1 || n_bits > 18 || k_max < 0 || k_max > n_bits) return SA_ERR_INVALID_ARG;
     DecodeArgs a;
     int GT;
-    st = make_decode_args(p, cache, Q, O, workspace, workspace_bytes, &a, &GT);
+    st = make_decode_args(p, cache, Q, O, workspace, workspace_bytes, &a, &GT, false);   // statistics per (split, sequence)
     if (st != SA_OK) return st;
     size_t zo, mo, go, total;
     shiftav_layout(p, cache->batch, cache->max_pages_per_seq, a.n_splits, GT, &zo, &mo, &go, &total);

@@ -105,7 +105,9 @@ def test_workspace_and_staging_sizes():
     assert w > 0 and w % (32 * 66 * 4) == 0
     n_splits = w // (32 * 66 * 4)
     assert 1 <= n_splits <= 512
-    assert sa.workspace_bytes(cfg, 16, 256) % (16 * 32 * 66 * 4) == 0
+    # batches of 2 .. 128 sequences: the partials plus two words per sequence (first slot, splits) for the merge kernel
+    assert (sa.workspace_bytes(cfg, 16, 256) - 16 * 8) % (16 * 32 * 66 * 4) == 0
+    assert sa.workspace_bytes(cfg, 129, 256) % (129 * 32 * 66 * 4) == 0
     assert sa.workspace_bytes(cfg, 1, 1) == 32 * 66 * 4          # a single page: no split
     assert _status(sa.workspace_bytes, cfg, 0, 4) == 1
     assert sa.staging_bytes(cfg, 2) >= 2 * (32 * 64 * 2 + 2 * 4 * 64 * 2 + 32 * 64 * 4)

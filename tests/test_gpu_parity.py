@@ -755,6 +755,40 @@ def test_length_ranked_batches_cover_every_sequence_once(dev, batch):
     assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
 
 
+@pytest.mark.parametrize("lens", [[20000] + [40] * 15, [3000, 1] + [0] * 6, [5000] + [33] * 127, [64 * k + 1 for k in range(1, 40)]])
+def test_splits_dealt_by_length_for_extreme_mixes(dev, lens):
+    """Batches of unequal lengths: the blocks of the grid are dealt to the sequences in proportion to their lengths
+    (one sequence may take nearly all of them, more than one pass of the merge kernel; others a single block; some
+    blocks none).  Integer scores and outputs as the oracle's, twice in a row bit for bit; the FP16 kernel likewise.
+    (The fused step over a batch of unequal lengths: test_decode_step_equals_append_then_decode.)"""
+    import torch
+    lens = np.asarray(lens)
+    case = synth.make_case("mix", lens, 8, 1, 64, 4, outliers=True, seed=6300 + len(lens))
+    cfg, cache = build_cache(case, dev, permute_seed=11)
+    outs = []
+    for _ in range(2):
+        O = torch.full((case.batch, 8, 64), float("nan"), dtype=torch.float32, device=dev)
+        dbg = torch.full((case.batch, 8, cache.max_pages * 64), -7, dtype=torch.int32, device=dev)
+        sa.decode_attention(cfg, cache.handle, t16(case.Q, dev), O, cache.workspace, dbg)
+        torch.cuda.synchronize()
+        outs.append(O.cpu().numpy())
+    check_against_oracle(case, outs[0], dbg.cpu().numpy())
+    assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
+    # the FP16 kernel deals its blocks the same way
+    fcfg = sa.make_config(64, 8, 1, sa.SA_KV_FP16)
+    _, fcache = build_cache(case, dev, cfg=fcfg, permute_seed=12)
+    O = torch.full((case.batch, 8, 64), float("nan"), dtype=torch.float32, device=dev)
+    sa.decode_attention_fp16(fcfg, fcache.handle, t16(case.Q, dev), O, fcache.workspace)
+    torch.cuda.synchronize()
+    O = O.cpu().numpy()
+    for b in range(case.batch):
+        if lens[b] == 0:
+            assert np.all(O[b] == 0)
+            continue
+        ref = ora.sdpa_fp16(case.Q[b], case.K[case.cu_lens[b]:case.cu_lens[b + 1]], case.V[case.cu_lens[b]:case.cu_lens[b + 1]])
+        assert np.max(np.abs(O[b] - ref)) <= TOL_O
+
+
 @pytest.mark.parametrize("fp16", [False, True])
 def test_rank_follows_lengths_rewritten_by_the_preceding_kernel(dev, fp16):
     """The decode kernels rank the sequences twice: ahead of their dependency wait (a guess, so that the query prologue
