@@ -52,8 +52,9 @@ struct DecodeArgs {
 //     grid, rounded down to whole waves of resident blocks); a sequence's tiles are then cut evenly into its splits.
 //     Blocks of about equal work fill the machine whatever the mix of lengths — with the same n_splits for all, the
 //     blocks of a batch's longest sequences set the time of the launch while the others' slots idle.
+// (Sequences of equal tile counts are simply taken in index order.)
 // Block i = z * n_splits + x of a grid row takes the i-th (sequence, split) pair in that order; its partial goes to
-// slot i, and {first slot, splits} of every sequence is left in `plan` for the merge kernel.  Blocks beyond the last
+// slot i (the kernels recompute i from their grid coordinates), and {first slot, splits} of every sequence is left in `plan` for the merge kernel.  Blocks beyond the last
 // pair have nothing to do (b = -1).
 // Every block must work from the same lengths, so the plan that counts is made after the wait on the preceding
 // kernels; one made before that wait is a guess (lengths read past L1, so that it leaves nothing stale behind).
@@ -62,7 +63,7 @@ constexpr int kRankedBatchMax = 128;
 constexpr int kPlanScratchInts = 3 * kRankedBatchMax + 48;
 SA_HD bool batch_is_ranked(int batch) { return batch > 1 && batch <= kRankedBatchMax; }
 struct BlockPlan {
-    int b, split, n_splits, slot, len;
+    int b, split, n_splits, len;      // sequence (-1: none), which of its n_splits parts, the length the plan was made from
 };
 // sum of v over the block (every thread gets it); red: 2 x 16 ints, phase alternates between calls
 SA_D int plan_block_sum(int v, int* red, int& phase) {
@@ -76,7 +77,15 @@ SA_D int plan_block_sum(int v, int* red, int& phase) {
 }
 // z, x: the block's grid coordinates (z may be falsified by a test hook's guess); recheck: a plan made from `scratch`
 // earlier (prev) stands if the lengths have not changed; counts: this is the plan that counts (it is left for the merge)
-SA_D BlockPlan plan_block(const DecodeArgs& a, int z, int x, bool recheck, bool counts, const BlockPlan& prev, int* scratch) {
+struct PlanArgs {              // what plan_block reads of the kernel arguments (by value: the call takes no address of them)
+    const int32_t* seq_lens;
+    int32_t* plan;
+    int batch, n_splits, bal_target, max_pages, Knew;
+};
+SA_D PlanArgs plan_args(const DecodeArgs& a) {
+    return PlanArgs{a.seq_lens, a.plan, a.batch, a.n_splits, a.bal_target, a.max_pages, a.Knew ? 1 : 0};
+}
+SA_D BlockPlan plan_block(PlanArgs a, int z, int x, bool recheck, bool counts, BlockPlan prev, int* scratch) {
     const int B = a.batch, S = a.n_splits, j = threadIdx.x;     // one thread per sequence (a block has >= 128 threads)
     int* len_s = scratch;
     int* cnt_s = scratch + kRankedBatchMax;
@@ -101,7 +110,26 @@ SA_D BlockPlan plan_block(const DecodeArgs& a, int z, int x, bool recheck, bool 
     __syncthreads();
     const int tiles0 = (min(max(len_s[0] + (a.Knew ? 1 : 0), 0), cap) + 31) >> 5;
     int cnt = S;                                                // splits of sequence j
-    if (a.bal_target > 0 && !__syncthreads_and((j >= B || tiles == tiles0) ? 1 : 0)) {
+    const bool uniform = __syncthreads_and((j >= B || tiles == tiles0) ? 1 : 0) != 0;
+    if (uniform) {
+        // equal tile counts: the blocks are equal whatever the order, so sequence z keeps the grid's own blocks
+        if (j < B) {
+            cnt_s[j] = S;
+            pre_s[j] = j * S;
+            if (writer) {
+                a.plan[2 * j] = j * S;
+                a.plan[2 * j + 1] = S;
+            }
+        }
+        BlockPlan r;
+        r.b = z;
+        r.split = x;
+        r.n_splits = S;
+        r.len = len_s[z];
+        __syncthreads();                                        // (as at the end of the general case)
+        return r;
+    }
+    if (a.bal_target > 0) {
         int phase = 0;
         const int G = a.bal_target, N = plan_block_sum(tiles, red_s, phase);
         int tpb = max(1, (N + G - 1) / G);
@@ -138,7 +166,6 @@ SA_D BlockPlan plan_block(const DecodeArgs& a, int z, int x, bool recheck, bool 
     r.b = out_s[0];
     r.split = out_s[1];
     r.n_splits = out_s[2];
-    r.slot = z * S + x;
     r.len = r.b >= 0 ? len_s[r.b] : 0;
     __syncthreads();                                            // out_s may be written again by a later call
     return r;

@@ -71,9 +71,9 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
     // guessed ahead of the dependency wait and settled after it (see the quantised kernel)
     const bool ranked = batch_is_ranked(a.batch);
     int* plan_scratch = reinterpret_cast<int*>(smem + SM::kStageOff);
-    BlockPlan bp{(int)blockIdx.z, (int)blockIdx.x, a.n_splits, (int)(blockIdx.x * a.batch + blockIdx.z), 0};
+    BlockPlan bp{(int)blockIdx.z, (int)blockIdx.x, a.n_splits, 0};
     if (a.wait_first) pdl_wait();
-    if (ranked) bp = plan_block(a, blockIdx.z, blockIdx.x, false, a.wait_first != 0, bp, plan_scratch);
+    if (ranked) bp = plan_block(plan_args(a), blockIdx.z, blockIdx.x, false, a.wait_first != 0, bp, plan_scratch);
     int b = bp.b;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * kStages * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * kStages * Stage::kBytes;
@@ -128,13 +128,13 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)bq * a.max_pages + (tile_g >> 1)];
         again = false;
         if (ranked && !a.wait_first) {
-            bp = plan_block(a, blockIdx.z, blockIdx.x, true, true, bp, plan_scratch);
+            bp = plan_block(plan_args(a), blockIdx.z, blockIdx.x, true, true, bp, plan_scratch);
             again = bp.b != bq && bp.b >= 0;
             if (bp.split != split_g || bp.n_splits != nsp_g) tile_g = -1;     // the hint was for other tiles
             b = bp.b;
         }
     } while (again);
-    if (b < 0) return;                                            // more blocks than (sequence, split) pairs
+    if (ranked && b < 0) return;                                  // more blocks than (sequence, split) pairs
     const int split = bp.split, n_splits = bp.n_splits;
 
     int len = ranked ? bp.len : a.seq_lens[b];
@@ -296,7 +296,8 @@ __global__ void __launch_bounds__(128, 3) decode_fp16_kernel(DecodeArgs a) {
         }
     }
     __syncthreads();
-    block_combine_and_store<D, GT>(a, red_s, bp.slot, h0);
+    const int slot = ranked ? blockIdx.z * a.n_splits + blockIdx.x : blockIdx.x * a.batch + blockIdx.z;
+    block_combine_and_store<D, GT>(a, red_s, slot, h0);
 }
 
 }  // namespace sa

@@ -105,10 +105,10 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
     // that its tests walk the repeat.
     const bool ranked = batch_is_ranked(a.batch);
     int* plan_scratch = reinterpret_cast<int*>(smem + SM::kStageOff);
-    BlockPlan bp{(int)blockIdx.z, (int)blockIdx.x, a.n_splits, (int)(blockIdx.x * a.batch + blockIdx.z), 0};
+    BlockPlan bp{(int)blockIdx.z, (int)blockIdx.x, a.n_splits, 0};
     if (a.wait_first) pdl_wait();
-    if (ranked)
-        bp = plan_block(a, LOST ? (blockIdx.z + 1) % a.batch : blockIdx.z, blockIdx.x, false, a.wait_first != 0, bp, plan_scratch);
+    if (__builtin_expect(ranked, 0))
+        bp = plan_block(plan_args(a), LOST ? (blockIdx.z + 1) % a.batch : blockIdx.z, blockIdx.x, false, a.wait_first != 0, bp, plan_scratch);
     int b = bp.b;
     const uint32_t mbar0 = smem_addr(smem + SM::kMbarOff) + warp * NS * 8;
     const uint32_t stage0 = smem_addr(smem + SM::kStageOff) + warp * NS * Stage::kBytes;
@@ -255,14 +255,15 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         // (one round trip instead of two when the guess holds, which it does unless the length crossed a tile boundary)
         if (lane == 0 && tile_g >= 0) pidx_g = a.page_table[(size_t)bq * a.max_pages + (tile_g >> 1)];
         again = false;
-        if (ranked && !a.wait_first) {                            // the plan that counts; wait_first made it after the wait already
-            bp = plan_block(a, blockIdx.z, blockIdx.x, true, true, bp, plan_scratch);
+        if (__builtin_expect(ranked && !a.wait_first, 0)) {       // the plan that counts; wait_first made it after the wait already
+            // (the test hook's guess was made for another block's coordinates: it never stands)
+            bp = plan_block(plan_args(a), blockIdx.z, blockIdx.x, !LOST, true, bp, plan_scratch);
             again = bp.b != bq && bp.b >= 0;
             if (bp.split != split_g || bp.n_splits != nsp_g) tile_g = -1;     // the hint was for other tiles
             b = bp.b;
         }
     } while (again);
-    if (b < 0) return;                                            // more blocks than (sequence, split) pairs
+    if (ranked && b < 0) return;                                  // more blocks than (sequence, split) pairs
     const int split = bp.split, n_splits = bp.n_splits;
 
     // ---- this warp's tiles; start the first copies ----
@@ -626,7 +627,9 @@ __global__ void __launch_bounds__((32 * DecodeSmem<D, KB, NIB, GT>::NW), (Decode
         }
         return;
     }
-    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, bp.slot, h0, failed);
+    // the block's slot among the partials (recomputed here rather than carried through the tile loop)
+    const int slot = ranked ? blockIdx.z * a.n_splits + blockIdx.x : blockIdx.x * a.batch + blockIdx.z;
+    block_merge_and_store<D, GT, NW>(a, red_s, M, l, acc, lane, warp, slot, h0, failed);
 }
 
 template <int D, int KB, bool NIB, int GT, int MODE>
