@@ -139,7 +139,10 @@ sa_status sa_get_layout(const sa_config* cfg, sa_layout* out);
 
 /* Bytes of scratch that sa_decode_attention / sa_decode_attention_fp16 need for a cache with
  * `batch` sequences of at most `max_pages_per_seq` pages (split-K partial results, section II-F:
- * the kernel grid has a split dimension).  Host only; the one CUDA call it may make reads the number of
+ * the kernel grid has a split dimension; for batches of 2 to 128 sequences also two words per sequence,
+ * in which the decode kernel tells the merge kernel how it dealt the grid's blocks to the sequences: in
+ * proportion to their cached lengths, so that a batch of unequal lengths keeps the machine as full as one
+ * of equal lengths).  Host only; the one CUDA call it may make reads the number of
  * multiprocessors of the CURRENT device (once per device), because the split count is planned for it: ask on
  * the device the decode calls will run on (without a device the figure of a B200 is used).  The scratch needs
  * no initialisation and may be shared by calls that do not overlap on the GPU. */
@@ -279,7 +282,8 @@ sa_status sa_decode_attention_fp16_stages(const sa_config* cfg, const sa_cache* 
  *     library's code is loaded on it until the process exits, whether or not this entry point is
  *     ever called.
  *   - The scratch bounds the problem: with S the split count the library picks for the cache
- *     shape, S * batch * n_q_heads * (head_dim + 2) * 4 bytes must fit.  A larger problem is
+ *     shape, S * batch * n_q_heads * (head_dim + 2) * 4 bytes (plus 8 bytes per sequence for batches of
+ *     2 to 128 sequences: exactly sa_workspace_bytes()) must fit.  A larger problem is
  *     refused with SA_ERR_CAPACITY and nothing is launched; use sa_decode_attention with a
  *     workspace of sa_workspace_bytes() for it.  (Batch 1, 32 query heads, head_dim 64 at any
  *     length fits; so does the ragged batch-16 configuration.)
