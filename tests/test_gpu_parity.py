@@ -789,6 +789,44 @@ def test_splits_dealt_by_length_for_extreme_mixes(dev, lens):
         assert np.max(np.abs(O[b] - ref)) <= TOL_O
 
 
+@pytest.mark.parametrize("lens", [[4000, 100, 2500, 100, 37], [640] * 6, [641, 650, 672, 655], [9000] + [1] * 30, [0, 0, 500]])
+def test_block_plan_left_for_the_merge_kernel(dev, lens):
+    """The words the decode kernel leaves behind the partials for the merge kernel ({first slot, splits} per
+    sequence) describe a sound deal of the grid's blocks: at least one split each, no more splits than blocks, the
+    sequences' slots back to back in the order longest first (ties by index), equal tile counts -> the host's split
+    count each in index order, and otherwise split counts that all come from one tiles-per-block."""
+    import torch
+    lens = np.asarray(lens)
+    B, Hq, d = len(lens), 8, 64
+    case = synth.make_case("plan", lens, Hq, 1, d, 4, seed=6400 + B)
+    cfg, cache = build_cache(case, dev)
+    O = torch.zeros((B, Hq, d), dtype=torch.float32, device=dev)
+    ws = cache.workspace
+    ws.view(torch.uint8).fill_(0xEE)
+    sa.decode_attention(cfg, cache.handle, t16(case.Q, dev), O, ws, None)
+    torch.cuda.synchronize()
+    need = sa.workspace_bytes(cfg, B, cache.max_pages)
+    plan_bytes = (B * 8 + 15) // 16 * 16
+    S, rem = divmod(need - plan_bytes, B * Hq * (d + 2) * 4)
+    assert rem == 0 and S >= 1
+    plan = ws.view(torch.uint8)[need - plan_bytes:need - plan_bytes + B * 8].cpu().numpy().view(np.int32).reshape(B, 2)
+    first, cnt = plan[:, 0].astype(np.int64), plan[:, 1].astype(np.int64)
+    tiles = (lens + 31) // 32
+    assert (cnt >= 1).all() and cnt.sum() <= S * B
+    if len(set(tiles.tolist())) == 1:
+        assert (cnt == S).all() and (first == np.arange(B) * S).all()
+    else:
+        order = sorted(range(B), key=lambda j: (-lens[j], j))
+        assert [first[j] for j in order] == np.concatenate([[0], np.cumsum(cnt[order])[:-1]]).tolist()
+        ok = [tpb for tpb in range(1, int(tiles.max()) + 2) if all(cnt[j] == max(1, -(-tiles[j] // tpb)) for j in range(B))]
+        assert ok, "split counts %s do not come from one tiles-per-block (tiles %s)" % (cnt, tiles)
+        # ... and the smallest tiles-per-block that fits the grid row was taken, or one close to it
+        fits = [tpb for tpb in range(1, int(tiles.max()) + 2) if sum(max(1, -(-t // tpb)) for t in tiles) <= S * B]
+        assert min(ok) <= fits[0] * 1.25 + 1
+    ref = ora.decode_attention(case.Q, case.K, case.V, case.cu_lens, 4, 10, n_threads=4)["O"]
+    assert np.max(np.abs(O.cpu().numpy() - ref)) <= TOL_O
+
+
 @pytest.mark.parametrize("fp16", [False, True])
 def test_rank_follows_lengths_rewritten_by_the_preceding_kernel(dev, fp16):
     """The decode kernels rank the sequences twice: ahead of their dependency wait (a guess, so that the query prologue
