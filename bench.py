@@ -911,6 +911,11 @@ def run_sweep(args):
     cell("cfg4 ragged B=16 [2048,16384] potm2", lens4, 32, 4, 64, 2)
     cell("cfg4 uniform B=16 T=%d potm2 (same mean length)" % int(lens4.mean()), [int(lens4.mean())] * 16, 32, 4, 64, 2, oracle=False)
     cell("cfg4 ragged B=16 [2048,16384] fp16", lens4, 32, 4, 64, 16)
+    for draw in ([] if quick else [2, 3]):          # other draws of the same distribution (other capacities, other split counts)
+        lens_d = np.random.Generator(np.random.PCG64(4000 + draw)).integers(2048, 16385, size=16)
+        cell("cfg4 ragged B=16 [2048,16384] potm2, draw %d" % draw, lens_d, 32, 4, 64, 2, oracle=False)
+        cell("cfg4 uniform B=16 T=%d potm2 (mean of draw %d)" % (int(lens_d.mean()), draw), [int(lens_d.mean())] * 16, 32, 4, 64, 2,
+             oracle=False)
     Ts = [1024, 16384] if quick else [1024, 4096, 16384, 65536, 131072]
     Bs = [1, 8] if quick else [1, 8, 32]
     for T in Ts:
