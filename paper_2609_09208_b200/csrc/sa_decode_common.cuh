@@ -95,10 +95,12 @@ SA_D BlockPlan plan_block(PlanArgs a, int z, int x, bool recheck, bool counts, B
     const bool writer = counts && a.plan != nullptr && z == 0 && x == 0 && blockIdx.y == 0;
     const int len_now = (j < B) ? __ldcg(a.seq_lens + j) : 0;
     if (recheck) {
+        // (the scratch is read before the barrier only: once the guess stands, the first copies may land on it)
+        const int pre_old = (writer && j < B) ? pre_s[j] : 0, cnt_old = (writer && j < B) ? cnt_s[j] : 0;
         if (!__syncthreads_or((j < B && len_now != len_s[j]) ? 1 : 0)) {
             if (writer && j < B) {
-                a.plan[2 * j] = pre_s[j];
-                a.plan[2 * j + 1] = cnt_s[j];
+                a.plan[2 * j] = pre_old;
+                a.plan[2 * j + 1] = cnt_old;
             }
             return prev;
         }

@@ -51,6 +51,7 @@ struct Fp16Smem {
     static constexpr int kMbarOff = 4 * kStages * Stage::kBytes;
     static constexpr int kBytes = kMbarOff + 128;
     static_assert(4 * GT * (D + 2) * 4 <= 4 * kStages * Stage::kBytes, "merge scratch must fit in the stage buffers");
+    static_assert(kPlanScratchInts * 4 <= 4 * kStages * Stage::kBytes, "the block plan's scratch must fit in the stage buffers");
 };
 
 template <int D, int GT>

@@ -63,6 +63,7 @@ struct DecodeSmem {
     static constexpr int kBlocksPerSM = decode_shape(D, KB).blocks_per_sm;
     static_assert(NW * GT * (D + 2) * 4 <= NW * NS * Stage::kBytes && NW * NS * 8 <= 256, "merge scratch must fit in the stage buffers");
     static_assert(Stage::kCodeBytes >= 32 * 8 * 4, "the weights of a tile must fit in its code area");
+    static_assert(NW * NS * Stage::kBytes >= kPlanScratchInts * 4, "the block plan's scratch must fit in the stage buffers");
     static_assert(Stage::kBytes == half_block_bytes(D, KB, NIB), "a stage buffer is a verbatim copy of half a page block");
 };
 
